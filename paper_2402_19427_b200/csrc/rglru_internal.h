@@ -1,0 +1,65 @@
+// Internal declarations shared by the translation units of the RG-LRU CUDA library.
+// Not part of the public ABI (that is include/rglru.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "rglru.h"
+
+namespace rglru {
+
+// The first 256 bytes of every workspace hold the device-side status: word 0 carries
+// STATUS_MAGIC | code once a kernel has recorded a condition.  A word without the magic
+// (fresh, uninitialised scratch) reads as "nothing recorded".
+constexpr uint32_t STATUS_MAGIC = 0x52474C00u;  // 'R','G','L', code in the low byte
+constexpr size_t WS_HEADER_BYTES = 256;
+
+struct FwdArgs {
+    int B, T, D, H;
+    float c;
+    const void *x;            // [B,T,D] io  (decode: [B,D])
+    const void *conv_w;       // [4,D] io
+    const float *conv_b;      // [D] or null
+    const void *W_a, *W_x;    // [H,Dh,Dh] io
+    const float *b_a, *b_x, *lambda;
+    const float *h0;          // [B,D] or null
+    const void *cs_in;        // [B,3,D] io or null
+    void *y;                  // [B,T,D] io
+    float *h_T;               // [B,D]
+    void *cs_out;             // [B,3,D] io
+    // optional fp32 saves for the backward, each [B,T,D] (null when not saving)
+    float *save_u, *save_r, *save_i, *save_hprev;
+    uint32_t *status;         // workspace header
+};
+
+struct BwdArgs {
+    int B, T, D, H;
+    float c;
+    const void *x, *conv_w, *W_a, *W_x, *cs_in, *dy;
+    const float *lambda;
+    void *dx;
+    float *dconv_w, *dconv_b, *dW_a, *db_a, *dW_x, *db_x, *dlambda;
+    // workspace arrays, each [B,T,D] fp32: u, r -> dz_a, i -> dz_x, hprev -> du
+    float *u, *r, *gi, *hp;
+    float *part_vec;   // [B][3][D]        partial sums of dlambda, db_a, db_x
+    float *part_conv;  // [B*nchunk][5][D] partial sums of dconv_w (4 rows) and dconv_b
+    float *part_dw;    // [S][2][H*Dh*Dh]  partial sums of dW_a, dW_x
+    int nchunk, S;
+};
+
+// ---- shape-generic CUDA-core kernels (any D_h <= GENERIC_MAX_DH, fp32 or bf16 io) ----
+constexpr int GENERIC_MAX_DH = 1024;
+constexpr int GENERIC_BWD_CHUNK = 64;  // tokens per thread in the conv backward
+size_t generic_backward_workspace_bytes(int B, int T, int D, int H);
+cudaError_t generic_prefill(const FwdArgs &a, int io, cudaStream_t st);
+cudaError_t generic_decode(const FwdArgs &a, int io, cudaStream_t st);
+cudaError_t generic_backward(const FwdArgs &fwd, BwdArgs &b, int io, void *ws_body, cudaStream_t st);
+
+// ---- sm_100a tensor-core kernels (bf16 io, D_h = 256) ----
+bool sm100_prefill_supported(int B, int T, int D, int H, int io);
+size_t sm100_prefill_workspace_bytes(int B, int T, int D, int H);
+cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes, cudaStream_t st);
+
+}  // namespace rglru

@@ -1,8 +1,649 @@
-// sm_100a tensor-core path (placeholder until the tcgen05 kernels land).
+// sm_100a fused prefill for the RG-LRU temporal core (bf16 io, head width 256).
+//
+// One persistent CTA per SM owns HALF a head (128 channels): its 2 x 128 rows of W_a and W_x stay
+// resident in tensor memory as the A operand of tcgen05.mma for the whole launch.  The CTA walks
+// tiles of 128 tokens:
+//   TMA warp       x rows of the whole head (the gates need all 256 input channels) -> shared memory
+//   conv warps     causal width-4 depthwise conv in fp32 -> bf16 tile U[128 tokens][256 ch] in the
+//                  K-major 128B-swizzled layout tcgen05.mma reads as its B operand
+//   MMA warp       Z_a^T = W_a U^T and Z_x^T = W_x U^T: channels on TMEM lanes, time along TMEM columns
+//   epilogue warps tcgen05.ld (time runs along registers, so the scan needs no shuffles), gates,
+//                  log-space decay, the linear recurrence in fp32, y written straight to HBM
+// x is read from HBM once per head (the two half-head CTAs share it through L2), y is written once;
+// u, r, i, a never leave the SM.
+//
+// Time is split across CTAs so that every SM has work even for a single long sequence: the S CTAs
+// of a half-head take its 128-token tiles round-robin.  A tile first folds itself to the aggregate
+// (prod a_t, h_end from zero state), publishes it, and obtains its incoming state from its own
+// previous tile plus the S-1 aggregates published by the other CTAs (decoupled look-back); only
+// then does it run the real scan and write y.  Waits on other CTAs are bounded and end in
+// RGLRU_ERR_TIMEOUT; the launch is cooperative so that all CTAs are co-resident.
+#include <cooperative_groups.h>
+#include <cuda_bf16.h>
+
+#include <atomic>
+#include <chrono>
+
 #include "rglru_internal.h"
 
 namespace rglru {
-bool sm100_prefill_supported(int, int, int, int, int) { return false; }
-size_t sm100_prefill_workspace_bytes(int, int, int, int) { return 0; }
-cudaError_t sm100_prefill(const FwdArgs &, void *, size_t, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int DH = 256;            // head width handled by this kernel
+constexpr int CH = 128;            // channels per CTA (half a head)
+constexpr int TILE_N = 128;        // tokens per MMA tile
+constexpr int SLAB = 32;           // tokens per TMA slab
+constexpr int SLAB_ROWS = SLAB + 3;
+constexpr int XS = 3;              // x slab ring depth
+constexpr int US = 2;              // U tile stages
+constexpr int NUM_THREADS = 512;
+constexpr int EPI_TOK = 64;        // tokens per epilogue warp
+constexpr int MAX_S = 8;           // at most this many CTAs share one half-head's time axis
+constexpr uint32_t U_STAGE_BYTES = TILE_N * DH * 2;       // 65536
+constexpr uint32_t U_KBLOCK_BYTES = TILE_N * 128;          // 16384: one 64-channel K block
+constexpr uint32_t X_ROW_BYTES = DH * 2;                   // 512
+constexpr uint32_t X_SLAB_BYTES = SLAB_ROWS * X_ROW_BYTES; // 17920
+constexpr uint32_t SMEM_U = 0;
+constexpr uint32_t SMEM_X = SMEM_U + US * U_STAGE_BYTES;
+constexpr uint32_t SMEM_H = SMEM_X + XS * X_SLAB_BYTES;    // float h_s[4][2][32]
+constexpr uint32_t SMEM_AGG = SMEM_H + 4 * 2 * 32 * 4;
+constexpr uint32_t SMEM_BAR = SMEM_AGG + 2 * 4 * 32 * 8; // float2 agg_s[2][4][32], indexed by tile parity
+constexpr int NUM_BARS = 2 * XS + 2 * US + 2 + 8 + 4;
+constexpr uint32_t SMEM_MISC = SMEM_BAR + NUM_BARS * 8;    // tmem base, abort flag
+constexpr uint32_t SMEM_TOTAL = SMEM_MISC + 16;
+constexpr uint32_t SMEM_ALLOC = SMEM_TOTAL + 1024;         // slack for 1024-byte alignment
+
+// TMEM columns
+constexpr uint32_t TM_ACC_A = 0, TM_ACC_X = 128, TM_W_A = 256, TM_W_X = 384;
+
+// Channels whose decay rate s = c*softplus(-Lambda) is at most S_POLY evaluate exp on the FMA pipe.
+constexpr float S_POLY = 0.25f;
+
+struct Sm100Args {
+    FwdArgs f;
+    int S;             // CTAs per half-head (time split factor)
+    int tps;           // tiles per sequence
+    int tiles_total;   // B * tps
+    uint32_t tag;      // validity tag of this call's aggregate records
+    uint4 *agg;        // [H*2][tiles_total][128] records {P, tag, h_loc, tag}
+    unsigned long long spin_ns;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint64_t gtimer() { uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the limit ran out or the CTA is aborting.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
+    if (mbar_try(bar, parity)) return true;
+    const uint64_t t0 = gtimer();
+    while (!mbar_try(bar, parity)) {
+        if (*abort_flag) return false;
+        if (gtimer() - t0 > limit_ns) return false;
+    }
+    return true;
+}
+// All lanes wait; the verdict is made warp-uniform so that a warp never splits on a timeout.
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, limit_ns, abort_flag));
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]^T, kind::f16 (bf16 inputs, fp32 accumulate), one CTA
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
+    uint32_t r[32];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+                   "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]),
+                   "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]),
+                   "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, uint4 lo, uint4 hi) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"r"(taddr), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
+// K-major, 128B-swizzled shared-memory operand: rows of 128 B, 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t make_desc_sw128(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+           ((uint64_t)2 << 61);
+}
+// kind::f16 instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M x N
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// ---- packed fp32x2 arithmetic (one issue slot for two lanes' worth of FP32 work)
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) { return ((f32x2)__float_as_uint(hi) << 32) | __float_as_uint(lo); }
+__device__ __forceinline__ float lo2(f32x2 v) { return __uint_as_float((uint32_t)v); }
+__device__ __forceinline__ float hi2(f32x2 v) { return __uint_as_float((uint32_t)(v >> 32)); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ float tanh_approx(float x) { float y; asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float sqrt_approx(float x) { float y; asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float ex2_approx(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+
+__device__ __forceinline__ void record_timeout(uint32_t *status, volatile int *abort_flag) {
+    *abort_flag = 1;
+    atomicExch(status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
+}
+
+// (z_a, z_x) of two consecutive tokens of one channel -> (a_t, v_t) of Eq. 3-4, in place.
+//   r = sigmoid(z_a + b_a) = 1/2 + 1/2 tanh((z_a + b_a)/2),  x = 2 s r,  f = 1 - a_t = -expm1(-x/2),
+//   m/2 = sqrt(f (1/2 - f/4)) = sqrt(1 - a_t^2)/2,  v = (m/2 u)(1 + tanh((z_x + b_x)/2)) = m i u.
+template <bool POLY>
+__device__ __forceinline__ void gate_pair(float &za0, float &za1, float &zx0, float &zx1, float u0, float u1, f32x2 hba2, f32x2 hbx2,
+                                          f32x2 s2) {
+    const f32x2 HALF2 = pack2(0.5f, 0.5f);
+    f32x2 ta = fma2(pack2(za0, za1), HALF2, hba2);
+    ta = pack2(tanh_approx(lo2(ta)), tanh_approx(hi2(ta)));
+    const f32x2 x = fma2(ta, s2, s2);
+    f32x2 f, a;
+    if (POLY) {
+        // f = x/2 - x^2/8 + x^3/48 - x^4/384  (|x| <= 2 S_POLY: relative truncation error < 4e-5)
+        f32x2 p = fma2(x, pack2(-1.0f / 384.0f, -1.0f / 384.0f), pack2(1.0f / 48.0f, 1.0f / 48.0f));
+        p = fma2(p, x, pack2(-0.125f, -0.125f));
+        p = fma2(p, x, HALF2);
+        f = mul2(p, x);
+        a = fma2(f, pack2(-1.0f, -1.0f), pack2(1.0f, 1.0f));
+    } else {
+        const f32x2 e = mul2(x, pack2(-0.72134752f, -0.72134752f));  // -x/2 * log2(e)
+        a = pack2(ex2_approx(lo2(e)), ex2_approx(hi2(e)));
+        f = fma2(a, pack2(-1.0f, -1.0f), pack2(1.0f, 1.0f));
+    }
+    f32x2 q = mul2(f, fma2(f, pack2(-0.25f, -0.25f), HALF2));  // (1 - a^2)/4 = f (2 - f)/4
+    if (!POLY) q = pack2(fmaxf(lo2(q), 0.0f), fmaxf(hi2(q), 0.0f));  // a from ex2.approx may round above 1
+    const f32x2 mh = pack2(sqrt_approx(lo2(q)), sqrt_approx(hi2(q)));
+    f32x2 tx = fma2(pack2(zx0, zx1), HALF2, hbx2);
+    tx = pack2(tanh_approx(lo2(tx)), tanh_approx(hi2(tx)));
+    const f32x2 g = mul2(mh, pack2(u0, u1));
+    const f32x2 v = fma2(g, tx, g);
+    za0 = lo2(a); za1 = hi2(a);
+    zx0 = lo2(v); zx1 = hi2(v);
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __grid_constant__ Sm100Args p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (base - raw_addr);
+    const uint32_t bar0 = base + SMEM_BAR;
+    // barrier indices
+    auto BAR_XFULL = [&](int s) { return bar0 + 8u * s; };
+    auto BAR_XEMPTY = [&](int s) { return bar0 + 8u * (XS + s); };
+    auto BAR_UFULL = [&](int s) { return bar0 + 8u * (2 * XS + s); };
+    auto BAR_UEMPTY = [&](int s) { return bar0 + 8u * (2 * XS + US + s); };
+    const uint32_t BAR_ACCFULL = bar0 + 8u * (2 * XS + 2 * US);
+    const uint32_t BAR_ACCEMPTY = BAR_ACCFULL + 8u;
+    auto BAR_CHAIN = [&](int q, int k) { return BAR_ACCEMPTY + 8u + 8u * (q * 2 + k); };
+    auto BAR_AGG = [&](int q) { return BAR_ACCEMPTY + 8u + 8u * (8 + q); };
+    uint32_t *tmem_base_s = (uint32_t *)(smem + SMEM_MISC);
+    volatile int *abort_flag = (volatile int *)(smem + SMEM_MISC + 4);
+    float *h_s = (float *)(smem + SMEM_H);
+    float2 *agg_s = (float2 *)(smem + SMEM_AGG);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const FwdArgs &f = p.f;
+    const int T = f.T, D = f.D, S = p.S;
+    const int group = blockIdx.x / S, kcta = blockIdx.x % S;  // group = head * 2 + half
+    const int head = group >> 1, half = group & 1;
+    const int n_my_tiles = (p.tiles_total - kcta + S - 1) / S;
+    const unsigned long long spin = p.spin_ns;
+
+    if (tid == 0) {
+        for (int s = 0; s < XS; ++s) { mbar_init(BAR_XFULL(s), 1); mbar_init(BAR_XEMPTY(s), 4); }
+        for (int s = 0; s < US; ++s) { mbar_init(BAR_UFULL(s), 4); mbar_init(BAR_UEMPTY(s), 9); }
+        mbar_init(BAR_ACCFULL, 1);
+        mbar_init(BAR_ACCEMPTY, 8);
+        for (int q = 0; q < 4; ++q) { mbar_init(BAR_CHAIN(q, 0), 1); mbar_init(BAR_CHAIN(q, 1), 1); mbar_init(BAR_AGG(q), 1); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 5) { tmem_alloc(smem_u32(tmem_base_s), 512); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_base_s;
+
+    // Gate weights of this half-head into tensor memory: lane = output channel, 32-bit column j holds
+    // input channels 2j (low half) and 2j+1 (high half), i.e. consecutive bf16 of the row as stored.
+    if (warp >= 8) {
+        const int q = warp & 3, g = (warp - 8) >> 2;  // g = 0: W_a, 1: W_x
+        const __nv_bfloat16 *W = (const __nv_bfloat16 *)(g ? f.W_x : f.W_a);
+        const uint4 *row = (const uint4 *)(W + ((size_t)head * DH + half * CH + q * 32 + lane) * DH);
+        const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (g ? TM_W_X : TM_W_A);
+#pragma unroll 4
+        for (int c = 0; c < 16; ++c) tmem_st8(taddr + c * 8, __ldg(row + 2 * c), __ldg(row + 2 * c + 1));
+        tmem_st_wait();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    if (warp < 4) {
+        // ================================================================ conv producers
+        reg_dec<72>();
+        const int pblk = warp;                       // K block = 64 channels of the head
+        const int l16 = lane & 15, tg = lane >> 4;   // 4-channel chunk, token group of 16
+        const int hc = pblk * 64 + l16 * 4;          // channel within the head
+        const __nv_bfloat16 *cw = (const __nv_bfloat16 *)f.conv_w;
+        f32x2 w01[4], w23[4], b01, b23;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const __nv_bfloat16 *wp = cw + (size_t)j * D + head * DH + hc;
+            w01[j] = pack2(__bfloat162float(wp[0]), __bfloat162float(wp[1]));
+            w23[j] = pack2(__bfloat162float(wp[2]), __bfloat162float(wp[3]));
+        }
+        if (f.conv_b) {
+            const float *bp = f.conv_b + head * DH + hc;
+            b01 = pack2(bp[0], bp[1]); b23 = pack2(bp[2], bp[3]);
+        } else { b01 = pack2(0.f, 0.f); b23 = b01; }
+        const uint32_t x_thread_off = (uint32_t)hc * 2;
+        const uint32_t u_chunk = (uint32_t)(l16 >> 1), u_half = (uint32_t)(l16 & 1) * 8;
+        int slab_n = 0;
+        bool ok = true;
+        for (int it = 0; it < n_my_tiles && ok; ++it) {
+            const int g = kcta + it * S, ti = g % p.tps;
+            const int t0 = ti * TILE_N;
+            const int st = it % US;
+            ok = warp_wait(BAR_UEMPTY(st), ((it / US) & 1) ^ 1, spin, abort_flag);
+            if (!ok) break;
+            const uint32_t u_base = base + SMEM_U + st * U_STAGE_BYTES + pblk * U_KBLOCK_BYTES;
+            const int nslab = min(TILE_N / SLAB, (T - t0 + SLAB - 1) / SLAB);
+            for (int s = 0; s < nslab; ++s, ++slab_n) {
+                const int slot = slab_n % XS;
+                ok = warp_wait(BAR_XFULL(slot), (slab_n / XS) & 1, spin, abort_flag);
+                if (!ok) break;
+                const int ts0 = t0 + s * SLAB;
+                const bool zero_halo = (ts0 == 0) && (f.cs_in == nullptr);
+                const int nvalid = min(SLAB, T - ts0) - tg * 16;  // tokens of this thread's group that exist
+                const uint8_t *xs = smem + SMEM_X + slot * X_SLAB_BYTES + x_thread_off;
+                auto load_row = [&](int r, f32x2 &v01, f32x2 &v23) {
+                    uint2 w = *(const uint2 *)(xs + r * X_ROW_BYTES);
+                    if (zero_halo && r < 3) { w.x = 0u; w.y = 0u; }
+                    v01 = pack2(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xFFFF0000u));
+                    v23 = pack2(__uint_as_float(w.y << 16), __uint_as_float(w.y & 0xFFFF0000u));
+                };
+                if (nvalid > 0) {
+                    const int r0 = tg * 16;
+                    f32x2 a01, a23, b01x, b23x, c01, c23;  // x_{t-3}, x_{t-2}, x_{t-1}
+                    load_row(r0, a01, a23); load_row(r0 + 1, b01x, b23x); load_row(r0 + 2, c01, c23);
+#pragma unroll 4
+                    for (int i = 0; i < 16; ++i) {
+                        if (i < nvalid) {
+                            f32x2 d01, d23;
+                            load_row(r0 + 3 + i, d01, d23);
+                            f32x2 u01 = fma2(w01[0], d01, b01), u23 = fma2(w23[0], d23, b23);
+                            u01 = fma2(w01[1], c01, u01); u23 = fma2(w23[1], c23, u23);
+                            u01 = fma2(w01[2], b01x, u01); u23 = fma2(w23[2], b23x, u23);
+                            u01 = fma2(w01[3], a01, u01); u23 = fma2(w23[3], a23, u23);
+                            __nv_bfloat162 o01 = __floats2bfloat162_rn(lo2(u01), hi2(u01));
+                            __nv_bfloat162 o23 = __floats2bfloat162_rn(lo2(u23), hi2(u23));
+                            const int row = s * SLAB + r0 + i;
+                            const uint32_t off = (uint32_t)row * 128u + ((u_chunk ^ (uint32_t)(row & 7)) << 4) + u_half;
+                            uint2 o;
+                            o.x = *(uint32_t *)&o01; o.y = *(uint32_t *)&o23;
+                            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(u_base + off), "r"(o.x), "r"(o.y) : "memory");
+                            a01 = b01x; a23 = b23x; b01x = c01; b23x = c23; c01 = d01; c23 = d23;
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(BAR_XEMPTY(slot));
+            }
+            if (!ok) break;
+            fence_async_smem();  // make the generic-proxy writes of U visible to the tensor core
+            __syncwarp();
+            if (lane == 0) mbar_arrive(BAR_UFULL(st));
+        }
+        if (!ok && lane == 0) record_timeout(f.status, abort_flag);
+    } else if (warp == 4) {
+        // ================================================================ TMA loader
+        reg_dec<24>();
+        const __nv_bfloat16 *x = (const __nv_bfloat16 *)f.x;
+        const __nv_bfloat16 *cs_in = (const __nv_bfloat16 *)f.cs_in;
+        int slab_n = 0;
+        bool ok = true;
+        for (int it = 0; it < n_my_tiles && ok; ++it) {
+            const int g = kcta + it * S, b = g / p.tps, ti = g % p.tps;
+            const int t0 = ti * TILE_N;
+            const int nslab = min(TILE_N / SLAB, (T - t0 + SLAB - 1) / SLAB);
+            for (int s = 0; s < nslab; ++s, ++slab_n) {
+                const int slot = slab_n % XS;
+                ok = warp_wait(BAR_XEMPTY(slot), ((slab_n / XS) & 1) ^ 1, spin, abort_flag);
+                if (!ok) break;
+                const int ts0 = t0 + s * SLAB;
+                const int lo_row = (ts0 == 0 && cs_in == nullptr) ? 3 : 0;   // rows with no source stay untouched
+                const int hi_row = min(SLAB_ROWS, T - ts0 + 3);
+                if (lane == 0) mbar_expect_tx(BAR_XFULL(slot), (uint32_t)(hi_row - lo_row) * X_ROW_BYTES);
+                __syncwarp();
+                for (int r = lane; r < SLAB_ROWS; r += 32) {
+                    if (r < lo_row || r >= hi_row) continue;
+                    const int t = ts0 - 3 + r;
+                    const __nv_bfloat16 *src = t >= 0 ? x + ((size_t)b * T + t) * D + head * DH
+                                                      : cs_in + ((size_t)b * 3 + (3 + t)) * D + head * DH;
+                    bulk_g2s(base + SMEM_X + slot * X_SLAB_BYTES + r * X_ROW_BYTES, src, X_ROW_BYTES, BAR_XFULL(slot));
+                }
+            }
+        }
+        if (!ok && lane == 0) record_timeout(f.status, abort_flag);
+    } else if (warp == 5) {
+        // ================================================================ MMA issuer
+        reg_dec<24>();
+        constexpr uint32_t idesc = make_idesc(128, TILE_N);
+        bool ok = true;
+        if (lane == 0) {
+            for (int it = 0; it < n_my_tiles; ++it) {
+                const int st = it % US;
+                ok = mbar_wait(BAR_UFULL(st), (it / US) & 1, spin, abort_flag);
+                if (!ok) break;
+                ok = mbar_wait(BAR_ACCEMPTY, (it & 1) ^ 1, spin, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t u_base = base + SMEM_U + st * U_STAGE_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < DH / 16; ++ks) {
+                    const uint64_t bd = make_desc_sw128(u_base + (ks >> 2) * U_KBLOCK_BYTES + (ks & 3) * 32);
+                    mma_ts(tmem + TM_ACC_A, tmem + TM_W_A + ks * 8, bd, idesc, ks > 0);
+                    mma_ts(tmem + TM_ACC_X, tmem + TM_W_X + ks * 8, bd, idesc, ks > 0);
+                }
+                tc_commit(BAR_UEMPTY(st));
+                tc_commit(BAR_ACCFULL);
+            }
+            if (!ok) record_timeout(f.status, abort_flag);
+        }
+        __syncwarp();
+    } else if (warp >= 8) {
+        // ================================================================ epilogue
+        reg_inc<208>();
+        const int q = warp & 3, k = (warp - 8) >> 2;
+        const int c_own = q * 32 + lane;                 // channel within the CTA
+        const int hc = half * CH + c_own;                // channel within the head
+        const int d = head * DH + hc;                    // global channel
+        // per-channel constants; s = c softplus(-Lambda) with libm-grade log1p/exp (Appendix A)
+        const float lam = f.lambda[d];
+        const float zl = -lam;
+        const float s = f.c * (zl > 0.0f ? zl + log1pf(expf(-zl)) : log1pf(expf(zl)));
+        const f32x2 s2 = pack2(s, s);
+        const f32x2 hba2 = pack2(0.5f * f.b_a[d], 0.5f * f.b_a[d]), hbx2 = pack2(0.5f * f.b_x[d], 0.5f * f.b_x[d]);
+        const bool poly = __all_sync(0xffffffffu, s <= S_POLY);
+        // u[token][channel] in the swizzled U tile: 8 row phases
+        uint32_t u_off[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            u_off[j] = (uint32_t)(hc >> 6) * U_KBLOCK_BYTES + ((((uint32_t)(hc & 63) >> 3) ^ (uint32_t)j) << 4) + (uint32_t)(hc & 7) * 2 +
+                       (uint32_t)(k * EPI_TOK) * 128u;
+        const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16);
+        __nv_bfloat16 *y = (__nv_bfloat16 *)f.y;
+        const __nv_bfloat16 *x = (const __nv_bfloat16 *)f.x;
+        const __nv_bfloat16 *cs_in = (const __nv_bfloat16 *)f.cs_in;
+        float h_prev_own = 0.0f;  // warp 0: state after this CTA's previous tile
+        bool ok = true;
+        for (int it = 0; it < n_my_tiles && ok; ++it) {
+            const int g = kcta + it * S, b = g / p.tps, ti = g % p.tps;
+            const int t0 = ti * TILE_N;
+            const int st = it % US;
+            const int nv = max(0, min(EPI_TOK, T - t0 - k * EPI_TOK));  // valid tokens of this warp
+            ok = warp_wait(BAR_ACCFULL, it & 1, spin, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            float za[EPI_TOK], zx[EPI_TOK];
+            tmem_ld32(tm_lane + TM_ACC_A + k * EPI_TOK, za);
+            tmem_ld32(tm_lane + TM_ACC_A + k * EPI_TOK + 32, za + 32);
+            tmem_ld32(tm_lane + TM_ACC_X + k * EPI_TOK, zx);
+            tmem_ld32(tm_lane + TM_ACC_X + k * EPI_TOK + 32, zx + 32);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(BAR_ACCEMPTY);  // the accumulators now live in registers
+            // gates, decay, input scale: (z_a, z_x) -> (a_t, v_t) in place
+            const uint32_t u_base = base + SMEM_U + st * U_STAGE_BYTES;
+#pragma unroll
+            for (int i = 0; i < EPI_TOK; i += 2) {
+                uint16_t ub0, ub1;
+                asm volatile("ld.shared.u16 %0, [%1];" : "=h"(ub0) : "r"(u_base + u_off[i & 7] + (uint32_t)i * 128u));
+                asm volatile("ld.shared.u16 %0, [%1];" : "=h"(ub1) : "r"(u_base + u_off[(i + 1) & 7] + (uint32_t)(i + 1) * 128u));
+                const float u0 = __uint_as_float((uint32_t)ub0 << 16), u1 = __uint_as_float((uint32_t)ub1 << 16);
+                if (poly) gate_pair<true>(za[i], za[i + 1], zx[i], zx[i + 1], u0, u1, hba2, hbx2, s2);
+                else gate_pair<false>(za[i], za[i + 1], zx[i], zx[i + 1], u0, u1, hba2, hbx2, s2);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(BAR_UEMPTY(st));  // done reading u
+            // ---- incoming state
+            float h;
+            if (S > 1) {
+                // fold this warp's tokens to (P, h_loc): h_out = P h_in + h_loc
+                float P = 1.0f, hl = 0.0f;
+#pragma unroll
+                for (int i = 0; i < EPI_TOK; ++i)
+                    if (i < nv) { P *= za[i]; hl = fmaf(za[i], hl, zx[i]); }
+                if (k == 0) {
+                    agg_s[((it & 1) * 4 + q) * 32 + lane] = make_float2(P, hl);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(BAR_AGG(q));
+                } else {
+                    ok = warp_wait(BAR_AGG(q), it & 1, spin, abort_flag);
+                    if (!ok) break;
+                    const float2 a0 = agg_s[((it & 1) * 4 + q) * 32 + lane];
+                    const float Pt = P * a0.x, hlt = fmaf(P, a0.y, hl);
+                    uint4 rec;
+                    rec.x = __float_as_uint(Pt); rec.y = p.tag; rec.z = __float_as_uint(hlt); rec.w = p.tag;
+                    uint4 *dst = p.agg + ((size_t)group * p.tiles_total + g) * CH + c_own;
+                    asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "r"(rec.x), "r"(rec.y), "r"(rec.z), "r"(rec.w) : "memory");
+                }
+            }
+            if (k == 0) {
+                if (it > 0) {  // state after this CTA's previous tile (written by warp 1)
+                    ok = warp_wait(BAR_CHAIN(q, 0), (it - 1) & 1, spin, abort_flag);
+                    if (!ok) break;
+                    h_prev_own = h_s[(q * 2 + 0) * 32 + lane];
+                }
+                int nback;
+                if (ti == 0 || (S > 1 && ti < S)) {
+                    h = f.h0 ? f.h0[(size_t)b * D + d] : 0.0f;
+                    nback = ti;
+                } else {
+                    h = h_prev_own;
+                    nback = S - 1;
+                }
+                // decoupled look-back: the aggregates of the (at most MAX_S - 1) tiles between that state and
+                // this tile.  All records are requested at once, then polled until every lane sees this
+                // call's tag in both halves of each record (8-byte words are written atomically).
+                if (nback > 0) {
+                    const uint4 *src = p.agg + ((size_t)group * p.tiles_total + g) * CH + c_own;
+                    uint4 rec[MAX_S - 1];
+                    const uint64_t tstart = gtimer();
+                    for (;;) {
+                        bool ready = true;
+#pragma unroll
+                        for (int j = 1; j < MAX_S; ++j) {
+                            if (j <= nback) {
+                                const uint4 *sj = src - (size_t)j * CH;
+                                asm volatile("ld.volatile.global.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                             : "=r"(rec[j - 1].x), "=r"(rec[j - 1].y), "=r"(rec[j - 1].z), "=r"(rec[j - 1].w) : "l"(sj) : "memory");
+                            }
+                        }
+#pragma unroll
+                        for (int j = 1; j < MAX_S; ++j)
+                            if (j <= nback) ready = ready && rec[j - 1].y == p.tag && rec[j - 1].w == p.tag;
+                        if (__all_sync(0xffffffffu, ready)) break;
+                        if (*abort_flag || gtimer() - tstart > spin) { ok = false; break; }
+                        __nanosleep(100);
+                    }
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (ok) {
+#pragma unroll
+                        for (int j = MAX_S - 1; j >= 1; --j)
+                            if (j <= nback) h = fmaf(__uint_as_float(rec[j - 1].x), h, __uint_as_float(rec[j - 1].z));
+                    }
+                }
+                if (!ok) break;
+            } else {
+                ok = warp_wait(BAR_CHAIN(q, 1), it & 1, spin, abort_flag);
+                if (!ok) break;
+                h = h_s[(q * 2 + 1) * 32 + lane];
+            }
+            // ---- the recurrence h_t = a_t h_{t-1} + v_t (Eq. 4) and y_t = h_t
+            __nv_bfloat16 *yp = y + ((size_t)b * T + t0 + k * EPI_TOK) * D + d;
+            if (nv == EPI_TOK) {
+#pragma unroll
+                for (int i = 0; i < EPI_TOK; i += 2) {
+                    const float h0v = fmaf(za[i], h, zx[i]);
+                    h = fmaf(za[i + 1], h0v, zx[i + 1]);
+                    const __nv_bfloat162 o = __floats2bfloat162_rn(h0v, h);
+                    yp[(size_t)i * D] = o.x;
+                    yp[(size_t)(i + 1) * D] = o.y;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < EPI_TOK; ++i) {
+                    if (i < nv) {
+                        h = fmaf(za[i], h, zx[i]);
+                        yp[(size_t)i * D] = __float2bfloat16_rn(h);
+                    }
+                }
+            }
+            // ---- hand the state on
+            h_s[(q * 2 + (k ^ 1)) * 32 + lane] = h;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(BAR_CHAIN(q, k ^ 1));
+            if (k == 1 && ti == p.tps - 1) {
+                // end of a sequence: h_T (unrounded state) and the last three raw inputs, bit-exact
+                f.h_T[(size_t)b * D + d] = h;
+                __nv_bfloat16 keep[3];
+#pragma unroll
+                for (int kk = 0; kk < 3; ++kk) {
+                    const int t = T - 3 + kk;
+                    keep[kk] = t >= 0 ? x[((size_t)b * T + t) * D + d]
+                                      : (cs_in ? cs_in[((size_t)b * 3 + (3 + t)) * D + d] : __float2bfloat16_rn(0.0f));
+                }
+                __nv_bfloat16 *cs_out = (__nv_bfloat16 *)f.cs_out;
+#pragma unroll
+                for (int kk = 0; kk < 3; ++kk) cs_out[((size_t)b * 3 + kk) * D + d] = keep[kk];
+            }
+        }
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok && lane == 0) record_timeout(f.status, abort_flag);
+    } else {
+        reg_dec<24>();
+    }
+
+    // ---- teardown: every role falls through to here, also after a timeout
+    if (*abort_flag) {
+        // let copies and MMAs in flight land before shared and tensor memory are given back
+        const uint64_t tw = gtimer();
+        while (gtimer() - tw < 50000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) tmem_dealloc(tmem, 512);
+}
+
+int num_sms() {
+    static int cached = 0;
+    if (cached == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+            cached = n;
+        else
+            return 148;
+    }
+    return cached;
+}
+
+std::atomic<uint32_t> g_call_counter{0};
+
+uint32_t next_tag() {
+    static const uint32_t salt = (uint32_t)std::chrono::steady_clock::now().time_since_epoch().count() * 2654435761u;
+    uint32_t t = salt + 0x9E3779B9u * (g_call_counter.fetch_add(1) + 1u);
+    return t == 0 ? 1u : t;
+}
+
+}  // namespace
+
+unsigned long long g_spin_limit_ns = 2000000000ull;  // bounded waits give up after this long
+
+bool sm100_prefill_supported(int B, int T, int D, int H, int io) {
+    return io == RGLRU_BF16 && B > 0 && T > 0 && H > 0 && D == H * DH;
+}
+
+size_t sm100_prefill_workspace_bytes(int B, int T, int D, int H) {
+    const size_t tps = (T + TILE_N - 1) / TILE_N;
+    return (size_t)H * 2 * B * tps * CH * sizeof(uint4);
+}
+
+cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes, cudaStream_t st) {
+    static bool attr_set = false;
+    cudaError_t e;
+    if (!attr_set) {
+        e = cudaFuncSetAttribute(sm100_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    Sm100Args p;
+    p.f = a;
+    p.tps = (a.T + TILE_N - 1) / TILE_N;
+    p.tiles_total = a.B * p.tps;
+    const int groups = a.H * 2;
+    const int nsm = num_sms();
+    int S = nsm / groups;
+    if (S < 1) S = 1;
+    if (S > MAX_S) S = MAX_S;
+    if (S > p.tiles_total) S = p.tiles_total;
+    p.S = S;
+    p.tag = next_tag();
+    p.agg = (uint4 *)ws_body;
+    p.spin_ns = g_spin_limit_ns;
+    if (ws_body_bytes < sm100_prefill_workspace_bytes(a.B, a.T, a.D, a.H)) return cudaErrorInvalidValue;
+    dim3 grid(groups * S), block(NUM_THREADS);
+    if (S > 1) {
+        // CTAs wait on one another's aggregates: they must all be resident
+        void *args[] = {(void *)&p};
+        return cudaLaunchCooperativeKernel((const void *)sm100_prefill_kernel, grid, block, args, SMEM_ALLOC, st);
+    }
+    sm100_prefill_kernel<<<grid, block, SMEM_ALLOC, st>>>(p);
+    return cudaGetLastError();
+}
+
 }  // namespace rglru

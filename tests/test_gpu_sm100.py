@@ -1,0 +1,92 @@
+"""GPU parity of the tcgen05 fused prefill (bf16 io, head width 256) against the fp64 oracle, through the C ABI.
+Covers ragged tails, T < 3, incoming state, several heads, the cross-CTA carry of the time split, long-memory
+channels, channels outside the polynomial-exp range, and sampled heads of the full-size workloads."""
+import numpy as np
+import pytest
+
+from paper_2402_19427_b200 import inputs as synth
+from util import assert_close, f64, gpu_prefill, oracle_prefill, to_dev, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+def uses_sm100(B, T, D, H):
+    from paper_2402_19427_b200 import binding
+    import torch
+    return binding.workspace_bytes(binding.make_shape(B, T, D, H, torch.bfloat16), binding.OP_PREFILL) > 256
+
+
+@pytest.mark.parametrize("B,T,H", [(1, 1, 1), (2, 2, 1), (1, 3, 2), (1, 31, 1), (2, 64, 1), (1, 65, 1), (1, 128, 2), (3, 129, 1),
+                                   (2, 320, 2), (1, 1000, 1), (5, 257, 3)])
+def test_shapes_with_state_and_bias(oracle, B, T, H):
+    D = 256 * H
+    assert uses_sm100(B, T, D, H)
+    inp = synth.make_inputs(B, T, D, H, io="bf16", seed=500 + T, with_state=True, bias_scale=0.5)
+    y, hT, cso = gpu_prefill(inp, h0=inp["h0"], cs=inp["conv_state"])
+    yr, hr, cr = oracle_prefill(oracle, inp, h0=inp["h0"].astype(np.float64), cs=inp["conv_state"].astype(np.float64))
+    assert_close("y", y, yr, "bf16"); assert_close("h_T", hT, hr, "bf16")
+    assert np.array_equal(cso, cr)
+
+
+def test_zero_state_defaults_and_generic_agreement(oracle):
+    inp = synth.make_inputs(2, 200, 512, 2, io="bf16", seed=3)
+    y, hT, cso = gpu_prefill(inp)
+    yg, hg, cg = gpu_prefill(inp, flags=1)
+    yr, hr, cr = oracle_prefill(oracle, inp)
+    assert_close("y", y, yr, "bf16"); assert_close("h_T", hT, hr, "bf16")
+    assert_close("y generic", yg, yr, "bf16")
+    assert np.array_equal(cso, cr) and np.array_equal(cg, cr)
+
+
+def test_long_sequence_cross_cta_carry_and_long_memory(oracle):
+    """One sequence of 40 tiles on two half-head groups: every tile's state arrives through the look-back;
+    5 % of the channels have a^c = 0.9999 so the carry matters over thousands of tokens."""
+    inp = synth.make_inputs(1, 5000, 256, 1, io="bf16", seed=9, long_memory_frac=0.05, with_state=True)
+    y, hT, cso = gpu_prefill(inp, h0=inp["h0"], cs=inp["conv_state"])
+    yr, hr, cr = oracle_prefill(oracle, inp, h0=inp["h0"].astype(np.float64), cs=inp["conv_state"].astype(np.float64))
+    assert_close("y", y, yr, "bf16"); assert_close("h_T", hT, hr, "bf16")
+    assert np.array_equal(cso, cr)
+
+
+def test_wide_lambda_range_uses_exp_path(oracle):
+    """Lambda down to -3 (a = 0.047): decay rates far outside the polynomial range; and up to 16 (a^c ~ 1 - 1e-6)."""
+    inp = synth.make_inputs(2, 300, 256, 1, io="bf16", seed=21, bias_scale=0.3)
+    rng = np.random.default_rng(1)
+    inp["params"]["lam"] = rng.uniform(-3.0, 16.0, size=256).astype(np.float32)
+    y, hT, _ = gpu_prefill(inp)
+    yr, hr, _ = oracle_prefill(oracle, inp)
+    assert_close("y", y, yr, "bf16"); assert_close("h_T", hT, hr, "bf16")
+
+
+def test_split_prefill_and_aliased_state(oracle):
+    import torch
+    from paper_2402_19427_b200 import binding
+    inp = synth.make_inputs(2, 700, 512, 2, io="bf16", seed=17, with_state=True)
+    params = binding.Params.from_numpy(inp["params"], "bf16")
+    x = to_dev(inp["x"], "bf16")
+    h = to_dev(inp["h0"]); cs = to_dev(inp["conv_state"], "bf16")
+    y1, _, _ = binding.prefill(x[:, :2].contiguous(), params, h0=h, conv_state_in=cs, h_T=h, conv_state_out=cs)
+    y2, _, _ = binding.prefill(x[:, 2:301].contiguous(), params, h0=h, conv_state_in=cs, h_T=h, conv_state_out=cs)
+    y3, _, _ = binding.prefill(x[:, 301:].contiguous(), params, h0=h, conv_state_in=cs, h_T=h, conv_state_out=cs)
+    torch.cuda.synchronize()
+    yr, hr, cr = oracle_prefill(oracle, inp, h0=inp["h0"].astype(np.float64), cs=inp["conv_state"].astype(np.float64))
+    assert_close("y", np.concatenate([to_np(y1), to_np(y2), to_np(y3)], 1), yr, "bf16")
+    assert_close("h_T", to_np(h), hr, "bf16")
+    assert np.array_equal(to_np(cs), cr)
+
+
+def test_status_ok_and_repeatable():
+    import torch
+    from paper_2402_19427_b200 import binding
+    inp = synth.make_inputs(1, 2000, 512, 2, io="bf16", seed=2)
+    params = binding.Params.from_numpy(inp["params"], "bf16")
+    x = to_dev(inp["x"], "bf16")
+    shape = binding.make_shape(1, 2000, 512, 2, torch.bfloat16)
+    ws = binding.alloc_workspace(shape, binding.OP_PREFILL, x.device)
+    outs = []
+    for _ in range(3):
+        y, hT, _ = binding.prefill(x, params, workspace=ws)
+        outs.append((y.clone(), hT.clone()))
+    assert binding.query_status(ws) == binding.OK
+    for y, hT in outs[1:]:
+        assert torch.equal(y, outs[0][0]) and torch.equal(hT, outs[0][1])   # same reduction order every run

@@ -261,6 +261,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
     __syncthreads();
     tc_fence_after();
 
+    // Register budget per warpgroup (the four warps of a group execute the same setmaxnreg):
+    // conv producers 72, loader / MMA issuer / idle 24, epilogue 208.
     if (warp < 4) {
         // ================================================================ conv producers
         reg_dec<72>();
@@ -338,9 +340,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             if (lane == 0) mbar_arrive(BAR_UFULL(st));
         }
         if (!ok && lane == 0) record_timeout(f.status, abort_flag);
-    } else if (warp == 4) {
+    } else if (warp < 8) {
+      reg_dec<24>();
+      if (warp == 4) {
         // ================================================================ TMA loader
-        reg_dec<24>();
         const __nv_bfloat16 *x = (const __nv_bfloat16 *)f.x;
         const __nv_bfloat16 *cs_in = (const __nv_bfloat16 *)f.cs_in;
         int slab_n = 0;
@@ -368,9 +371,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             }
         }
         if (!ok && lane == 0) record_timeout(f.status, abort_flag);
-    } else if (warp == 5) {
+      } else if (warp == 5) {
         // ================================================================ MMA issuer
-        reg_dec<24>();
         constexpr uint32_t idesc = make_idesc(128, TILE_N);
         bool ok = true;
         if (lane == 0) {
@@ -394,7 +396,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             if (!ok) record_timeout(f.status, abort_flag);
         }
         __syncwarp();
-    } else if (warp >= 8) {
+      }
+    } else {
         // ================================================================ epilogue
         reg_inc<208>();
         const int q = warp & 3, k = (warp - 8) >> 2;
@@ -565,8 +568,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         }
         ok = __all_sync(0xffffffffu, ok);
         if (!ok && lane == 0) record_timeout(f.status, abort_flag);
-    } else {
-        reg_dec<24>();
     }
 
     // ---- teardown: every role falls through to here, also after a timeout
@@ -608,9 +609,25 @@ bool sm100_prefill_supported(int B, int T, int D, int H, int io) {
     return io == RGLRU_BF16 && B > 0 && T > 0 && H > 0 && D == H * DH;
 }
 
-size_t sm100_prefill_workspace_bytes(int B, int T, int D, int H) {
+namespace {
+inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
+size_t agg_bytes(int B, int T, int H) {
     const size_t tps = (T + TILE_N - 1) / TILE_N;
-    return (size_t)H * 2 * B * tps * CH * sizeof(uint4);
+    return up256((size_t)H * 2 * B * tps * CH * sizeof(uint4));
+}
+inline bool ranges_overlap(const void *a, const void *b, size_t n) {
+    if (!a || !b) return false;
+    const uintptr_t pa = (uintptr_t)a, pb = (uintptr_t)b;
+    return pa < pb + n && pb < pa + n;
+}
+}  // namespace
+
+// Workspace body: aggregate records | private copy of h0 | private copy of conv_state_in.
+// The copies are used only when the caller's state outputs alias the state inputs: CTAs of
+// different tiles and of the two halves of a head read the incoming state at unrelated times,
+// so an in-place update must not be visible to them.
+size_t sm100_prefill_workspace_bytes(int B, int T, int D, int H) {
+    return agg_bytes(B, T, H) + up256((size_t)B * D * sizeof(float)) + up256((size_t)B * 3 * D * sizeof(__nv_bfloat16));
 }
 
 cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes, cudaStream_t st) {
@@ -636,6 +653,16 @@ cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes,
     p.agg = (uint4 *)ws_body;
     p.spin_ns = g_spin_limit_ns;
     if (ws_body_bytes < sm100_prefill_workspace_bytes(a.B, a.T, a.D, a.H)) return cudaErrorInvalidValue;
+    const size_t h_bytes = (size_t)a.B * a.D * sizeof(float), cs_bytes = (size_t)a.B * 3 * a.D * sizeof(__nv_bfloat16);
+    char *h0_copy = (char *)ws_body + agg_bytes(a.B, a.T, a.H), *cs_copy = h0_copy + up256(h_bytes);
+    if (ranges_overlap(a.h0, a.h_T, h_bytes)) {
+        if ((e = cudaMemcpyAsync(h0_copy, a.h0, h_bytes, cudaMemcpyDeviceToDevice, st)) != cudaSuccess) return e;
+        p.f.h0 = (const float *)h0_copy;
+    }
+    if (ranges_overlap(a.cs_in, a.cs_out, cs_bytes)) {
+        if ((e = cudaMemcpyAsync(cs_copy, a.cs_in, cs_bytes, cudaMemcpyDeviceToDevice, st)) != cudaSuccess) return e;
+        p.f.cs_in = cs_copy;
+    }
     dim3 grid(groups * S), block(NUM_THREADS);
     if (S > 1) {
         // CTAs wait on one another's aggregates: they must all be resident

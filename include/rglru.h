@@ -148,6 +148,32 @@ int32_t rglru_prefill_host(const rglru_shape_t *shape, const rglru_params_t *par
                            size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * rglru_prefill for callers that cannot allocate device memory (the paper has no counterpart;
+ * this is a deployment convenience).  A serving loop that runs on a memory pool sized and frozen at
+ * start-up, code under a framework allocator that forbids side allocations, or a process whose
+ * device memory is fully handed to other components has no way to provide the workspace that
+ * rglru_prefill asks for.  Here the scratch of the tensor-core prefill kernel lives in one array of
+ * RGLRU_STATIC_SCRATCH_BYTES that is part of the library image; the call allocates and frees nothing.
+ *   - Arguments x ... conv_state_out are those of rglru_prefill (device pointers, same aliasing rules).
+ *   - status_word: optional device pointer to a 4-byte-aligned uint32 owned by the caller, zero before the
+ *     first use.  A device-side wait that runs out is recorded there, and the pointer may be given to
+ *     rglru_query_status in place of a workspace.  NULL: such a condition is not reported.
+ *   - Only shapes served by the tensor-core kernel (bf16 io, head width 256) are accepted; others return
+ *     RGLRU_ERR_UNSUPPORTED.  A shape whose scratch (256 bytes + rglru_workspace_bytes(shape, PREFILL))
+ *     exceeds RGLRU_STATIC_SCRATCH_BYTES returns RGLRU_ERR_WORKSPACE; nothing is launched.
+ *   - Every GPU on which the library is loaded holds the array until the process exits.
+ *   - All calls on a device share the array: calls that overlap on the GPU (different streams without
+ *     ordering) race.  Order them on one stream or with events.  The array keeps the previous call's
+ *     contents; the call clears what has to start at zero on `cuda_stream` before its launch.
+ *   - The first call on each device looks up the array's device address (with that device current) and
+ *     caches it; make that first call outside any stream capture.
+ */
+#define RGLRU_STATIC_SCRATCH_BYTES ((size_t)8 << 20)
+int32_t rglru_prefill_static_scratch(const rglru_shape_t *shape, const rglru_params_t *params, const void *x,
+                                     const float *h0, const void *conv_state_in, void *y, float *h_T,
+                                     void *conv_state_out, void *status_word, void *cuda_stream);
+
+/*
  * Synchronises `cuda_stream` and returns the device-side status recorded in `workspace` by the
  * calls issued so far (RGLRU_OK, RGLRU_ERR_TIMEOUT, or RGLRU_ERR_CUDA if the stream itself
  * reports an error), then clears it.

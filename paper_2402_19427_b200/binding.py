@@ -22,7 +22,7 @@ FLAG_NONE, FLAG_FORCE_GENERIC = 0, 1
 
 EXPORTED = ["rglru_abi_version", "rglru_status_string", "rglru_workspace_bytes", "rglru_prefill",
             "rglru_decode_step", "rglru_backward", "rglru_host_staging_bytes", "rglru_prefill_host",
-            "rglru_query_status"]
+            "rglru_query_status", "rglru_prefill_static_scratch"]
 
 
 class Shape(ctypes.Structure):
@@ -70,6 +70,8 @@ def load() -> ctypes.CDLL:
         lib.rglru_host_staging_bytes.restype = sz
         lib.rglru_prefill_host.argtypes = [sp, pp] + [vp] * 7 + [sz, vp, sz, vp]
         lib.rglru_prefill_host.restype = i32
+        lib.rglru_prefill_static_scratch.argtypes = [sp, pp] + [vp] * 8
+        lib.rglru_prefill_static_scratch.restype = i32
         lib.rglru_query_status.argtypes = [vp, vp]
         lib.rglru_query_status.restype = i32
         _lib = lib
@@ -167,6 +169,31 @@ def prefill(x, params: Params, h0=None, conv_state_in=None, c=8.0, flags=0, y=No
                            _ptr(y), _ptr(h_T), _ptr(conv_state_out), _ptr(ws), ws.numel(), _stream())
     if rc != OK:
         raise RglruError(rc, "rglru_prefill")
+    return y, h_T, conv_state_out
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def prefill_static_scratch(x, params: Params, y, h_T, conv_state_out, h0=None, conv_state_in=None, c=8.0,
+                           status_word=None):
+    """rglru_prefill_static_scratch: the prefill for callers that cannot allocate device memory.  Every buffer,
+    outputs included, comes from the caller; the kernel's scratch is an array inside the library (shared by all
+    calls on the device, so calls must not overlap on the GPU).  ``status_word``: optional uint32 device tensor
+    that receives a device-side timeout and can be passed to :func:`query_status`."""
+    lib = load()
+    B, T, D = x.shape
+    shape = make_shape(B, T, D, params.H, x.dtype, c, 0)
+    dev = x.device
+    _chk(x, (B, T, D), params.io, "x", params.conv_w.device)
+    _chk(h0, (B, D), torch.float32, "h0", dev); _chk(conv_state_in, (B, 3, D), x.dtype, "conv_state_in", dev)
+    _chk(y, (B, T, D), x.dtype, "y", dev); _chk(h_T, (B, D), torch.float32, "h_T", dev)
+    _chk(conv_state_out, (B, 3, D), x.dtype, "conv_state_out", dev)
+    rc = lib.rglru_prefill_static_scratch(ctypes.byref(shape), ctypes.byref(params.ptrs), _ptr(x), _ptr(h0),
+                                          _ptr(conv_state_in), _ptr(y), _ptr(h_T), _ptr(conv_state_out),
+                                          _ptr(status_word), _stream())
+    if rc != OK:
+        raise RglruError(rc, "rglru_prefill_static_scratch")
     return y, h_T, conv_state_out
 
 

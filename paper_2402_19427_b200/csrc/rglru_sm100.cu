@@ -19,10 +19,12 @@
 // then does it run the real scan and write y.  Waits on other CTAs are bounded and end in
 // RGLRU_ERR_TIMEOUT; the launch is cooperative so that all CTAs are co-resident.
 #include <cooperative_groups.h>
+#include <cuda.h>
 #include <cuda_bf16.h>
 
 #include <atomic>
 #include <chrono>
+#include <type_traits>
 
 #include "rglru_internal.h"
 
@@ -45,10 +47,13 @@ constexpr uint32_t X_ROW_BYTES = DH * 2;                   // 512
 constexpr uint32_t X_SLAB_BYTES = SLAB_ROWS * X_ROW_BYTES; // 17920
 constexpr uint32_t SMEM_U = 0;
 constexpr uint32_t SMEM_X = SMEM_U + US * U_STAGE_BYTES;
-constexpr uint32_t SMEM_H = SMEM_X + XS * X_SLAB_BYTES;    // float h_s[4][2][32]
+constexpr uint32_t Y_ROW_BYTES = CH * 2;                   // 256: one token row of this CTA's channels
+constexpr uint32_t Y_HALF_BYTES = EPI_TOK * Y_ROW_BYTES;   // 16384: the 64 tokens of one epilogue half
+constexpr uint32_t SMEM_Y = SMEM_X + XS * X_SLAB_BYTES;    // bf16 y_s[2][64][128], staged for bulk stores
+constexpr uint32_t SMEM_H = SMEM_Y + 2 * Y_HALF_BYTES;     // float h_s[4][2][32]
 constexpr uint32_t SMEM_AGG = SMEM_H + 4 * 2 * 32 * 4;
 constexpr uint32_t SMEM_BAR = SMEM_AGG + 2 * 4 * 32 * 8; // float2 agg_s[2][4][32], indexed by tile parity
-constexpr int NUM_BARS = 2 * XS + 2 * US + 2 + 8 + 4;
+constexpr int NUM_BARS = 2 * XS + 2 * US + 2 + 8 + 4 + 4;
 constexpr uint32_t SMEM_MISC = SMEM_BAR + NUM_BARS * 8;    // tmem base, abort flag
 constexpr uint32_t SMEM_TOTAL = SMEM_MISC + 16;
 constexpr uint32_t SMEM_ALLOC = SMEM_TOTAL + 1024;         // slack for 1024-byte alignment
@@ -60,6 +65,9 @@ constexpr uint32_t TM_ACC_A = 0, TM_ACC_X = 128, TM_W_A = 256, TM_W_X = 384;
 constexpr float S_POLY = 0.25f;
 
 struct Sm100Args {
+    // x as [B][T][D] with a box of SLAB_ROWS token rows x one head; y with a box of EPI_TOK rows x CH channels
+    alignas(64) CUtensorMap tm_x;
+    alignas(64) CUtensorMap tm_y;
     FwdArgs f;
     int S;             // CTAs per half-head (time split factor)
     int tps;           // tiles per sequence
@@ -87,15 +95,21 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false when the limit ran out or the CTA is aborting.
+// Bounded wait.  Returns false when the limit ran out or the CTA is aborting.  mbarrier.try_wait
+// suspends the thread for a hardware-chosen window, so the loop polls rarely; the abort flag and the
+// global timer are consulted once every 32 polls to keep the loop itself cheap.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
     if (mbar_try(bar, parity)) return true;
-    const uint64_t t0 = gtimer();
-    while (!mbar_try(bar, parity)) {
-        if (*abort_flag) return false;
-        if (gtimer() - t0 > limit_ns) return false;
+    uint64_t t0 = 0;
+    for (uint32_t n = 1;; ++n) {
+        if (mbar_try(bar, parity)) return true;
+        if ((n & 31u) == 0u) {
+            if (*abort_flag) return false;
+            const uint64_t t = gtimer();
+            if (t0 == 0) t0 = t;
+            else if (t - t0 > limit_ns) return false;
+        }
     }
-    return true;
 }
 // All lanes wait; the verdict is made warp-uniform so that a warp never splits on a timeout.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
@@ -119,7 +133,9 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
     asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
                  ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
+typedef unsigned long long f32x2;
+// 32 consecutive columns of this thread's lane as 16 register pairs (column 2j in the low half).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, f32x2 *v) {
     uint32_t r[32];
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
@@ -128,7 +144,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
                    "=r"(r[30]), "=r"(r[31])
                  : "r"(taddr) : "memory");
 #pragma unroll
-    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+    for (int j = 0; j < 16; ++j) asm("mov.b64 %0, {%1, %2};" : "=l"(v[j]) : "r"(r[2 * j]), "r"(r[2 * j + 1]));
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st8(uint32_t taddr, uint4 lo, uint4 hi) {
@@ -136,6 +152,23 @@ __device__ __forceinline__ void tmem_st8(uint32_t taddr, uint4 lo, uint4 hi) {
                  ::"r"(taddr), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// shared -> global bulk copy, tracked by this thread's bulk async-group
+__device__ __forceinline__ void bulk_s2g(void *dst, uint32_t src_smem, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem), "r"(bytes) : "memory");
+}
+// one tiled TMA load of a [rows x channels] box at (channel c0, token t, sequence b); rows outside [0, T) read as zero
+__device__ __forceinline__ void tma_load_3d(uint32_t dst_smem, const CUtensorMap *tm, int c0, int t, int b, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst_smem), "l"(tm), "r"(c0), "r"(t), "r"(b), "r"(bar) : "memory");
+}
+// one tiled TMA store; rows at or beyond T are clipped by the tensor bounds
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *tm, int c0, int t, int b, uint32_t src_smem) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+                 ::"l"(tm), "r"(c0), "r"(t), "r"(b), "r"(src_smem) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
@@ -154,10 +187,9 @@ __host__ __device__ constexpr uint32_t make_idesc(int M, int N) {
 }
 
 // ---- packed fp32x2 arithmetic (one issue slot for two lanes' worth of FP32 work)
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pack2(float lo, float hi) { return ((f32x2)__float_as_uint(hi) << 32) | __float_as_uint(lo); }
-__device__ __forceinline__ float lo2(f32x2 v) { return __uint_as_float((uint32_t)v); }
-__device__ __forceinline__ float hi2(f32x2 v) { return __uint_as_float((uint32_t)(v >> 32)); }
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) { f32x2 v; asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi)); return v; }
+__device__ __forceinline__ float lo2(f32x2 v) { float lo, hi; asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); return lo; }
+__device__ __forceinline__ float hi2(f32x2 v) { float lo, hi; asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); return hi; }
 __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
 __device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
 __device__ __forceinline__ float tanh_approx(float x) { float y; asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
@@ -169,14 +201,14 @@ __device__ __forceinline__ void record_timeout(uint32_t *status, volatile int *a
     atomicExch(status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
 }
 
-// (z_a, z_x) of two consecutive tokens of one channel -> (a_t, v_t) of Eq. 3-4, in place.
+// (z_a, z_x) of two tokens of one channel, one token per half of the register pair -> (a_t, v_t) of
+// Eq. 3-4, in place.
 //   r = sigmoid(z_a + b_a) = 1/2 + 1/2 tanh((z_a + b_a)/2),  x = 2 s r,  f = 1 - a_t = -expm1(-x/2),
 //   m/2 = sqrt(f (1/2 - f/4)) = sqrt(1 - a_t^2)/2,  v = (m/2 u)(1 + tanh((z_x + b_x)/2)) = m i u.
 template <bool POLY>
-__device__ __forceinline__ void gate_pair(float &za0, float &za1, float &zx0, float &zx1, float u0, float u1, f32x2 hba2, f32x2 hbx2,
-                                          f32x2 s2) {
+__device__ __forceinline__ void gate_pair(f32x2 &za, f32x2 &zx, float u0, float u1, f32x2 hba2, f32x2 hbx2, f32x2 s2) {
     const f32x2 HALF2 = pack2(0.5f, 0.5f);
-    f32x2 ta = fma2(pack2(za0, za1), HALF2, hba2);
+    f32x2 ta = fma2(za, HALF2, hba2);
     ta = pack2(tanh_approx(lo2(ta)), tanh_approx(hi2(ta)));
     const f32x2 x = fma2(ta, s2, s2);
     f32x2 f, a;
@@ -195,12 +227,11 @@ __device__ __forceinline__ void gate_pair(float &za0, float &za1, float &zx0, fl
     f32x2 q = mul2(f, fma2(f, pack2(-0.25f, -0.25f), HALF2));  // (1 - a^2)/4 = f (2 - f)/4
     if (!POLY) q = pack2(fmaxf(lo2(q), 0.0f), fmaxf(hi2(q), 0.0f));  // a from ex2.approx may round above 1
     const f32x2 mh = pack2(sqrt_approx(lo2(q)), sqrt_approx(hi2(q)));
-    f32x2 tx = fma2(pack2(zx0, zx1), HALF2, hbx2);
+    f32x2 tx = fma2(zx, HALF2, hbx2);
     tx = pack2(tanh_approx(lo2(tx)), tanh_approx(hi2(tx)));
     const f32x2 g = mul2(mh, pack2(u0, u1));
-    const f32x2 v = fma2(g, tx, g);
-    za0 = lo2(a); za1 = hi2(a);
-    zx0 = lo2(v); zx1 = hi2(v);
+    za = a;
+    zx = fma2(g, tx, g);
 }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __grid_constant__ Sm100Args p) {
@@ -218,6 +249,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
     const uint32_t BAR_ACCEMPTY = BAR_ACCFULL + 8u;
     auto BAR_CHAIN = [&](int q, int k) { return BAR_ACCEMPTY + 8u + 8u * (q * 2 + k); };
     auto BAR_AGG = [&](int q) { return BAR_ACCEMPTY + 8u + 8u * (8 + q); };
+    auto BAR_YFREE = [&](int k) { return BAR_ACCEMPTY + 8u + 8u * (12 + k); };
+    auto BAR_YFULL = [&](int k) { return BAR_ACCEMPTY + 8u + 8u * (14 + k); };
     uint32_t *tmem_base_s = (uint32_t *)(smem + SMEM_MISC);
     volatile int *abort_flag = (volatile int *)(smem + SMEM_MISC + 4);
     float *h_s = (float *)(smem + SMEM_H);
@@ -237,6 +270,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         mbar_init(BAR_ACCFULL, 1);
         mbar_init(BAR_ACCEMPTY, 8);
         for (int q = 0; q < 4; ++q) { mbar_init(BAR_CHAIN(q, 0), 1); mbar_init(BAR_CHAIN(q, 1), 1); mbar_init(BAR_AGG(q), 1); }
+        for (int k = 0; k < 2; ++k) { mbar_init(BAR_YFREE(k), 4); mbar_init(BAR_YFULL(k), 4); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -283,6 +317,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         } else { b01 = pack2(0.f, 0.f); b23 = b01; }
         const uint32_t x_thread_off = (uint32_t)hc * 2;
         const uint32_t u_chunk = (uint32_t)(l16 >> 1), u_half = (uint32_t)(l16 & 1) * 8;
+        // Token tt of a tile is stored in row perm(tt) of the U tile (= accumulator column perm(tt)):
+        // within each group of 64 tokens, tokens j and j + 32 sit in adjacent rows 2j and 2j + 1, so that
+        // the epilogue finds them in one register pair and can run the two halves of its 64 tokens as
+        // the two lanes of packed fp32x2 arithmetic.
         int slab_n = 0;
         bool ok = true;
         for (int it = 0; it < n_my_tiles && ok; ++it) {
@@ -291,7 +329,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             const int st = it % US;
             ok = warp_wait(BAR_UEMPTY(st), ((it / US) & 1) ^ 1, spin, abort_flag);
             if (!ok) break;
-            const uint32_t u_base = base + SMEM_U + st * U_STAGE_BYTES + pblk * U_KBLOCK_BYTES;
+            const uint32_t u_base = SMEM_U + st * U_STAGE_BYTES + pblk * U_KBLOCK_BYTES + u_half;  // offset from smem
             const int nslab = min(TILE_N / SLAB, (T - t0 + SLAB - 1) / SLAB);
             for (int s = 0; s < nslab; ++s, ++slab_n) {
                 const int slot = slab_n % XS;
@@ -300,33 +338,55 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
                 const int ts0 = t0 + s * SLAB;
                 const bool zero_halo = (ts0 == 0) && (f.cs_in == nullptr);
                 const int nvalid = min(SLAB, T - ts0) - tg * 16;  // tokens of this thread's group that exist
-                const uint8_t *xs = smem + SMEM_X + slot * X_SLAB_BYTES + x_thread_off;
-                auto load_row = [&](int r, f32x2 &v01, f32x2 &v23) {
-                    uint2 w = *(const uint2 *)(xs + r * X_ROW_BYTES);
-                    if (zero_halo && r < 3) { w.x = 0u; w.y = 0u; }
+                const uint8_t *xs = smem + SMEM_X + slot * X_SLAB_BYTES + x_thread_off + (uint32_t)(tg * 16) * X_ROW_BYTES;
+                auto load_row = [&](int r, f32x2 &v01, f32x2 &v23) {   // r: row relative to this thread's first halo row
+                    const uint2 w = *(const uint2 *)(xs + (uint32_t)r * X_ROW_BYTES);
                     v01 = pack2(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xFFFF0000u));
                     v23 = pack2(__uint_as_float(w.y << 16), __uint_as_float(w.y & 0xFFFF0000u));
                 };
+                // row of token i of this thread: rowbase + 2 i; its 16-byte chunk is swizzled by (row & 7) = (p + 2 i) & 7
+                const uint32_t pbit = (uint32_t)(s & 1);
+                const uint32_t row_addr = u_base + (uint32_t)((s >> 1) * 64 + (s & 1) + 32 * tg) * 128u;
+                uint32_t sw[4];
+#pragma unroll
+                for (int m = 0; m < 4; ++m) sw[m] = row_addr + ((u_chunk ^ ((pbit + 2u * m) & 7u)) << 4);
                 if (nvalid > 0) {
-                    const int r0 = tg * 16;
                     f32x2 a01, a23, b01x, b23x, c01, c23;  // x_{t-3}, x_{t-2}, x_{t-1}
-                    load_row(r0, a01, a23); load_row(r0 + 1, b01x, b23x); load_row(r0 + 2, c01, c23);
-#pragma unroll 4
-                    for (int i = 0; i < 16; ++i) {
-                        if (i < nvalid) {
+                    load_row(0, a01, a23); load_row(1, b01x, b23x); load_row(2, c01, c23);
+                    if (zero_halo && tg == 0) { a01 = a23 = b01x = b23x = c01 = c23 = pack2(0.f, 0.f); }
+                    auto one_token = [&](int i, f32x2 &xa01, f32x2 &xa23, f32x2 &xb01, f32x2 &xb23, f32x2 &xc01, f32x2 &xc23) {
+                        f32x2 d01, d23;
+                        load_row(3 + i, d01, d23);
+                        f32x2 u01 = fma2(w01[0], d01, b01), u23 = fma2(w23[0], d23, b23);
+                        u01 = fma2(w01[1], xc01, u01); u23 = fma2(w23[1], xc23, u23);
+                        u01 = fma2(w01[2], xb01, u01); u23 = fma2(w23[2], xb23, u23);
+                        u01 = fma2(w01[3], xa01, u01); u23 = fma2(w23[3], xa23, u23);
+                        __nv_bfloat162 o01 = __floats2bfloat162_rn(lo2(u01), hi2(u01));
+                        __nv_bfloat162 o23 = __floats2bfloat162_rn(lo2(u23), hi2(u23));
+                        *(uint2 *)(smem + sw[i & 3] + (uint32_t)i * 256u) = make_uint2(*(uint32_t *)&o01, *(uint32_t *)&o23);
+                        xa01 = d01; xa23 = d23;   // the oldest slot now holds the newest row
+                    };
+                    if (nvalid >= 16) {
+                        // three rotating history slots: the roles cycle with period 3, fully unrolled
+#pragma unroll
+                        for (int i = 0; i < 15; i += 3) {
+                            one_token(i, a01, a23, b01x, b23x, c01, c23);
+                            one_token(i + 1, b01x, b23x, c01, c23, a01, a23);
+                            one_token(i + 2, c01, c23, a01, a23, b01x, b23x);
+                        }
+                        one_token(15, a01, a23, b01x, b23x, c01, c23);
+                    } else {
+                        for (int i = 0; i < nvalid; ++i) {
                             f32x2 d01, d23;
-                            load_row(r0 + 3 + i, d01, d23);
+                            load_row(3 + i, d01, d23);
                             f32x2 u01 = fma2(w01[0], d01, b01), u23 = fma2(w23[0], d23, b23);
                             u01 = fma2(w01[1], c01, u01); u23 = fma2(w23[1], c23, u23);
                             u01 = fma2(w01[2], b01x, u01); u23 = fma2(w23[2], b23x, u23);
                             u01 = fma2(w01[3], a01, u01); u23 = fma2(w23[3], a23, u23);
                             __nv_bfloat162 o01 = __floats2bfloat162_rn(lo2(u01), hi2(u01));
                             __nv_bfloat162 o23 = __floats2bfloat162_rn(lo2(u23), hi2(u23));
-                            const int row = s * SLAB + r0 + i;
-                            const uint32_t off = (uint32_t)row * 128u + ((u_chunk ^ (uint32_t)(row & 7)) << 4) + u_half;
-                            uint2 o;
-                            o.x = *(uint32_t *)&o01; o.y = *(uint32_t *)&o23;
-                            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(u_base + off), "r"(o.x), "r"(o.y) : "memory");
+                            const uint32_t addr = row_addr + ((u_chunk ^ ((pbit + 2u * (uint32_t)i) & 7u)) << 4) + (uint32_t)i * 256u;
+                            *(uint2 *)(smem + addr) = make_uint2(*(uint32_t *)&o01, *(uint32_t *)&o23);
                             a01 = b01x; a23 = b23x; b01x = c01; b23x = c23; c01 = d01; c23 = d23;
                         }
                     }
@@ -357,17 +417,26 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
                 ok = warp_wait(BAR_XEMPTY(slot), ((slab_n / XS) & 1) ^ 1, spin, abort_flag);
                 if (!ok) break;
                 const int ts0 = t0 + s * SLAB;
-                const int lo_row = (ts0 == 0 && cs_in == nullptr) ? 3 : 0;   // rows with no source stay untouched
-                const int hi_row = min(SLAB_ROWS, T - ts0 + 3);
-                if (lane == 0) mbar_expect_tx(BAR_XFULL(slot), (uint32_t)(hi_row - lo_row) * X_ROW_BYTES);
-                __syncwarp();
-                for (int r = lane; r < SLAB_ROWS; r += 32) {
-                    if (r < lo_row || r >= hi_row) continue;
-                    const int t = ts0 - 3 + r;
-                    const __nv_bfloat16 *src = t >= 0 ? x + ((size_t)b * T + t) * D + head * DH
-                                                      : cs_in + ((size_t)b * 3 + (3 + t)) * D + head * DH;
-                    bulk_g2s(base + SMEM_X + slot * X_SLAB_BYTES + r * X_ROW_BYTES, src, X_ROW_BYTES, BAR_XFULL(slot));
+                const uint32_t dst = base + SMEM_X + slot * X_SLAB_BYTES;
+                if (ts0 == 0 && cs_in != nullptr) {
+                    // first slab of a sequence with an incoming conv state: the three halo rows come from
+                    // conv_state_in, so the slab is assembled from row copies
+                    const int hi_row = min(SLAB_ROWS, T + 3);
+                    if (lane == 0) mbar_expect_tx(BAR_XFULL(slot), (uint32_t)hi_row * X_ROW_BYTES);
+                    __syncwarp();
+                    for (int r = lane; r < hi_row; r += 32) {
+                        const int t = r - 3;
+                        const __nv_bfloat16 *src = t >= 0 ? x + ((size_t)b * T + t) * D + head * DH
+                                                          : cs_in + ((size_t)b * 3 + (3 + t)) * D + head * DH;
+                        bulk_g2s(dst + r * X_ROW_BYTES, src, X_ROW_BYTES, BAR_XFULL(slot));
+                    }
+                } else if (lane == 0) {
+                    // one tiled copy per slab: SLAB_ROWS token rows of this head starting three tokens early
+                    // (tokens before the sequence start and past its end read as zero)
+                    mbar_expect_tx(BAR_XFULL(slot), X_SLAB_BYTES);
+                    tma_load_3d(dst, &p.tm_x, head * DH, ts0 - 3, b, BAR_XFULL(slot));
                 }
+                __syncwarp();
             }
         }
         if (!ok && lane == 0) record_timeout(f.status, abort_flag);
@@ -411,17 +480,18 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         const f32x2 s2 = pack2(s, s);
         const f32x2 hba2 = pack2(0.5f * f.b_a[d], 0.5f * f.b_a[d]), hbx2 = pack2(0.5f * f.b_x[d], 0.5f * f.b_x[d]);
         const bool poly = __all_sync(0xffffffffu, s <= S_POLY);
-        // u[token][channel] in the swizzled U tile: 8 row phases
+        // u[row][channel] in the swizzled U tile, one offset per row phase (row & 7)
         uint32_t u_off[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j)
             u_off[j] = (uint32_t)(hc >> 6) * U_KBLOCK_BYTES + ((((uint32_t)(hc & 63) >> 3) ^ (uint32_t)j) << 4) + (uint32_t)(hc & 7) * 2 +
                        (uint32_t)(k * EPI_TOK) * 128u;
         const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16);
+        uint16_t *y_s = (uint16_t *)(smem + SMEM_Y + (uint32_t)k * Y_HALF_BYTES + (uint32_t)c_own * 2u);  // this thread's column of the y staging tile
         __nv_bfloat16 *y = (__nv_bfloat16 *)f.y;
         const __nv_bfloat16 *x = (const __nv_bfloat16 *)f.x;
         const __nv_bfloat16 *cs_in = (const __nv_bfloat16 *)f.cs_in;
-        float h_prev_own = 0.0f;  // warp 0: state after this CTA's previous tile
+        float h_prev_own = 0.0f;  // k == 0: state after this CTA's previous tile
         bool ok = true;
         for (int it = 0; it < n_my_tiles && ok; ++it) {
             const int g = kcta + it * S, b = g / p.tps, ti = g % p.tps;
@@ -431,36 +501,49 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             ok = warp_wait(BAR_ACCFULL, it & 1, spin, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            float za[EPI_TOK], zx[EPI_TOK];
-            tmem_ld32(tm_lane + TM_ACC_A + k * EPI_TOK, za);
-            tmem_ld32(tm_lane + TM_ACC_A + k * EPI_TOK + 32, za + 32);
-            tmem_ld32(tm_lane + TM_ACC_X + k * EPI_TOK, zx);
-            tmem_ld32(tm_lane + TM_ACC_X + k * EPI_TOK + 32, zx + 32);
+            // A2[j] / V2[j]: tokens j (low half) and j + 32 (high half) of this warp's 64 tokens
+            f32x2 A2[EPI_TOK / 2], V2[EPI_TOK / 2];
+            tmem_ld32(tm_lane + TM_ACC_A + k * EPI_TOK, A2);
+            tmem_ld32(tm_lane + TM_ACC_A + k * EPI_TOK + 32, A2 + 16);
+            tmem_ld32(tm_lane + TM_ACC_X + k * EPI_TOK, V2);
+            tmem_ld32(tm_lane + TM_ACC_X + k * EPI_TOK + 32, V2 + 16);
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(BAR_ACCEMPTY);  // the accumulators now live in registers
             // gates, decay, input scale: (z_a, z_x) -> (a_t, v_t) in place
-            const uint32_t u_base = base + SMEM_U + st * U_STAGE_BYTES;
+            const uint8_t *u_tile = smem + SMEM_U + st * U_STAGE_BYTES;
+            auto gates = [&](auto poly_tag) {
+                constexpr bool POLY = decltype(poly_tag)::value;
 #pragma unroll
-            for (int i = 0; i < EPI_TOK; i += 2) {
-                uint16_t ub0, ub1;
-                asm volatile("ld.shared.u16 %0, [%1];" : "=h"(ub0) : "r"(u_base + u_off[i & 7] + (uint32_t)i * 128u));
-                asm volatile("ld.shared.u16 %0, [%1];" : "=h"(ub1) : "r"(u_base + u_off[(i + 1) & 7] + (uint32_t)(i + 1) * 128u));
-                const float u0 = __uint_as_float((uint32_t)ub0 << 16), u1 = __uint_as_float((uint32_t)ub1 << 16);
-                if (poly) gate_pair<true>(za[i], za[i + 1], zx[i], zx[i + 1], u0, u1, hba2, hbx2, s2);
-                else gate_pair<false>(za[i], za[i + 1], zx[i], zx[i + 1], u0, u1, hba2, hbx2, s2);
-            }
+                for (int j = 0; j < EPI_TOK / 2; ++j) {
+                    // rows 2j (token j) and 2j + 1 (token j + 32)
+                    const uint32_t ub0 = *(const uint16_t *)(u_tile + u_off[(2 * j) & 7] + (uint32_t)(2 * j) * 128u);
+                    const uint32_t ub1 = *(const uint16_t *)(u_tile + u_off[(2 * j + 1) & 7] + (uint32_t)(2 * j + 1) * 128u);
+                    gate_pair<POLY>(A2[j], V2[j], __uint_as_float(ub0 << 16), __uint_as_float(ub1 << 16), hba2, hbx2, s2);
+                }
+            };
+            if (poly) gates(std::true_type{}); else gates(std::false_type{});
             __syncwarp();
             if (lane == 0) mbar_arrive(BAR_UEMPTY(st));  // done reading u
+            if (nv < EPI_TOK) {
+                // ragged tail: tokens that do not exist hold the state (a = 1, v = 0)
+#pragma unroll
+                for (int j = 0; j < EPI_TOK / 2; ++j) {
+                    const bool v0 = j < nv, v1 = j + 32 < nv;
+                    A2[j] = pack2(v0 ? lo2(A2[j]) : 1.0f, v1 ? hi2(A2[j]) : 1.0f);
+                    V2[j] = pack2(v0 ? lo2(V2[j]) : 0.0f, v1 ? hi2(V2[j]) : 0.0f);
+                }
+            }
+            // ---- fold both halves at once: h_out = P h_in + hl for tokens [0,32) (low) and [32,64) (high)
+            f32x2 P2 = pack2(1.0f, 1.0f), HL2 = pack2(0.0f, 0.0f);
+#pragma unroll
+            for (int j = 0; j < EPI_TOK / 2; ++j) { P2 = mul2(P2, A2[j]); HL2 = fma2(A2[j], HL2, V2[j]); }
+            const float P_lo = lo2(P2), hl_lo = lo2(HL2);
+            const float P = P_lo * hi2(P2), hl = fmaf(hi2(P2), hl_lo, hi2(HL2));
             // ---- incoming state
             float h;
             if (S > 1) {
-                // fold this warp's tokens to (P, h_loc): h_out = P h_in + h_loc
-                float P = 1.0f, hl = 0.0f;
-#pragma unroll
-                for (int i = 0; i < EPI_TOK; ++i)
-                    if (i < nv) { P *= za[i]; hl = fmaf(za[i], hl, zx[i]); }
                 if (k == 0) {
                     agg_s[((it & 1) * 4 + q) * 32 + lane] = make_float2(P, hl);
                     __syncwarp();
@@ -477,7 +560,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
                 }
             }
             if (k == 0) {
-                if (it > 0) {  // state after this CTA's previous tile (written by warp 1)
+                if (it > 0) {  // state after this CTA's previous tile (written by the k == 1 warp)
                     ok = warp_wait(BAR_CHAIN(q, 0), (it - 1) & 1, spin, abort_flag);
                     if (!ok) break;
                     h_prev_own = h_s[(q * 2 + 0) * 32 + lane];
@@ -496,8 +579,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
                 if (nback > 0) {
                     const uint4 *src = p.agg + ((size_t)group * p.tiles_total + g) * CH + c_own;
                     uint4 rec[MAX_S - 1];
-                    const uint64_t tstart = gtimer();
-                    for (;;) {
+                    uint64_t tstart = 0;
+                    for (uint32_t npoll = 0;; ++npoll) {
                         bool ready = true;
 #pragma unroll
                         for (int j = 1; j < MAX_S; ++j) {
@@ -511,8 +594,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
                         for (int j = 1; j < MAX_S; ++j)
                             if (j <= nback) ready = ready && rec[j - 1].y == p.tag && rec[j - 1].w == p.tag;
                         if (__all_sync(0xffffffffu, ready)) break;
-                        if (*abort_flag || gtimer() - tstart > spin) { ok = false; break; }
-                        __nanosleep(100);
+                        if ((npoll & 15u) == 15u) {
+                            const uint64_t tnow = gtimer();
+                            if (tstart == 0) tstart = tnow;
+                            if (*abort_flag || tnow - tstart > spin) { ok = false; break; }
+                        }
+                        __nanosleep(64);
                     }
                     ok = __all_sync(0xffffffffu, ok);
                     if (ok) {
@@ -527,30 +614,30 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
                 if (!ok) break;
                 h = h_s[(q * 2 + 1) * 32 + lane];
             }
-            // ---- the recurrence h_t = a_t h_{t-1} + v_t (Eq. 4) and y_t = h_t
-            __nv_bfloat16 *yp = y + ((size_t)b * T + t0 + k * EPI_TOK) * D + d;
-            if (nv == EPI_TOK) {
-#pragma unroll
-                for (int i = 0; i < EPI_TOK; i += 2) {
-                    const float h0v = fmaf(za[i], h, zx[i]);
-                    h = fmaf(za[i + 1], h0v, zx[i + 1]);
-                    const __nv_bfloat162 o = __floats2bfloat162_rn(h0v, h);
-                    yp[(size_t)i * D] = o.x;
-                    yp[(size_t)(i + 1) * D] = o.y;
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < EPI_TOK; ++i) {
-                    if (i < nv) {
-                        h = fmaf(za[i], h, zx[i]);
-                        yp[(size_t)i * D] = __float2bfloat16_rn(h);
-                    }
-                }
+            // ---- the y staging rows of this half must have been read out by the previous tile's bulk stores
+            if (it > 0) {
+                if (q == 0 && lane == 0) bulk_wait_read0();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(BAR_YFREE(k));
+                ok = warp_wait(BAR_YFREE(k), (it - 1) & 1, spin, abort_flag);
+                if (!ok) break;
             }
+            // ---- the recurrence h_t = a_t h_{t-1} + v_t (Eq. 4), both halves in lock step; y_t = h_t
+            f32x2 H2 = pack2(h, fmaf(P_lo, h, hl_lo));
+#pragma unroll
+            for (int j = 0; j < EPI_TOK / 2; ++j) {
+                H2 = fma2(A2[j], H2, V2[j]);
+                const __nv_bfloat162 o = __floats2bfloat162_rn(lo2(H2), hi2(H2));
+                const uint32_t ow = *(const uint32_t *)&o;
+                y_s[j * (Y_ROW_BYTES / 2)] = (uint16_t)(ow & 0xFFFFu);
+                y_s[(j + 32) * (Y_ROW_BYTES / 2)] = (uint16_t)(ow >> 16);
+            }
+            h = hi2(H2);
             // ---- hand the state on
             h_s[(q * 2 + (k ^ 1)) * 32 + lane] = h;
+            fence_async_smem();   // y rows become visible to the bulk-copy engine
             __syncwarp();
-            if (lane == 0) mbar_arrive(BAR_CHAIN(q, k ^ 1));
+            if (lane == 0) { mbar_arrive(BAR_CHAIN(q, k ^ 1)); mbar_arrive(BAR_YFULL(k)); }
             if (k == 1 && ti == p.tps - 1) {
                 // end of a sequence: h_T (unrounded state) and the last three raw inputs, bit-exact
                 f.h_T[(size_t)b * D + d] = h;
@@ -565,7 +652,16 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
 #pragma unroll
                 for (int kk = 0; kk < 3; ++kk) cs_out[((size_t)b * 3 + kk) * D + d] = keep[kk];
             }
+            // ---- y: once the four warps of this half have written their columns, one thread sends the
+            //      64 x 128 tile to HBM with a single tiled TMA store
+            ok = warp_wait(BAR_YFULL(k), it & 1, spin, abort_flag);
+            if (!ok) break;
+            if (q == 0 && lane == 0) {
+                if (nv > 0) tma_store_3d(&p.tm_y, head * DH + half * CH, t0 + k * EPI_TOK, b, base + SMEM_Y + (uint32_t)k * Y_HALF_BYTES);
+                bulk_commit();
+            }
         }
+        if (q == 0 && lane == 0) bulk_wait0();
         ok = __all_sync(0xffffffffu, ok);
         if (!ok && lane == 0) record_timeout(f.status, abort_flag);
     }
@@ -591,6 +687,33 @@ int num_sms() {
             return 148;
     }
     return cached;
+}
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point lookup (the library does not link libcuda)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = [] {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+            ptr = nullptr;
+        return (EncodeTiledFn)ptr;
+    }();
+    return fn;
+}
+
+// Tensor map of a bf16 [B][T][D] activation tensor with a box of box_t token rows x box_c channels.
+bool make_activation_map(CUtensorMap *tm, const void *ptr, int B, int T, int D, int box_c, int box_t) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (enc == nullptr) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)T, (cuuint64_t)B};
+    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)T * D * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)box_c, (cuuint32_t)box_t, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 std::atomic<uint32_t> g_call_counter{0};
@@ -639,6 +762,8 @@ cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes,
         attr_set = true;
     }
     Sm100Args p;
+    if (!make_activation_map(&p.tm_x, a.x, a.B, a.T, a.D, DH, SLAB_ROWS) || !make_activation_map(&p.tm_y, a.y, a.B, a.T, a.D, CH, EPI_TOK))
+        return cudaErrorNotSupported;
     p.f = a;
     p.tps = (a.T + TILE_N - 1) / TILE_N;
     p.tiles_total = a.B * p.tps;

@@ -50,10 +50,9 @@ constexpr uint32_t SMEM_X = SMEM_U + US * U_STAGE_BYTES;
 constexpr uint32_t Y_ROW_BYTES = CH * 2;                   // 256: one token row of this CTA's channels
 constexpr uint32_t Y_HALF_BYTES = EPI_TOK * Y_ROW_BYTES;   // 16384: the 64 tokens of one epilogue half
 constexpr uint32_t SMEM_Y = SMEM_X + XS * X_SLAB_BYTES;    // bf16 y_s[2][64][128], staged for bulk stores
-constexpr uint32_t SMEM_H = SMEM_Y + 2 * Y_HALF_BYTES;     // float h_s[4][2][32]
-constexpr uint32_t SMEM_AGG = SMEM_H + 4 * 2 * 32 * 4;
-constexpr uint32_t SMEM_BAR = SMEM_AGG + 2 * 4 * 32 * 8; // float2 agg_s[2][4][32], indexed by tile parity
-constexpr int NUM_BARS = 2 * XS + 2 * US + 2 + 8 + 4 + 4;
+constexpr uint32_t SMEM_AGG = SMEM_Y + 2 * Y_HALF_BYTES;   // float2 agg_s[2 tile parity][2 halves][4][32]
+constexpr uint32_t SMEM_BAR = SMEM_AGG + 2 * 2 * 4 * 32 * 8;
+constexpr int NUM_BARS = 2 * XS + 2 * US + 4 + 8 + 4;
 constexpr uint32_t SMEM_MISC = SMEM_BAR + NUM_BARS * 8;    // tmem base, abort flag
 constexpr uint32_t SMEM_TOTAL = SMEM_MISC + 16;
 constexpr uint32_t SMEM_ALLOC = SMEM_TOTAL + 1024;         // slack for 1024-byte alignment
@@ -245,15 +244,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
     auto BAR_XEMPTY = [&](int s) { return bar0 + 8u * (XS + s); };
     auto BAR_UFULL = [&](int s) { return bar0 + 8u * (2 * XS + s); };
     auto BAR_UEMPTY = [&](int s) { return bar0 + 8u * (2 * XS + US + s); };
-    const uint32_t BAR_ACCFULL = bar0 + 8u * (2 * XS + 2 * US);
-    const uint32_t BAR_ACCEMPTY = BAR_ACCFULL + 8u;
-    auto BAR_CHAIN = [&](int q, int k) { return BAR_ACCEMPTY + 8u + 8u * (q * 2 + k); };
-    auto BAR_AGG = [&](int q) { return BAR_ACCEMPTY + 8u + 8u * (8 + q); };
-    auto BAR_YFREE = [&](int k) { return BAR_ACCEMPTY + 8u + 8u * (12 + k); };
-    auto BAR_YFULL = [&](int k) { return BAR_ACCEMPTY + 8u + 8u * (14 + k); };
+    auto BAR_ACCFULL = [&](int k) { return bar0 + 8u * (2 * XS + 2 * US + k); };       // accumulators of token half k
+    auto BAR_ACCEMPTY = [&](int k) { return bar0 + 8u * (2 * XS + 2 * US + 2 + k); };
+    auto BAR_AGG = [&](int q, int k) { return bar0 + 8u * (2 * XS + 2 * US + 4 + q * 2 + k); };  // fold of half k, channel group q
+    auto BAR_YFREE = [&](int k) { return bar0 + 8u * (2 * XS + 2 * US + 12 + k); };
+    auto BAR_YFULL = [&](int k) { return bar0 + 8u * (2 * XS + 2 * US + 14 + k); };
     uint32_t *tmem_base_s = (uint32_t *)(smem + SMEM_MISC);
     volatile int *abort_flag = (volatile int *)(smem + SMEM_MISC + 4);
-    float *h_s = (float *)(smem + SMEM_H);
     float2 *agg_s = (float2 *)(smem + SMEM_AGG);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -267,9 +264,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
     if (tid == 0) {
         for (int s = 0; s < XS; ++s) { mbar_init(BAR_XFULL(s), 1); mbar_init(BAR_XEMPTY(s), 4); }
         for (int s = 0; s < US; ++s) { mbar_init(BAR_UFULL(s), 4); mbar_init(BAR_UEMPTY(s), 9); }
-        mbar_init(BAR_ACCFULL, 1);
-        mbar_init(BAR_ACCEMPTY, 8);
-        for (int q = 0; q < 4; ++q) { mbar_init(BAR_CHAIN(q, 0), 1); mbar_init(BAR_CHAIN(q, 1), 1); mbar_init(BAR_AGG(q), 1); }
+        for (int k = 0; k < 2; ++k) { mbar_init(BAR_ACCFULL(k), 1); mbar_init(BAR_ACCEMPTY(k), 4); }
+        for (int q = 0; q < 4; ++q) { mbar_init(BAR_AGG(q, 0), 1); mbar_init(BAR_AGG(q, 1), 1); }
         for (int k = 0; k < 2; ++k) { mbar_init(BAR_YFREE(k), 4); mbar_init(BAR_YFULL(k), 4); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -296,7 +292,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
     tc_fence_after();
 
     // Register budget per warpgroup (the four warps of a group execute the same setmaxnreg):
-    // conv producers 72, loader / MMA issuer / idle 24, epilogue 208.
+    // conv producers 72, loader / MMA issuer / idle 40, epilogue 200.
     if (warp < 4) {
         // ================================================================ conv producers
         reg_dec<72>();
@@ -401,7 +397,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         }
         if (!ok && lane == 0) record_timeout(f.status, abort_flag);
     } else if (warp < 8) {
-      reg_dec<24>();
+      reg_dec<40>();
       if (warp == 4) {
         // ================================================================ TMA loader
         const __nv_bfloat16 *x = (const __nv_bfloat16 *)f.x;
@@ -442,25 +438,32 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         if (!ok && lane == 0) record_timeout(f.status, abort_flag);
       } else if (warp == 5) {
         // ================================================================ MMA issuer
-        constexpr uint32_t idesc = make_idesc(128, TILE_N);
+        // The 128-token tile is issued as two 64-token halves with separate accumulators, so the MMAs of
+        // one half overlap the epilogue of the other and of the previous tile.
+        constexpr uint32_t idesc = make_idesc(128, EPI_TOK);
         bool ok = true;
         if (lane == 0) {
-            for (int it = 0; it < n_my_tiles; ++it) {
+            for (int it = 0; it < n_my_tiles && ok; ++it) {
                 const int st = it % US;
                 ok = mbar_wait(BAR_UFULL(st), (it / US) & 1, spin, abort_flag);
                 if (!ok) break;
-                ok = mbar_wait(BAR_ACCEMPTY, (it & 1) ^ 1, spin, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
                 const uint32_t u_base = base + SMEM_U + st * U_STAGE_BYTES;
+                for (int kh = 0; kh < 2; ++kh) {
+                    ok = mbar_wait(BAR_ACCEMPTY(kh), (it & 1) ^ 1, spin, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    // rows kh*64 .. kh*64+63 of every K block; the start-address field of the descriptor counts 16-byte units
+                    const uint64_t bd0 = make_desc_sw128(u_base + (uint32_t)kh * EPI_TOK * 128u);
+                    const uint32_t acc = tmem + kh * EPI_TOK;
 #pragma unroll
-                for (int ks = 0; ks < DH / 16; ++ks) {
-                    const uint64_t bd = make_desc_sw128(u_base + (ks >> 2) * U_KBLOCK_BYTES + (ks & 3) * 32);
-                    mma_ts(tmem + TM_ACC_A, tmem + TM_W_A + ks * 8, bd, idesc, ks > 0);
-                    mma_ts(tmem + TM_ACC_X, tmem + TM_W_X + ks * 8, bd, idesc, ks > 0);
+                    for (int ks = 0; ks < DH / 16; ++ks) {
+                        const uint64_t bd = bd0 + (uint64_t)(((ks >> 2) * U_KBLOCK_BYTES + (ks & 3) * 32) >> 4);
+                        mma_ts(acc + TM_ACC_A, tmem + TM_W_A + ks * 8, bd, idesc, ks > 0);
+                        mma_ts(acc + TM_ACC_X, tmem + TM_W_X + ks * 8, bd, idesc, ks > 0);
+                    }
+                    if (kh == 1) tc_commit(BAR_UEMPTY(st));
+                    tc_commit(BAR_ACCFULL(kh));
                 }
-                tc_commit(BAR_UEMPTY(st));
-                tc_commit(BAR_ACCFULL);
             }
             if (!ok) record_timeout(f.status, abort_flag);
         }
@@ -468,7 +471,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
       }
     } else {
         // ================================================================ epilogue
-        reg_inc<208>();
+        reg_inc<200>();
         const int q = warp & 3, k = (warp - 8) >> 2;
         const int c_own = q * 32 + lane;                 // channel within the CTA
         const int hc = half * CH + c_own;                // channel within the head
@@ -491,14 +494,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         __nv_bfloat16 *y = (__nv_bfloat16 *)f.y;
         const __nv_bfloat16 *x = (const __nv_bfloat16 *)f.x;
         const __nv_bfloat16 *cs_in = (const __nv_bfloat16 *)f.cs_in;
-        float h_prev_own = 0.0f;  // k == 0: state after this CTA's previous tile
+        float h_prev_own = 0.0f;  // state at the end of this CTA's previous tile
         bool ok = true;
         for (int it = 0; it < n_my_tiles && ok; ++it) {
             const int g = kcta + it * S, b = g / p.tps, ti = g % p.tps;
             const int t0 = ti * TILE_N;
             const int st = it % US;
             const int nv = max(0, min(EPI_TOK, T - t0 - k * EPI_TOK));  // valid tokens of this warp
-            ok = warp_wait(BAR_ACCFULL, it & 1, spin, abort_flag);
+            ok = warp_wait(BAR_ACCFULL(k), it & 1, spin, abort_flag);
             if (!ok) break;
             tc_fence_after();
             // A2[j] / V2[j]: tokens j (low half) and j + 32 (high half) of this warp's 64 tokens
@@ -510,7 +513,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(BAR_ACCEMPTY);  // the accumulators now live in registers
+            if (lane == 0) mbar_arrive(BAR_ACCEMPTY(k));  // the accumulators now live in registers
             // gates, decay, input scale: (z_a, z_x) -> (a_t, v_t) in place
             const uint8_t *u_tile = smem + SMEM_U + st * U_STAGE_BYTES;
             auto gates = [&](auto poly_tag) {
@@ -541,79 +544,69 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             for (int j = 0; j < EPI_TOK / 2; ++j) { P2 = mul2(P2, A2[j]); HL2 = fma2(A2[j], HL2, V2[j]); }
             const float P_lo = lo2(P2), hl_lo = lo2(HL2);
             const float P = P_lo * hi2(P2), hl = fmaf(hi2(P2), hl_lo, hi2(HL2));
-            // ---- incoming state
+            // ---- the two halves of the tile exchange their folds; the second half publishes the tile's
+            agg_s[(((it & 1) * 2 + k) * 4 + q) * 32 + lane] = make_float2(P, hl);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(BAR_AGG(q, k));
+            ok = warp_wait(BAR_AGG(q, k ^ 1), it & 1, spin, abort_flag);
+            if (!ok) break;
+            const float2 other = agg_s[(((it & 1) * 2 + (k ^ 1)) * 4 + q) * 32 + lane];
+            const float P_0 = k ? other.x : P, hl_0 = k ? other.y : hl;     // tokens [0, 64)
+            const float P_1 = k ? P : other.x, hl_1 = k ? hl : other.y;     // tokens [64, 128)
+            const float P_t = P_0 * P_1, hl_t = fmaf(P_1, hl_0, hl_1);      // whole tile
+            if (S > 1 && k == 1) {
+                uint4 rec;
+                rec.x = __float_as_uint(P_t); rec.y = p.tag; rec.z = __float_as_uint(hl_t); rec.w = p.tag;
+                uint4 *dst = p.agg + ((size_t)group * p.tiles_total + g) * CH + c_own;
+                asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "r"(rec.x), "r"(rec.y), "r"(rec.z), "r"(rec.w) : "memory");
+            }
+            // ---- incoming state of the tile (both halves work it out for themselves): the state this CTA
+            //      reached at the end of its previous tile, or h0 near the start of a sequence, advanced by
+            //      the aggregates that the other CTAs published for the tiles in between (decoupled look-back)
             float h;
-            if (S > 1) {
-                if (k == 0) {
-                    agg_s[((it & 1) * 4 + q) * 32 + lane] = make_float2(P, hl);
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(BAR_AGG(q));
-                } else {
-                    ok = warp_wait(BAR_AGG(q), it & 1, spin, abort_flag);
-                    if (!ok) break;
-                    const float2 a0 = agg_s[((it & 1) * 4 + q) * 32 + lane];
-                    const float Pt = P * a0.x, hlt = fmaf(P, a0.y, hl);
-                    uint4 rec;
-                    rec.x = __float_as_uint(Pt); rec.y = p.tag; rec.z = __float_as_uint(hlt); rec.w = p.tag;
-                    uint4 *dst = p.agg + ((size_t)group * p.tiles_total + g) * CH + c_own;
-                    asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "r"(rec.x), "r"(rec.y), "r"(rec.z), "r"(rec.w) : "memory");
-                }
-            }
-            if (k == 0) {
-                if (it > 0) {  // state after this CTA's previous tile (written by the k == 1 warp)
-                    ok = warp_wait(BAR_CHAIN(q, 0), (it - 1) & 1, spin, abort_flag);
-                    if (!ok) break;
-                    h_prev_own = h_s[(q * 2 + 0) * 32 + lane];
-                }
-                int nback;
-                if (ti == 0 || (S > 1 && ti < S)) {
-                    h = f.h0 ? f.h0[(size_t)b * D + d] : 0.0f;
-                    nback = ti;
-                } else {
-                    h = h_prev_own;
-                    nback = S - 1;
-                }
-                // decoupled look-back: the aggregates of the (at most MAX_S - 1) tiles between that state and
-                // this tile.  All records are requested at once, then polled until every lane sees this
-                // call's tag in both halves of each record (8-byte words are written atomically).
-                if (nback > 0) {
-                    const uint4 *src = p.agg + ((size_t)group * p.tiles_total + g) * CH + c_own;
-                    uint4 rec[MAX_S - 1];
-                    uint64_t tstart = 0;
-                    for (uint32_t npoll = 0;; ++npoll) {
-                        bool ready = true;
-#pragma unroll
-                        for (int j = 1; j < MAX_S; ++j) {
-                            if (j <= nback) {
-                                const uint4 *sj = src - (size_t)j * CH;
-                                asm volatile("ld.volatile.global.v4.b32 {%0, %1, %2, %3}, [%4];"
-                                             : "=r"(rec[j - 1].x), "=r"(rec[j - 1].y), "=r"(rec[j - 1].z), "=r"(rec[j - 1].w) : "l"(sj) : "memory");
-                            }
-                        }
-#pragma unroll
-                        for (int j = 1; j < MAX_S; ++j)
-                            if (j <= nback) ready = ready && rec[j - 1].y == p.tag && rec[j - 1].w == p.tag;
-                        if (__all_sync(0xffffffffu, ready)) break;
-                        if ((npoll & 15u) == 15u) {
-                            const uint64_t tnow = gtimer();
-                            if (tstart == 0) tstart = tnow;
-                            if (*abort_flag || tnow - tstart > spin) { ok = false; break; }
-                        }
-                        __nanosleep(64);
-                    }
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (ok) {
-#pragma unroll
-                        for (int j = MAX_S - 1; j >= 1; --j)
-                            if (j <= nback) h = fmaf(__uint_as_float(rec[j - 1].x), h, __uint_as_float(rec[j - 1].z));
-                    }
-                }
-                if (!ok) break;
+            int nback;
+            if (ti == 0 || (S > 1 && ti < S)) {
+                h = f.h0 ? f.h0[(size_t)b * D + d] : 0.0f;
+                nback = ti;
             } else {
-                ok = warp_wait(BAR_CHAIN(q, 1), it & 1, spin, abort_flag);
-                if (!ok) break;
-                h = h_s[(q * 2 + 1) * 32 + lane];
+                h = h_prev_own;
+                nback = S - 1;
             }
+            if (nback > 0) {
+                // All records are requested at once, then polled until every lane sees this call's tag in
+                // both halves of each record (8-byte words are written atomically).
+                const uint4 *src = p.agg + ((size_t)group * p.tiles_total + g) * CH + c_own;
+                uint4 rec[MAX_S - 1];
+                uint64_t tstart = 0;
+                for (uint32_t npoll = 0;; ++npoll) {
+                    bool ready = true;
+#pragma unroll
+                    for (int j = 1; j < MAX_S; ++j) {
+                        if (j <= nback) {
+                            const uint4 *sj = src - (size_t)j * CH;
+                            asm volatile("ld.volatile.global.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                         : "=r"(rec[j - 1].x), "=r"(rec[j - 1].y), "=r"(rec[j - 1].z), "=r"(rec[j - 1].w) : "l"(sj) : "memory");
+                        }
+                    }
+#pragma unroll
+                    for (int j = 1; j < MAX_S; ++j)
+                        if (j <= nback) ready = ready && rec[j - 1].y == p.tag && rec[j - 1].w == p.tag;
+                    if (__all_sync(0xffffffffu, ready)) break;
+                    if ((npoll & 15u) == 15u) {
+                        const uint64_t tnow = gtimer();
+                        if (tstart == 0) tstart = tnow;
+                        if (*abort_flag || tnow - tstart > spin) { ok = false; break; }
+                    }
+                    __nanosleep(32);
+                }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+#pragma unroll
+                for (int j = MAX_S - 1; j >= 1; --j)
+                    if (j <= nback) h = fmaf(__uint_as_float(rec[j - 1].x), h, __uint_as_float(rec[j - 1].z));
+            }
+            h_prev_own = fmaf(P_t, h, hl_t);          // state at the end of this tile
+            if (k == 1) h = fmaf(P_0, h, hl_0);       // state at the start of the second half
             // ---- the y staging rows of this half must have been read out by the previous tile's bulk stores
             if (it > 0) {
                 if (q == 0 && lane == 0) bulk_wait_read0();
@@ -633,11 +626,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
                 y_s[(j + 32) * (Y_ROW_BYTES / 2)] = (uint16_t)(ow >> 16);
             }
             h = hi2(H2);
-            // ---- hand the state on
-            h_s[(q * 2 + (k ^ 1)) * 32 + lane] = h;
             fence_async_smem();   // y rows become visible to the bulk-copy engine
             __syncwarp();
-            if (lane == 0) { mbar_arrive(BAR_CHAIN(q, k ^ 1)); mbar_arrive(BAR_YFULL(k)); }
+            if (lane == 0) mbar_arrive(BAR_YFULL(k));
             if (k == 1 && ti == p.tps - 1) {
                 // end of a sequence: h_T (unrounded state) and the last three raw inputs, bit-exact
                 f.h_T[(size_t)b * D + d] = h;

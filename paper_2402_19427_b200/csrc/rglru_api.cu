@@ -126,7 +126,11 @@ int32_t rglru_decode_step(const rglru_shape_t *s, const rglru_params_t *p, const
     a.T = 1;
     a.x = x; a.y = y; a.h_T = h; a.cs_out = conv_state;
     a.status = (uint32_t *)workspace;
-    cudaError_t e = generic_decode(a, s->io, (cudaStream_t)cuda_stream);
+    cudaError_t e;
+    if (!(s->flags & RGLRU_FLAG_FORCE_GENERIC) && sm100_decode_supported(s->B, s->D, s->H, s->io))
+        e = sm100_decode(a, (cudaStream_t)cuda_stream);
+    else
+        e = generic_decode(a, s->io, (cudaStream_t)cuda_stream);
     return e == cudaSuccess ? RGLRU_OK : RGLRU_ERR_CUDA;
 }
 

@@ -2,6 +2,7 @@
 // Not part of the public ABI (that is include/rglru.h).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -61,5 +62,13 @@ cudaError_t generic_backward(const FwdArgs &fwd, BwdArgs &b, int io, void *ws_bo
 bool sm100_prefill_supported(int B, int T, int D, int H, int io);
 size_t sm100_prefill_workspace_bytes(int B, int T, int D, int H);
 cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes, cudaStream_t st);
+bool sm100_decode_supported(int B, int D, int H, int io);
+cudaError_t sm100_decode(const FwdArgs &a, cudaStream_t st);
+extern unsigned long long g_spin_limit_ns;  // every device-side wait gives up after this many nanoseconds
+// Tiled-TMA descriptor of a dense bf16 tensor [d2][d1][d0] (d0 innermost) with a box of box1 x box0 elements;
+// swizzle128 selects the 128-byte shared-memory swizzle that tcgen05.mma operands use.  False if the driver
+// entry point is unavailable or rejects the shape.
+bool encode_bf16_map_3d(CUtensorMap *tm, const void *ptr, uint64_t d0, uint64_t d1, uint64_t d2, uint32_t box0, uint32_t box1,
+                        bool swizzle128);
 
 }  // namespace rglru

@@ -1,0 +1,294 @@
+// sm_100a batched decode step of the RG-LRU temporal core (bf16 io, head width 256): one new token for each
+// of B sequences, recurrent state h [B,D] fp32 and the 3-row conv state [B,3,D] updated in place.
+//
+// A cluster of two CTAs owns one (head, batch tile) pair.  CTA r of the pair owns channels [128 r, 128 r + 128)
+// of the head, both as conv / state channels and as gate output channels:
+//   * its 2 x 128 rows of W_a, W_x arrive by tiled TMA in the 128-byte-swizzled K-major layout tcgen05.mma reads
+//     (the copy runs while the conv phase works);
+//   * all threads do the conv phase for the CTA's own 128 channels: one thread per (sequence, 8 channels) reads
+//     x and the three conv-state rows with 16-byte loads, writes the shifted conv state back (bit-exact copies),
+//     and stores the bf16 conv output u as one 16-byte swizzle chunk of the U tile, both into its own shared
+//     memory and into the peer CTA's (distributed shared memory), so that after one cluster barrier each CTA
+//     holds u for all 256 input channels.  Every conv-state element is read and written by exactly one thread.
+//     The rounding remainder u - bf16(u) is kept beside it (own channels only): the gate products take the
+//     bf16 value, the term i_t * u_t of Eq. 4 takes bf16(u) + remainder, which is u to 16 mantissa bits;
+//   * one thread issues Z^T = W U^T for both gates (M = 128 channels, N = sequences of the tile, K = 256) with
+//     fp32 accumulators in tensor memory;
+//   * all eight warps run the epilogue: channel on the TMEM lane, sequences along the columns; gates, log-space
+//     decay and h <- a h + sqrt(1 - a^2) (i u) in fp32, h and y written with lane-contiguous stores.
+// Waits on the two mbarriers are bounded and end in RGLRU_ERR_TIMEOUT; the only cluster barriers come before them.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "rglru_internal.h"
+#include "sm100_ptx.cuh"
+
+namespace rglru {
+namespace {
+
+using namespace ptx;
+
+constexpr int DH = 256;        // head width
+constexpr int CH = 128;        // channels per CTA
+constexpr int NB_MAX = 128;    // sequences per batch tile, at most
+constexpr int NTHREADS = 256;
+constexpr uint32_t KBLOCK_BYTES = 128 * 128;               // 128 rows x 64 bf16: one K block of an operand tile
+constexpr uint32_t SMEM_WA = 0;
+constexpr uint32_t SMEM_WX = SMEM_WA + 4 * KBLOCK_BYTES;
+constexpr uint32_t SMEM_U = SMEM_WX + 4 * KBLOCK_BYTES;
+constexpr uint32_t SMEM_R = SMEM_U + 4 * KBLOCK_BYTES;    // bf16 r_s[NB_MAX][CH]: u - bf16(u) for this CTA's channels
+constexpr uint32_t SMEM_BAR = SMEM_R + NB_MAX * CH * 2;   // two mbarriers
+constexpr uint32_t SMEM_MISC = SMEM_BAR + 16;             // tmem base
+constexpr uint32_t SMEM_TOTAL = SMEM_MISC + 16;
+constexpr uint32_t SMEM_ALLOC = SMEM_TOTAL + 1024;
+constexpr uint32_t TMEM_COLS = 256;                        // z_a in columns [0, NB), z_x in [128, 128 + NB)
+constexpr float S_POLY = 0.25f;                            // decay rates up to here use the polynomial for 1 - a_t
+
+struct DecArgs {
+    alignas(64) CUtensorMap tm_wa;   // W_a as [H][256 out][256 in], box 128 out x 64 in, 128-byte swizzle
+    alignas(64) CUtensorMap tm_wx;
+    FwdArgs f;
+    int NB;       // sequences per batch tile (multiple of 16)
+    int ntile;    // batch tiles
+    unsigned long long spin_ns;
+};
+
+__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *(const uint32_t *)&v;
+}
+
+// (z_a, z_x, u) -> (a_t, v_t) of Eq. 3-4 with the same formulation as the prefill kernel:
+//   r = 1/2 + 1/2 tanh((z_a + b_a)/2), x = 2 s r, f = 1 - a_t = -expm1(-x/2), sqrt(1 - a_t^2)/2 = sqrt(f (1/2 - f/4)),
+//   v = (sqrt(1 - a_t^2)/2 u)(1 + tanh((z_x + b_x)/2)).
+__device__ __forceinline__ void gate(float za, float zx, float u, float hba, float hbx, float s, bool poly, float &a, float &v) {
+    const float ta = tanh_approx(fmaf(za, 0.5f, hba));
+    const float x = fmaf(ta, s, s);
+    float f;
+    if (poly) {
+        float pl = fmaf(x, -1.0f / 384.0f, 1.0f / 48.0f);
+        pl = fmaf(pl, x, -0.125f);
+        pl = fmaf(pl, x, 0.5f);
+        f = pl * x;
+        a = 1.0f - f;
+    } else {
+        a = ex2_approx(x * -0.72134752f);
+        f = 1.0f - a;
+    }
+    const float mh = sqrt_approx(fmaxf(f * fmaf(f, -0.25f, 0.5f), 0.0f));
+    const float tx = tanh_approx(fmaf(zx, 0.5f, hbx));
+    const float g = mh * u;
+    v = fmaf(g, tx, g);
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_decode_kernel(const __grid_constant__ DecArgs p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;   // the same offset in both CTAs of the cluster
+    uint8_t *smem = smem_raw + (base - raw_addr);
+    const uint32_t BAR_W = base + SMEM_BAR, BAR_ACC = BAR_W + 8;
+    uint32_t *tmem_base_s = (uint32_t *)(smem + SMEM_MISC);
+
+    const FwdArgs &f = p.f;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int B = f.B, D = f.D, NB = p.NB;
+    const uint32_t rank = cluster_ctarank();
+    const int item = blockIdx.x >> 1, head = item % f.H, tile = item / f.H;
+    const int b0 = tile * NB;
+    const unsigned long long spin = p.spin_ns;
+    int timed_out = 0;
+    volatile int no_abort = 0;
+
+    if (tid == 0) {
+        mbar_init(BAR_W, 1);
+        mbar_init(BAR_ACC, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) { tmem_alloc(smem_u32(tmem_base_s), TMEM_COLS); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_base_s;
+    cluster_arrive();   // the peer must be running before anything is stored into its shared memory
+
+    // ---- this CTA's gate weights: 2 gates x 4 K blocks of [128 out rows x 64 in channels]
+    if (tid == 0) {
+        mbar_expect_tx(BAR_W, 8 * KBLOCK_BYTES);
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+            tma_load_3d(base + SMEM_WA + kb * KBLOCK_BYTES, &p.tm_wa, kb * 64, (int)rank * CH, head, BAR_W);
+            tma_load_3d(base + SMEM_WX + kb * KBLOCK_BYTES, &p.tm_wx, kb * 64, (int)rank * CH, head, BAR_W);
+        }
+    }
+
+    // ---- conv phase: thread = (8-channel chunk c, sequences n = tid/16, tid/16 + 16, ...)
+    {
+        const int c = tid & 15;
+        const int dl = (int)rank * CH + c * 8;          // channel within the head
+        const size_t d = (size_t)head * DH + dl;        // global channel
+        const __nv_bfloat16 *cw = (const __nv_bfloat16 *)f.conv_w;
+        uint4 w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) w[j] = *(const uint4 *)(cw + (size_t)j * D + d);
+        float cb[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) cb[e] = f.conv_b ? f.conv_b[d + e] : 0.0f;
+        const __nv_bfloat16 *x = (const __nv_bfloat16 *)f.x;
+        __nv_bfloat16 *cs = (__nv_bfloat16 *)f.cs_out;   // in/out
+        const uint32_t u_kb = SMEM_U + (uint32_t)(dl >> 6) * KBLOCK_BYTES;
+        const uint32_t chunk = (uint32_t)(dl & 63) >> 3;
+        cluster_wait();
+        const uint32_t peer_base = map_to_cta(base, rank ^ 1u);
+        for (int n = tid >> 4; n < NB; n += 16) {
+            const int b = b0 + n;
+            uint4 uo = make_uint4(0u, 0u, 0u, 0u);
+            if (b < B) {
+                const uint4 xv = *(const uint4 *)(x + (size_t)b * D + d);
+                uint4 *c0p = (uint4 *)(cs + ((size_t)b * 3 + 0) * D + d), *c1p = (uint4 *)(cs + ((size_t)b * 3 + 1) * D + d),
+                      *c2p = (uint4 *)(cs + ((size_t)b * 3 + 2) * D + d);
+                const uint4 r0 = *c0p, r1 = *c1p, r2 = *c2p;   // x_{t-3}, x_{t-2}, x_{t-1}
+                const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w}, a0[4] = {r0.x, r0.y, r0.z, r0.w}, a1[4] = {r1.x, r1.y, r1.z, r1.w},
+                               a2[4] = {r2.x, r2.y, r2.z, r2.w};
+                const uint32_t w0[4] = {w[0].x, w[0].y, w[0].z, w[0].w}, w1[4] = {w[1].x, w[1].y, w[1].z, w[1].w},
+                               w2[4] = {w[2].x, w[2].y, w[2].z, w[2].w}, w3[4] = {w[3].x, w[3].y, w[3].z, w[3].w};
+                uint32_t o[4], rem[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float ul = cb[2 * e], uh = cb[2 * e + 1];
+                    ul = fmaf(bf_lo(w0[e]), bf_lo(xw[e]), ul); uh = fmaf(bf_hi(w0[e]), bf_hi(xw[e]), uh);
+                    ul = fmaf(bf_lo(w1[e]), bf_lo(a2[e]), ul); uh = fmaf(bf_hi(w1[e]), bf_hi(a2[e]), uh);
+                    ul = fmaf(bf_lo(w2[e]), bf_lo(a1[e]), ul); uh = fmaf(bf_hi(w2[e]), bf_hi(a1[e]), uh);
+                    ul = fmaf(bf_lo(w3[e]), bf_lo(a0[e]), ul); uh = fmaf(bf_hi(w3[e]), bf_hi(a0[e]), uh);
+                    o[e] = pack_bf16(ul, uh);
+                    rem[e] = pack_bf16(ul - bf_lo(o[e]), uh - bf_hi(o[e]));
+                }
+                uo = make_uint4(o[0], o[1], o[2], o[3]);
+                *(uint4 *)(smem + SMEM_R + (uint32_t)n * (CH * 2) + (uint32_t)c * 16u) = make_uint4(rem[0], rem[1], rem[2], rem[3]);
+                *c0p = r1; *c1p = r2; *c2p = xv;   // the conv state moves up by one row: bit-exact copies
+            }
+            const uint32_t off = u_kb + (uint32_t)n * 128u + ((chunk ^ (uint32_t)(n & 7)) << 4);
+            *(uint4 *)(smem + off) = uo;
+            st_cluster_v4(peer_base + off, uo);
+        }
+    }
+    fence_async_all();   // generic-proxy writes (local and remote) before the tensor core reads them
+    cluster_arrive();
+    cluster_wait();      // both halves of the U tile are in place in both CTAs
+
+    // ---- gate products
+    if (tid == 0) {
+        if (mbar_wait(BAR_W, 0, spin, &no_abort)) {
+            fence_async_all();
+            tc_fence_after();
+            const uint32_t idesc = make_idesc(128, NB);
+#pragma unroll
+            for (int ks = 0; ks < DH / 16; ++ks) {
+                const uint32_t koff = (uint32_t)(ks >> 2) * KBLOCK_BYTES + (uint32_t)(ks & 3) * 32u;
+                const uint64_t bd = make_desc_sw128(base + SMEM_U + koff);
+                mma_ss(tmem, make_desc_sw128(base + SMEM_WA + koff), bd, idesc, ks > 0);
+                mma_ss(tmem + 128, make_desc_sw128(base + SMEM_WX + koff), bd, idesc, ks > 0);
+            }
+            tc_commit(BAR_ACC);
+        } else {
+            atomicExch(f.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
+        }
+    }
+    __syncwarp();
+
+    // ---- epilogue: warp (q, k) owns channels 32 q .. 32 q + 31 and half k of the tile's sequences
+    {
+        const int q = warp & 3, k = warp >> 2;
+        const int c_own = q * 32 + lane;
+        const int dl = (int)rank * CH + c_own;
+        const size_t d = (size_t)head * DH + dl;
+        const float lam = f.lambda[d];
+        const float zl = -lam;
+        const float s = f.c * (zl > 0.0f ? zl + log1pf(expf(-zl)) : log1pf(expf(zl)));
+        const bool poly = __all_sync(0xffffffffu, s <= S_POLY);
+        const float hba = 0.5f * f.b_a[d], hbx = 0.5f * f.b_x[d];
+        const uint8_t *u_col = smem + SMEM_U + (uint32_t)(dl >> 6) * KBLOCK_BYTES + (uint32_t)(dl & 7) * 2u;
+        const uint32_t u_chunk = (uint32_t)(dl & 63) >> 3;
+        const uint8_t *r_col = smem + SMEM_R + (uint32_t)c_own * 2u;
+        float *h = f.h_T;                                 // in/out
+        __nv_bfloat16 *y = (__nv_bfloat16 *)f.y;
+        const int nh = NB >> 1;                           // multiple of 8
+        const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16);
+        if (!warp_wait(BAR_ACC, 0, spin, &no_abort)) {
+            timed_out = 1;
+        } else {
+            tc_fence_after();
+            for (int n0 = k * nh; n0 < (k + 1) * nh; n0 += 8) {
+                float hv[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int b = b0 + n0 + j;
+                    hv[j] = b < B ? h[(size_t)b * D + d] : 0.0f;
+                }
+                float za[8], zx[8];
+                tmem_ld8(tm_lane + n0, za);
+                tmem_ld8(tm_lane + 128 + n0, zx);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int n = n0 + j, b = b0 + n;
+                    const uint32_t ub = *(const uint16_t *)(u_col + (uint32_t)n * 128u + ((u_chunk ^ (uint32_t)(n & 7)) << 4));
+                    const uint32_t rb = *(const uint16_t *)(r_col + (uint32_t)n * (CH * 2));
+                    float a, v;
+                    gate(za[j], zx[j], __uint_as_float(ub << 16) + __uint_as_float(rb << 16), hba, hbx, s, poly, a, v);
+                    const float hn = fmaf(a, hv[j], v);
+                    if (b < B) {
+                        h[(size_t)b * D + d] = hn;
+                        y[(size_t)b * D + d] = __float2bfloat16_rn(hn);
+                    }
+                }
+            }
+        }
+        if (__any_sync(0xffffffffu, timed_out) && lane == 0) atomicExch(f.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
+}
+
+int num_sms() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) return n;
+    return 148;
+}
+
+}  // namespace
+
+bool sm100_decode_supported(int B, int D, int H, int io) { return io == RGLRU_BF16 && B > 0 && H > 0 && D == H * DH; }
+
+cudaError_t sm100_decode(const FwdArgs &a, cudaStream_t st) {
+    static bool attr_set = false;
+    cudaError_t e;
+    if (!attr_set) {
+        e = cudaFuncSetAttribute(sm100_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    DecArgs p;
+    if (!encode_bf16_map_3d(&p.tm_wa, a.W_a, DH, DH, (uint64_t)a.H, 64, CH, true) ||
+        !encode_bf16_map_3d(&p.tm_wx, a.W_x, DH, DH, (uint64_t)a.H, 64, CH, true))
+        return cudaErrorNotSupported;
+    p.f = a;
+    // batch tile: as few tiles per head as fill the SM pairs once, rounded to the MMA's N granularity
+    const int pairs = num_sms() / 2;
+    const int tiles_wanted = pairs / a.H > 0 ? pairs / a.H : 1;
+    int NB = (a.B + tiles_wanted - 1) / tiles_wanted;
+    NB = ((NB + 15) / 16) * 16;
+    if (NB > NB_MAX) NB = NB_MAX;
+    if (NB < 16) NB = 16;
+    p.NB = NB;
+    p.ntile = (a.B + NB - 1) / NB;
+    p.spin_ns = g_spin_limit_ns;
+    dim3 grid(2u * (unsigned)a.H * (unsigned)p.ntile), block(NTHREADS);
+    sm100_decode_kernel<<<grid, block, SMEM_ALLOC, st>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace rglru

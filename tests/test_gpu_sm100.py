@@ -90,3 +90,41 @@ def test_status_ok_and_repeatable():
     assert binding.query_status(ws) == binding.OK
     for y, hT in outs[1:]:
         assert torch.equal(y, outs[0][0]) and torch.equal(hT, outs[0][1])   # same reduction order every run
+
+
+@pytest.mark.parametrize("B,H,T0,steps", [(1, 1, 4, 5), (19, 1, 6, 9), (130, 2, 3, 4), (77, 3, 1, 3), (300, 1, 2, 2)])
+def test_decode_chain_equals_oracle_prefill(oracle, B, H, T0, steps):
+    """Tensor-core decode step (cluster pair per head and batch tile): prefill of T0 tokens, then chained
+    single-token steps; outputs, final h and the shifted conv state against the oracle's prefill of T0 + steps."""
+    import torch
+    from paper_2402_19427_b200 import binding
+    D = 256 * H
+    inp = synth.make_inputs(B, T0 + steps, D, H, io="bf16", seed=700 + B, bias_scale=0.3)
+    params = binding.Params.from_numpy(inp["params"], "bf16")
+    x = to_dev(inp["x"], "bf16")
+    _, h, cs = binding.prefill(x[:, :T0].contiguous(), params)
+    ys = [binding.decode_step(x[:, t].contiguous(), params, h, cs) for t in range(T0, T0 + steps)]
+    torch.cuda.synchronize()
+    yr, hr, cr = oracle_prefill(oracle, inp)
+    assert_close("y", np.stack([to_np(v) for v in ys], 1), yr[:, T0:], "bf16")
+    assert_close("h", to_np(h), hr, "bf16")
+    assert np.array_equal(to_np(cs), cr)
+
+
+def test_decode_agrees_with_generic_decode_and_status():
+    import torch
+    from paper_2402_19427_b200 import binding
+    B, H = 48, 2
+    inp = synth.make_inputs(B, 4, 256 * H, H, io="bf16", seed=33, with_state=True, bias_scale=0.2)
+    params = binding.Params.from_numpy(inp["params"], "bf16")
+    x = to_dev(inp["x"], "bf16")
+    outs = []
+    for flags in (0, 1):
+        h = to_dev(inp["h0"]); cs = to_dev(inp["conv_state"], "bf16")
+        ws = binding.alloc_workspace(binding.make_shape(B, 1, 256 * H, H, torch.bfloat16), binding.OP_DECODE, x.device)
+        ys = [binding.decode_step(x[:, t].contiguous(), params, h, cs, flags=flags, workspace=ws) for t in range(4)]
+        assert binding.query_status(ws) == binding.OK
+        outs.append((torch.stack(ys, 1), h, cs))
+    assert_close("y", to_np(outs[0][0]), to_np(outs[1][0]), "bf16")
+    assert_close("h", to_np(outs[0][1]), to_np(outs[1][1]), "bf16")
+    assert torch.equal(outs[0][2], outs[1][2])

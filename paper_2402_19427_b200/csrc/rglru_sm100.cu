@@ -161,14 +161,24 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
     const uint32_t tmem = *tmem_base_s;
 
     // Gate weights of this half-head into tensor memory: lane = output channel, 32-bit column j holds
-    // input channels 2j (low half) and 2j+1 (high half), i.e. consecutive bf16 of the row as stored.
+    // input channels 2j (low half) and 2j+1 (high half).  The tensor core multiplies them with the conv output
+    // u, which is kept in fp16 (11 significant bits instead of bf16's 8, because u also enters i_t * u_t of
+    // Eq. 4 directly), and both operands of one MMA must have one type: the bf16 weights are converted to
+    // fp16 here, which is exact for every weight of magnitude within [2^-14, 65504] and rounds tinier ones
+    // to a multiple of 2^-24.
     if (warp >= 8) {
         const int q = warp & 3, g = (warp - 8) >> 2;  // g = 0: W_a, 1: W_x
         const __nv_bfloat16 *W = (const __nv_bfloat16 *)(g ? f.W_x : f.W_a);
         const uint4 *row = (const uint4 *)(W + ((size_t)head * DH + half * CH + q * 32 + lane) * DH);
         const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (g ? TM_W_X : TM_W_A);
+        auto cvt2 = [](uint32_t w) { return pack_f16_sat(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u)); };
 #pragma unroll 4
-        for (int c = 0; c < 16; ++c) tmem_st8(taddr + c * 8, __ldg(row + 2 * c), __ldg(row + 2 * c + 1));
+        for (int c = 0; c < 16; ++c) {
+            uint4 lo = __ldg(row + 2 * c), hi = __ldg(row + 2 * c + 1);
+            lo.x = cvt2(lo.x); lo.y = cvt2(lo.y); lo.z = cvt2(lo.z); lo.w = cvt2(lo.w);
+            hi.x = cvt2(hi.x); hi.y = cvt2(hi.y); hi.z = cvt2(hi.z); hi.w = cvt2(hi.w);
+            tmem_st8(taddr + c * 8, lo, hi);
+        }
         tmem_st_wait();
     }
     tc_fence_before();
@@ -241,9 +251,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
                         u01 = fma2(w01[1], xc01, u01); u23 = fma2(w23[1], xc23, u23);
                         u01 = fma2(w01[2], xb01, u01); u23 = fma2(w23[2], xb23, u23);
                         u01 = fma2(w01[3], xa01, u01); u23 = fma2(w23[3], xa23, u23);
-                        __nv_bfloat162 o01 = __floats2bfloat162_rn(lo2(u01), hi2(u01));
-                        __nv_bfloat162 o23 = __floats2bfloat162_rn(lo2(u23), hi2(u23));
-                        *(uint2 *)(smem + sw[i & 3] + (uint32_t)i * 256u) = make_uint2(*(uint32_t *)&o01, *(uint32_t *)&o23);
+                        *(uint2 *)(smem + sw[i & 3] + (uint32_t)i * 256u) =
+                            make_uint2(pack_f16_sat(lo2(u01), hi2(u01)), pack_f16_sat(lo2(u23), hi2(u23)));
                         xa01 = d01; xa23 = d23;   // the oldest slot now holds the newest row
                     };
                     if (nvalid >= 16) {
@@ -263,10 +272,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
                             u01 = fma2(w01[1], c01, u01); u23 = fma2(w23[1], c23, u23);
                             u01 = fma2(w01[2], b01x, u01); u23 = fma2(w23[2], b23x, u23);
                             u01 = fma2(w01[3], a01, u01); u23 = fma2(w23[3], a23, u23);
-                            __nv_bfloat162 o01 = __floats2bfloat162_rn(lo2(u01), hi2(u01));
-                            __nv_bfloat162 o23 = __floats2bfloat162_rn(lo2(u23), hi2(u23));
                             const uint32_t addr = row_addr + ((u_chunk ^ ((pbit + 2u * (uint32_t)i) & 7u)) << 4) + (uint32_t)i * 256u;
-                            *(uint2 *)(smem + addr) = make_uint2(*(uint32_t *)&o01, *(uint32_t *)&o23);
+                            *(uint2 *)(smem + addr) = make_uint2(pack_f16_sat(lo2(u01), hi2(u01)), pack_f16_sat(lo2(u23), hi2(u23)));
                             a01 = b01x; a23 = b23x; b01x = c01; b23x = c23; c01 = d01; c23 = d23;
                         }
                     }
@@ -324,7 +331,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         // ================================================================ MMA issuer
         // The 128-token tile is issued as two 64-token halves with separate accumulators, so the MMAs of
         // one half overlap the epilogue of the other and of the previous tile.
-        constexpr uint32_t idesc = make_idesc(128, EPI_TOK);
+        constexpr uint32_t idesc = make_idesc_f16(128, EPI_TOK);
         bool ok = true;
         if (lane == 0) {
             for (int it = 0; it < n_my_tiles && ok; ++it) {
@@ -405,9 +412,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
 #pragma unroll
                 for (int j = 0; j < EPI_TOK / 2; ++j) {
                     // rows 2j (token j) and 2j + 1 (token j + 32)
-                    const uint32_t ub0 = *(const uint16_t *)(u_tile + u_off[(2 * j) & 7] + (uint32_t)(2 * j) * 128u);
-                    const uint32_t ub1 = *(const uint16_t *)(u_tile + u_off[(2 * j + 1) & 7] + (uint32_t)(2 * j + 1) * 128u);
-                    gate_pair<POLY>(A2[j], V2[j], __uint_as_float(ub0 << 16), __uint_as_float(ub1 << 16), hba2, hbx2, s2);
+                    const uint16_t ub0 = *(const uint16_t *)(u_tile + u_off[(2 * j) & 7] + (uint32_t)(2 * j) * 128u);
+                    const uint16_t ub1 = *(const uint16_t *)(u_tile + u_off[(2 * j + 1) & 7] + (uint32_t)(2 * j + 1) * 128u);
+                    gate_pair<POLY>(A2[j], V2[j], f16_bits_to_f32(ub0), f16_bits_to_f32(ub1), hba2, hbx2, s2);
                 }
             };
             if (poly) gates(std::true_type{}); else gates(std::false_type{});

@@ -25,7 +25,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2402_19427_b200 import inputs as synth  # noqa: E402
+from paper_2402_19427_b200 import inputs as synth, sharding  # noqa: E402
 
 WORKLOAD = 1                 # index into synth.CONFIGS: the training-shape prefill
 N_ROTATE = 4                 # distinct input/output buffer sets cycled between steps (defeats L2 reuse)
@@ -103,44 +103,43 @@ class ClockSampler:
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def oracle_sample(cfg, seed):
-    """Bounded sample of the bench workload for the CPU oracle: every sequence, one head (heads are independent)."""
-    small = dict(cfg)
-    Dh = cfg["D"] // cfg["H"]
-    small.update(D=Dh, H=1)
-    inp = synth.make_inputs(small["B"], small["T"], Dh, 1, io=cfg["io"], seed=seed)
-    return inp, cfg["H"]
-
-
-def time_oracle(cfg, seed, repeats=1):
+def time_oracle(cfg, seed, heads):
+    """Times the fp64 oracle, as it stands, on `heads` of the workload's H heads for every sequence and token (heads are
+    independent, so this is heads/H of one step).  Returns (tokens/s scaled to full-width tokens, seconds, threads, text)."""
     import oracle
-    inp, head_div = oracle_sample(cfg, seed)
+    Dh = cfg["D"] // cfg["H"]
+    inp = synth.make_inputs(cfg["B"], cfg["T"], Dh * heads, heads, io=cfg["io"], seed=seed)
     p64 = {k: np.asarray(v, np.float64) for k, v in inp["params"].items()}
     x64 = inp["x"].astype(np.float64)
-    best = None
-    for _ in range(repeats):
-        t0 = time.perf_counter()
-        oracle.prefill(x64, p64, 1, c=inp["c"])
-        dt = time.perf_counter() - t0
-        best = dt if best is None else min(best, dt)
-    tokens_equiv = cfg["B"] * cfg["T"] / head_div      # full-width tokens' worth of work in the sample
-    return tokens_equiv / best, best, oracle.num_threads(), f"all {cfg['B']} sequences x {cfg['T']} tokens of 1 of {head_div} heads (1/{head_div} of a step), fp64"
+    t0 = time.perf_counter()
+    oracle.prefill(x64, p64, heads, c=inp["c"])
+    dt = time.perf_counter() - t0
+    tokens_equiv = cfg["B"] * cfg["T"] * heads / cfg["H"]      # full-width tokens' worth of work in the sample
+    what = (f"all {cfg['B']} sequences x {cfg['T']} tokens of {heads} of {cfg['H']} heads ({heads}/{cfg['H']} of a step), "
+            f"fp64, sequential in time")
+    return tokens_equiv / dt, dt, oracle.num_threads(), what
 
 
 def run_reference(args):
+    """The reference arm is the CPU oracle (there is no reference implementation to install).  Each step is a bounded
+    sample of the workload -- some of its heads -- sized so that the whole run stays within a few minutes."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     cfg = dict(synth.CONFIGS[WORKLOAD])
-    times = []
+    seed = synth.BASE_SEED + WORKLOAD
+    _, t_head, _, _ = time_oracle(cfg, seed, 1)               # untimed probe: cost of one head
+    budget_s = 150.0
+    heads = int(max(1, min(cfg["H"], budget_s / max(t_head, 1e-3) / (args.steps + args.warmup))))
+    times, sample, cores = [], "", 0
     for i in range(args.warmup + args.steps):
-        tps, dt, cores, sample = time_oracle(cfg, synth.BASE_SEED + WORKLOAD)
+        tps, dt, cores, sample = time_oracle(cfg, seed, heads)
         if i >= args.warmup:
             times.append(dt)
     mean_dt = float(np.mean(times))
-    value = cfg["B"] * cfg["T"] / cfg["H"] / mean_dt
+    value = cfg["B"] * cfg["T"] * heads / cfg["H"] / mean_dt
     line = {"impl": "reference", "metric": "rglru_prefill_tokens_per_s", "value": value, "unit": "tokens/s",
-            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": mean_dt * 1e3,
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": mean_dt * 1e3 * cfg["H"] / heads,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": workload_name(cfg)},
             "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
@@ -171,7 +170,7 @@ def run_ours(args):
     cfg = dict(synth.CONFIGS[WORKLOAD])
     B, T, D, H = cfg["B"], cfg["T"], cfg["D"], cfg["H"]
     dt = torch.bfloat16
-    base = synth.make_config(WORKLOAD, seed=synth.BASE_SEED + WORKLOAD + 1000 * rank)
+    base = synth.make_config(WORKLOAD, seed=sharding.rank_seed(synth.BASE_SEED + WORKLOAD, rank))
     params = binding.Params.from_numpy(base["params"], cfg["io"], device=dev)
     rng = np.random.Generator(np.random.PCG64(99 + rank))
     xs_host = [base["x"]] + [synth.round_to_bf16(rng.standard_normal((B, T, D), dtype=np.float32)) for _ in range(N_ROTATE - 1)]
@@ -209,10 +208,7 @@ def run_ours(args):
     status = binding.query_status(ws)
     if status != binding.OK:
         raise binding.RglruError(status, "device status after timed region")
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = sharding.max_over_ranks(total_ms, dist if world > 1 else None, dev)
     ms_per_step = total_ms / args.steps
     value = world * B * T / (ms_per_step * 1e-3)
 
@@ -237,10 +233,7 @@ def run_ours(args):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = sharding.max_over_ranks(e2e_ms, dist if world > 1 else None, dev)
     # the e2e result must be the same computation: spot check against the device-resident run
     torch.cuda.synchronize()
     k = (e2e_steps - 1) % 2
@@ -284,7 +277,7 @@ def run_ours(args):
                         "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps},
                 "roofline": roof}
         if world == 1 and not args.no_cpu_baseline:
-            tps, dt_s, cores, sample = time_oracle(cfg, synth.BASE_SEED + WORKLOAD)
+            tps, dt_s, cores, sample = time_oracle(cfg, synth.BASE_SEED + WORKLOAD, cfg["H"])   # one whole step
             line["cpu_baseline"] = {"value": tps, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample,
                                     "seconds": dt_s}
         line.update(extra)

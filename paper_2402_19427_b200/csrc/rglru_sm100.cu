@@ -84,37 +84,51 @@ __device__ __forceinline__ void record_timeout(uint32_t *status, volatile int *a
     atomicExch(status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
 }
 
-// (z_a, z_x) of two tokens of one channel, one token per half of the register pair -> (a_t, v_t) of
-// Eq. 3-4, in place.
+// (z_a, z_x) of two tokens of one channel, one token per half of each register pair -> (a_t, v_t) of Eq. 3-4,
+// in place, for W register pairs advanced in lock step (independent dependency chains side by side).
 //   r = sigmoid(z_a + b_a) = 1/2 + 1/2 tanh((z_a + b_a)/2),  x = 2 s r,  f = 1 - a_t = -expm1(-x/2),
 //   m/2 = sqrt(f (1/2 - f/4)) = sqrt(1 - a_t^2)/2,  v = (m/2 u)(1 + tanh((z_x + b_x)/2)) = m i u.
-template <bool POLY>
-__device__ __forceinline__ void gate_pair(f32x2 &za, f32x2 &zx, float u0, float u1, f32x2 hba2, f32x2 hbx2, f32x2 s2) {
-    const f32x2 HALF2 = pack2(0.5f, 0.5f);
-    f32x2 ta = fma2(za, HALF2, hba2);
-    ta = pack2(tanh_approx(lo2(ta)), tanh_approx(hi2(ta)));
-    const f32x2 x = fma2(ta, s2, s2);
-    f32x2 f, a;
+template <bool POLY, int W>
+__device__ __forceinline__ void gate_group(f32x2 *za, f32x2 *zx, const float *u, f32x2 hba2, f32x2 hbx2, f32x2 s2) {
+    const f32x2 HALF2 = pack2(0.5f, 0.5f), NEG1 = pack2(-1.0f, -1.0f), ONE2 = pack2(1.0f, 1.0f);
+    f32x2 ta[W], tx[W], x[W], f[W], q[W];
+#pragma unroll
+    for (int i = 0; i < W; ++i) { ta[i] = fma2(za[i], HALF2, hba2); tx[i] = fma2(zx[i], HALF2, hbx2); }
+#pragma unroll
+    for (int i = 0; i < W; ++i) ta[i] = pack2(tanh_approx(lo2(ta[i])), tanh_approx(hi2(ta[i])));
+#pragma unroll
+    for (int i = 0; i < W; ++i) tx[i] = pack2(tanh_approx(lo2(tx[i])), tanh_approx(hi2(tx[i])));
+#pragma unroll
+    for (int i = 0; i < W; ++i) x[i] = fma2(ta[i], s2, s2);
     if (POLY) {
         // f = x/2 - x^2/8 + x^3/48 - x^4/384  (|x| <= 2 S_POLY: relative truncation error < 4e-5)
-        f32x2 p = fma2(x, pack2(-1.0f / 384.0f, -1.0f / 384.0f), pack2(1.0f / 48.0f, 1.0f / 48.0f));
-        p = fma2(p, x, pack2(-0.125f, -0.125f));
-        p = fma2(p, x, HALF2);
-        f = mul2(p, x);
-        a = fma2(f, pack2(-1.0f, -1.0f), pack2(1.0f, 1.0f));
+        f32x2 p[W];
+#pragma unroll
+        for (int i = 0; i < W; ++i) p[i] = fma2(x[i], pack2(-1.0f / 384.0f, -1.0f / 384.0f), pack2(1.0f / 48.0f, 1.0f / 48.0f));
+#pragma unroll
+        for (int i = 0; i < W; ++i) p[i] = fma2(p[i], x[i], pack2(-0.125f, -0.125f));
+#pragma unroll
+        for (int i = 0; i < W; ++i) p[i] = fma2(p[i], x[i], HALF2);
+#pragma unroll
+        for (int i = 0; i < W; ++i) { f[i] = mul2(p[i], x[i]); za[i] = fma2(f[i], NEG1, ONE2); }
     } else {
-        const f32x2 e = mul2(x, pack2(-0.72134752f, -0.72134752f));  // -x/2 * log2(e)
-        a = pack2(ex2_approx(lo2(e)), ex2_approx(hi2(e)));
-        f = fma2(a, pack2(-1.0f, -1.0f), pack2(1.0f, 1.0f));
+#pragma unroll
+        for (int i = 0; i < W; ++i) {
+            const f32x2 e = mul2(x[i], pack2(-0.72134752f, -0.72134752f));  // -x/2 * log2(e)
+            za[i] = pack2(ex2_approx(lo2(e)), ex2_approx(hi2(e)));
+            f[i] = fma2(za[i], NEG1, ONE2);
+        }
     }
-    f32x2 q = mul2(f, fma2(f, pack2(-0.25f, -0.25f), HALF2));  // (1 - a^2)/4 = f (2 - f)/4
-    if (!POLY) q = pack2(fmaxf(lo2(q), 0.0f), fmaxf(hi2(q), 0.0f));  // a from ex2.approx may round above 1
-    const f32x2 mh = pack2(sqrt_approx(lo2(q)), sqrt_approx(hi2(q)));
-    f32x2 tx = fma2(zx, HALF2, hbx2);
-    tx = pack2(tanh_approx(lo2(tx)), tanh_approx(hi2(tx)));
-    const f32x2 g = mul2(mh, pack2(u0, u1));
-    za = a;
-    zx = fma2(g, tx, g);
+#pragma unroll
+    for (int i = 0; i < W; ++i) q[i] = mul2(f[i], fma2(f[i], pack2(-0.25f, -0.25f), HALF2));  // (1 - a^2)/4 = f (2 - f)/4
+    if (!POLY) {
+#pragma unroll
+        for (int i = 0; i < W; ++i) q[i] = pack2(fmaxf(lo2(q[i]), 0.0f), fmaxf(hi2(q[i]), 0.0f));  // a from ex2.approx may round above 1
+    }
+#pragma unroll
+    for (int i = 0; i < W; ++i) q[i] = pack2(sqrt_approx(lo2(q[i])), sqrt_approx(hi2(q[i])));
+#pragma unroll
+    for (int i = 0; i < W; ++i) { const f32x2 g = mul2(q[i], pack2(u[2 * i], u[2 * i + 1])); zx[i] = fma2(g, tx[i], g); }
 }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __grid_constant__ Sm100Args p) {
@@ -244,26 +258,31 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
                     f32x2 a01, a23, b01x, b23x, c01, c23;  // x_{t-3}, x_{t-2}, x_{t-1}
                     load_row(0, a01, a23); load_row(1, b01x, b23x); load_row(2, c01, c23);
                     if (zero_halo && tg == 0) { a01 = a23 = b01x = b23x = c01 = c23 = pack2(0.f, 0.f); }
-                    auto one_token = [&](int i, f32x2 &xa01, f32x2 &xa23, f32x2 &xb01, f32x2 &xb23, f32x2 &xc01, f32x2 &xc23) {
-                        f32x2 d01, d23;
-                        load_row(3 + i, d01, d23);
-                        f32x2 u01 = fma2(w01[0], d01, b01), u23 = fma2(w23[0], d23, b23);
-                        u01 = fma2(w01[1], xc01, u01); u23 = fma2(w23[1], xc23, u23);
-                        u01 = fma2(w01[2], xb01, u01); u23 = fma2(w23[2], xb23, u23);
-                        u01 = fma2(w01[3], xa01, u01); u23 = fma2(w23[3], xa23, u23);
-                        *(uint2 *)(smem + sw[i & 3] + (uint32_t)i * 256u) =
-                            make_uint2(pack_f16_sat(lo2(u01), hi2(u01)), pack_f16_sat(lo2(u23), hi2(u23)));
-                        xa01 = d01; xa23 = d23;   // the oldest slot now holds the newest row
-                    };
                     if (nvalid >= 16) {
-                        // three rotating history slots: the roles cycle with period 3, fully unrolled
+                        // four tokens at a time, tap by tap, so that eight independent FMA chains are in flight
+                        f32x2 h01[3] = {a01, b01x, c01}, h23[3] = {a23, b23x, c23};
 #pragma unroll
-                        for (int i = 0; i < 15; i += 3) {
-                            one_token(i, a01, a23, b01x, b23x, c01, c23);
-                            one_token(i + 1, b01x, b23x, c01, c23, a01, a23);
-                            one_token(i + 2, c01, c23, a01, a23, b01x, b23x);
+                        for (int i0 = 0; i0 < 16; i0 += 4) {
+                            f32x2 r01[7], r23[7];   // rows t-3 .. t+3 of the batch
+#pragma unroll
+                            for (int k = 0; k < 3; ++k) { r01[k] = h01[k]; r23[k] = h23[k]; }
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) load_row(3 + i0 + k, r01[3 + k], r23[3 + k]);
+                            f32x2 u01[4], u23[4];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) { u01[k] = fma2(w01[0], r01[3 + k], b01); u23[k] = fma2(w23[0], r23[3 + k], b23); }
+#pragma unroll
+                            for (int j = 1; j < 4; ++j) {
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) { u01[k] = fma2(w01[j], r01[3 + k - j], u01[k]); u23[k] = fma2(w23[j], r23[3 + k - j], u23[k]); }
+                            }
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                *(uint2 *)(smem + sw[(i0 + k) & 3] + (uint32_t)(i0 + k) * 256u) =
+                                    make_uint2(pack_f16_sat(lo2(u01[k]), hi2(u01[k])), pack_f16_sat(lo2(u23[k]), hi2(u23[k])));
+#pragma unroll
+                            for (int k = 0; k < 3; ++k) { h01[k] = r01[4 + k]; h23[k] = r23[4 + k]; }
                         }
-                        one_token(15, a01, a23, b01x, b23x, c01, c23);
                     } else {
                         for (int i = 0; i < nvalid; ++i) {
                             f32x2 d01, d23;
@@ -410,11 +429,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             auto gates = [&](auto poly_tag) {
                 constexpr bool POLY = decltype(poly_tag)::value;
 #pragma unroll
-                for (int j = 0; j < EPI_TOK / 2; ++j) {
-                    // rows 2j (token j) and 2j + 1 (token j + 32)
-                    const uint16_t ub0 = *(const uint16_t *)(u_tile + u_off[(2 * j) & 7] + (uint32_t)(2 * j) * 128u);
-                    const uint16_t ub1 = *(const uint16_t *)(u_tile + u_off[(2 * j + 1) & 7] + (uint32_t)(2 * j + 1) * 128u);
-                    gate_pair<POLY>(A2[j], V2[j], f16_bits_to_f32(ub0), f16_bits_to_f32(ub1), hba2, hbx2, s2);
+                for (int j = 0; j < EPI_TOK / 2; j += 4) {
+                    float u[8];   // rows 2j' (token j') and 2j' + 1 (token j' + 32) for j' = j .. j + 3
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        u[e] = f16_bits_to_f32(*(const uint16_t *)(u_tile + u_off[(2 * j + e) & 7] + (uint32_t)(2 * j + e) * 128u));
+                    gate_group<POLY, 4>(A2 + j, V2 + j, u, hba2, hbx2, s2);
                 }
             };
             if (poly) gates(std::true_type{}); else gates(std::false_type{});

@@ -11,7 +11,17 @@ namespace ptx {
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ uint64_t gtimer() { uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+// Nanosecond timer shared by all SMs.  The 64-bit value is assembled from two 32-bit halves that are re-read until
+// the high half is stable, so a reading taken while the low half wraps (every 4.29 s) cannot be off by 2^32 ns.
+__device__ __forceinline__ uint64_t gtimer() {
+    uint32_t hi0, lo, hi1;
+    do {
+        asm volatile("mov.u32 %0, %%globaltimer_hi;" : "=r"(hi0));
+        asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(lo));
+        asm volatile("mov.u32 %0, %%globaltimer_hi;" : "=r"(hi1));
+    } while (hi0 != hi1);
+    return ((uint64_t)hi1 << 32) | lo;
+}
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }

@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "librglru_b200.so")
-SOURCES = ["rglru_api.cu", "rglru_generic.cu", "rglru_sm100.cu", "rglru_sm100_decode.cu", "rglru_static_scratch.cu"]
+SOURCES = ["rglru_api.cu", "rglru_generic.cu", "rglru_sm100.cu", "rglru_sm100_decode.cu", "rglru_sm100_bwd.cu", "rglru_static_scratch.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 

@@ -40,6 +40,10 @@ bool use_sm100_prefill(const rglru_shape_t *s) {
     return !(s->flags & RGLRU_FLAG_FORCE_GENERIC) && sm100_prefill_supported(s->B, s->T, s->D, s->H, s->io);
 }
 
+bool use_sm100_backward(const rglru_shape_t *s) {
+    return !(s->flags & RGLRU_FLAG_FORCE_GENERIC) && sm100_backward_supported(s->B, s->T, s->D, s->H, s->io);
+}
+
 FwdArgs make_fwd(const rglru_shape_t *s, const rglru_params_t *p) {
     FwdArgs a{};
     a.B = s->B; a.T = s->T; a.D = s->D; a.H = s->H; a.c = s->c;
@@ -77,7 +81,10 @@ size_t rglru_workspace_bytes(const rglru_shape_t *s, int32_t op) {
             if (use_sm100_prefill(s)) body = sm100_prefill_workspace_bytes(s->B, s->T, s->D, s->H);
             break;
         case RGLRU_OP_DECODE: break;
-        case RGLRU_OP_BACKWARD: body = generic_backward_workspace_bytes(s->B, s->T, s->D, s->H); break;
+        case RGLRU_OP_BACKWARD:
+            body = use_sm100_backward(s) ? sm100_backward_workspace_bytes(s->B, s->T, s->D, s->H)
+                                         : generic_backward_workspace_bytes(s->B, s->T, s->D, s->H);
+            break;
         default: return 0;
     }
     return WS_HEADER_BYTES + body;
@@ -158,7 +165,12 @@ int32_t rglru_backward(const rglru_shape_t *s, const rglru_params_t *p, const vo
     q.x = x; q.conv_w = p->conv_w; q.W_a = p->W_a; q.W_x = p->W_x; q.cs_in = conv_state_in; q.dy = dy;
     q.lambda = p->lambda; q.dx = dx;
     q.dconv_w = dconv_w; q.dconv_b = dconv_b; q.dW_a = dW_a; q.db_a = db_a; q.dW_x = dW_x; q.db_x = db_x; q.dlambda = dlambda;
-    cudaError_t e = generic_backward(f, q, s->io, (char *)workspace + WS_HEADER_BYTES, (cudaStream_t)cuda_stream);
+    cudaError_t e;
+    if (use_sm100_backward(s))
+        e = sm100_backward(f, q, y, (char *)workspace + WS_HEADER_BYTES, workspace_bytes - WS_HEADER_BYTES, (uint32_t *)workspace,
+                           (cudaStream_t)cuda_stream);
+    else
+        e = generic_backward(f, q, s->io, (char *)workspace + WS_HEADER_BYTES, (cudaStream_t)cuda_stream);
     return e == cudaSuccess ? RGLRU_OK : RGLRU_ERR_CUDA;
 }
 

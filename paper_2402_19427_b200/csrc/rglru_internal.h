@@ -70,5 +70,16 @@ extern unsigned long long g_spin_limit_ns;  // every device-side wait gives up a
 // entry point is unavailable or rejects the shape.
 bool encode_bf16_map_3d(CUtensorMap *tm, const void *ptr, uint64_t d0, uint64_t d1, uint64_t d2, uint32_t box0, uint32_t box1,
                         bool swizzle128);
+// The general form for any 16-bit element type: dims (innermost first), byte strides of dims 1 and 2, box extents.
+bool encode_map16_3d(CUtensorMap *tm, const void *ptr, const uint64_t dims[3], const uint64_t strides_bytes[2], const uint32_t box[3],
+                     bool swizzle128);
+// ---- sm_100a backward (bf16 io, D_h = 256, T a multiple of 8): tensor-core GEMMs around element-wise scan kernels
+bool sm100_backward_supported(int B, int T, int D, int H, int io);
+size_t sm100_backward_workspace_bytes(int B, int T, int D, int H);
+cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &b, const void *y_saved, void *ws_body, size_t ws_body_bytes, uint32_t *status,
+                           cudaStream_t st);
+// pieces of the generic backward that the tensor-core backward reuses (du in b.hp -> dx and conv gradients; fixed-order sums)
+cudaError_t generic_bwd_conv_and_reduce(BwdArgs &q, int io, cudaStream_t st);
+cudaError_t reduce_partials(const float *in, int nparts, size_t stride, float *out, size_t n, cudaStream_t st);
 
 }  // namespace rglru

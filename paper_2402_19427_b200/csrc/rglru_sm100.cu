@@ -623,17 +623,24 @@ uint32_t next_tag() {
 
 unsigned long long g_spin_limit_ns = 2000000000ull;  // bounded waits give up after this long
 
-bool encode_bf16_map_3d(CUtensorMap *tm, const void *ptr, uint64_t d0, uint64_t d1, uint64_t d2, uint32_t box0, uint32_t box1,
-                        bool swizzle128) {
+bool encode_map16_3d(CUtensorMap *tm, const void *ptr, const uint64_t dims[3], const uint64_t strides_bytes[2], const uint32_t box[3],
+                     bool swizzle128) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (enc == nullptr) return false;
-    const cuuint64_t dims[3] = {d0, d1, d2};
-    const cuuint64_t strides[2] = {d0 * 2, d0 * d1 * 2};
-    const cuuint32_t box[3] = {box0, box1, 1};
+    const cuuint64_t d[3] = {dims[0], dims[1], dims[2]};
+    const cuuint64_t st[2] = {strides_bytes[0], strides_bytes[1]};
+    const cuuint32_t bx[3] = {box[0], box[1], box[2]};
     const cuuint32_t estr[3] = {1, 1, 1};
-    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), d, st, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool encode_bf16_map_3d(CUtensorMap *tm, const void *ptr, uint64_t d0, uint64_t d1, uint64_t d2, uint32_t box0, uint32_t box1,
+                        bool swizzle128) {
+    const uint64_t dims[3] = {d0, d1, d2}, strides[2] = {d0 * 2, d0 * d1 * 2};
+    const uint32_t box[3] = {box0, box1, 1};
+    return encode_map16_3d(tm, ptr, dims, strides, box, swizzle128);
 }
 
 bool sm100_prefill_supported(int B, int T, int D, int H, int io) {

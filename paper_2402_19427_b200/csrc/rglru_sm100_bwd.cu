@@ -1,0 +1,486 @@
+// sm_100a backward of the RG-LRU temporal core (bf16 io, head width 256, T a multiple of 8).
+//
+// The paper gives no backward; this is reverse-mode differentiation of Eq. 1-4 and the Conv1D.  The three dense
+// contractions run on tcgen05 tensor cores through one small GEMM kernel, the rest is element-wise and HBM-bound:
+//   1. conv_forward      u = Conv1D(x) in fp16, token-major [tok][D] and channel-major [D][tok]; fp16 copies of the weights
+//                        (every tensor-core operand here is fp16: 11 significant bits instead of bf16's 8 keep the
+//                        rounding of u and dz out of the gradients; finite overflow saturates at +-65504)
+//   2. GEMM              z_a | z_x = u W_a^T | u W_x^T per head (Eq. 1-2 before the sigmoid), fp16 out
+//   3. scan_fold / scan_carry / scan_apply
+//                        reverse-time scan g_t = dy_t + a_{t+1} g_{t+1} over chunks of 128 tokens (fold, carry across
+//                        chunks, re-run with the carry), then the element-wise adjoints: dz_a, dz_x (fp16, token-major
+//                        and channel-major), the direct part of du (fp32), partial sums of dLambda, db_a, db_x
+//   4. GEMM              du += dz_a W_a + dz_x W_x
+//   5. GEMM (split K)    dW_a | dW_x = dz^T u over all tokens, fp32 partial sums per split, reduced in fixed order
+//   6. Conv1D adjoint    dx, dconv_w, dconv_b (shared with the shape-generic backward), fixed-order reductions
+// h_{t-1} comes from the forward output y (bf16); when the caller has none the forward is run first.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "rglru_internal.h"
+#include "sm100_ptx.cuh"
+
+namespace rglru {
+namespace {
+
+using namespace ptx;
+
+constexpr int DH = 256;
+constexpr int CHUNK = 128;                 // tokens per scan chunk = rows of a GEMM tile
+constexpr int GEMM_THREADS = 192;          // TMA warp, MMA warp, four epilogue warps
+constexpr int GEMM_STAGES = 4;
+constexpr uint32_t A_STAGE_BYTES = 128 * 128;   // 128 rows x 64 bf16
+constexpr uint32_t B_STAGE_BYTES = 256 * 128;   // 256 rows x 64 bf16
+constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr uint32_t GEMM_SMEM_BAR = GEMM_STAGES * STAGE_BYTES;
+constexpr uint32_t GEMM_SMEM_TOTAL = GEMM_SMEM_BAR + (2 * GEMM_STAGES + 1) * 8 + 16;
+constexpr uint32_t GEMM_SMEM_ALLOC = GEMM_SMEM_TOTAL + 1024;
+
+enum { MODE_Z = 0, MODE_DU = 1, MODE_DW = 2 };
+
+struct GemmArgs {
+    alignas(64) CUtensorMap tm_a;    // A rows (M side), K innermost
+    alignas(64) CUtensorMap tm_b0;   // B rows (N side), K innermost
+    alignas(64) CUtensorMap tm_b1;   // MODE_Z: the second gate's weights (grid.y selects)
+    int mode, H, D;
+    int kblocks;       // 64-wide K blocks per CTA
+    int rows_valid;    // MODE_Z / MODE_DU: number of tokens; MODE_DW: 512
+    void *out;         // MODE_Z: __half z[tok][H][2][256]; MODE_DU: float du[tok][D] (+=); MODE_DW: float part[split][2][H][256][256]
+    uint32_t *status;
+    unsigned long long spin_ns;
+};
+
+// C[128 x 256] = A[128 x K] B[256 x K]^T for one tile; A and B tiles arrive by tiled TMA in the 128-byte-swizzled
+// K-major layout, accumulate in tensor memory (fp32), and leave through the four epilogue warps.
+//   MODE_Z : grid (token tiles, 2 gates, H)   A = u[tok][h][k]        B = W_gate[h][out][k]
+//   MODE_DU: grid (token tiles, 1, H)         A = dz[tok][h][k=512]   B = W^T[h][in][k=512]
+//   MODE_DW: grid (4 row tiles, splits, H)    A = dz^T[h][row][tok]   B = u^T[h][in][tok], K = this split's tokens
+__global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_constant__ GemmArgs p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (base - raw_addr);
+    const uint32_t bar0 = base + GEMM_SMEM_BAR;
+    auto BAR_FULL = [&](int s) { return bar0 + 8u * s; };
+    auto BAR_EMPTY = [&](int s) { return bar0 + 8u * (GEMM_STAGES + s); };
+    const uint32_t BAR_ACC = bar0 + 8u * (2 * GEMM_STAGES);
+    uint32_t *tmem_base_s = (uint32_t *)(smem + GEMM_SMEM_BAR + (2 * GEMM_STAGES + 1) * 8);
+    volatile int *abort_flag = (volatile int *)(tmem_base_s + 1);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int h = blockIdx.z;
+    const unsigned long long spin = p.spin_ns;
+
+    if (tid == 0) {
+        for (int s = 0; s < GEMM_STAGES; ++s) { mbar_init(BAR_FULL(s), 1); mbar_init(BAR_EMPTY(s), 1); }
+        mbar_init(BAR_ACC, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) { tmem_alloc(smem_u32(tmem_base_s), 256); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_base_s;
+    bool ok = true;
+
+    if (warp == 0) {
+        // ---- TMA producer
+        if (lane == 0) {
+            const CUtensorMap *tb = (p.mode == MODE_Z && blockIdx.y == 1) ? &p.tm_b1 : &p.tm_b0;
+            for (int kb = 0; kb < p.kblocks; ++kb) {
+                const int s = kb % GEMM_STAGES;
+                ok = mbar_wait(BAR_EMPTY(s), ((kb / GEMM_STAGES) & 1) ^ 1, spin, abort_flag);
+                if (!ok) break;
+                mbar_expect_tx(BAR_FULL(s), STAGE_BYTES);
+                const uint32_t a_dst = base + s * STAGE_BYTES, b_dst = a_dst + A_STAGE_BYTES;
+                if (p.mode == MODE_DW) {
+                    const int k0 = ((int)blockIdx.y * p.kblocks + kb) * 64;
+                    tma_load_3d(a_dst, &p.tm_a, k0, (int)blockIdx.x * 128, h, BAR_FULL(s));
+                    tma_load_3d(b_dst, tb, k0, 0, h, BAR_FULL(s));
+                } else {
+                    tma_load_3d(a_dst, &p.tm_a, kb * 64, h, (int)blockIdx.x * 128, BAR_FULL(s));
+                    tma_load_3d(b_dst, tb, kb * 64, 0, h, BAR_FULL(s));
+                }
+            }
+            if (!ok) { *abort_flag = 1; atomicExch(p.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT); }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_f16(128, 256);
+            for (int kb = 0; kb < p.kblocks; ++kb) {
+                const int s = kb % GEMM_STAGES;
+                ok = mbar_wait(BAR_FULL(s), (kb / GEMM_STAGES) & 1, spin, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_src = base + s * STAGE_BYTES, b_src = a_src + A_STAGE_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    mma_ss(tmem, make_desc_sw128(a_src + ks * 32), make_desc_sw128(b_src + ks * 32), idesc, (kb | ks) != 0);
+                tc_commit(BAR_EMPTY(s));
+            }
+            if (ok) tc_commit(BAR_ACC);
+            else { *abort_flag = 1; atomicExch(p.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT); }
+        }
+    } else {
+        // ---- epilogue: warp owns TMEM lanes 32 (warp & 3) .. +31 = rows of the tile
+        const int q = warp & 3;
+        const int row = (int)blockIdx.x * 128 + q * 32 + lane;
+        ok = warp_wait(BAR_ACC, 0, spin, abort_flag);
+        if (ok) {
+            tc_fence_after();
+            const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16);
+            const bool valid = row < p.rows_valid;
+#pragma unroll 1
+            for (int c0 = 0; c0 < 256; c0 += 32) {
+                f32x2 v[16];
+                tmem_ld32(tm_lane + c0, v);
+                tmem_ld_wait();
+                if (!valid) continue;
+                if (p.mode == MODE_Z) {
+                    __half *dst = (__half *)p.out + (((size_t)row * p.H + h) * 2 + blockIdx.y) * 256 + c0;
+                    uint32_t w[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) { const __half2 hh = __floats2half2_rn(lo2(v[j]), hi2(v[j])); w[j] = *(const uint32_t *)&hh; }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) ((uint4 *)dst)[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                } else if (p.mode == MODE_DU) {
+                    float4 *dst = (float4 *)((float *)p.out + (size_t)row * p.D + h * DH + c0);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        float4 o = dst[j];
+                        o.x += lo2(v[2 * j]); o.y += hi2(v[2 * j]); o.z += lo2(v[2 * j + 1]); o.w += hi2(v[2 * j + 1]);
+                        dst[j] = o;
+                    }
+                } else {
+                    const int g = row >> 8, o_row = row & 255;
+                    float4 *dst = (float4 *)((float *)p.out + ((((size_t)blockIdx.y * 2 + g) * p.H + h) * 256 + o_row) * 256 + c0);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) dst[j] = make_float4(lo2(v[2 * j]), hi2(v[2 * j]), lo2(v[2 * j + 1]), hi2(v[2 * j + 1]));
+                }
+            }
+        } else if (lane == 0) {
+            *abort_flag = 1; atomicExch(p.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
+        }
+    }
+    if (*abort_flag) {   // let copies and MMAs in flight land before shared and tensor memory are given back
+        const uint64_t tw = gtimer();
+        while (gtimer() - tw < 50000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, 256);
+}
+
+// ------------------------------------------------------------------ element-wise kernels
+__device__ __forceinline__ float bf2f(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float sigmoid_acc(float z) { return 1.0f / (1.0f + expf(-z)); }
+// s = c softplus(-Lambda)   (Appendix A, with a = sigmoid(Lambda))
+__device__ __forceinline__ float decay_rate(float lambda, float c) {
+    const float z = -lambda;
+    return c * (z > 0.0f ? z + log1pf(expf(-z)) : log1pf(expf(z)));
+}
+
+struct EwArgs {
+    int B, T, D, H, nchunk;
+    size_t BTp;                       // padded token count = row pitch of the channel-major arrays
+    float c;
+    const __nv_bfloat16 *x, *conv_w, *cs_in, *dy, *y;
+    const float *conv_b, *b_a, *b_x, *lambda, *h0;
+    __half *u, *uT, *dz, *dzT;
+    const __half *z;
+    float *du;                        // [tok][D]
+    float2 *fold;                     // [B][nchunk][D]: (prod a_t, carry out of the chunk for zero carry in)
+    float *xin;                       // [B][nchunk][D]: a_{t+1} g_{t+1} entering the chunk from later tokens
+    float *part_vec;                  // [B*nchunk][3][D]
+};
+
+// fp16 copies of the gate weights: W16[g][h][o][n] = W_g[h][o][n] and WT[h][n][g*256 + o] = W_g[h][o][n]
+__global__ void convert_w_kernel(const __nv_bfloat16 *Wa, const __nv_bfloat16 *Wx, __half *W16, __half *WT, int H) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;   // over [g][h][o][n]
+    if (i >= (size_t)H * 2 * DH * DH) return;
+    const int n = (int)(i % DH), o = (int)((i / DH) % DH), h = (int)((i / (DH * DH)) % H), g = (int)(i / ((size_t)H * DH * DH));
+    const float v = __bfloat162float((g ? Wx : Wa)[((size_t)h * DH + o) * DH + n]);
+    const __half hv = __float2half_rn(fminf(fmaxf(v, -65504.0f), 65504.0f));
+    W16[i] = hv;
+    WT[((size_t)h * DH + n) * (2 * DH) + g * DH + o] = hv;
+}
+
+__device__ __forceinline__ __half to_half_sat(float v) { return __float2half_rn(fminf(fmaxf(v, -65504.0f), 65504.0f)); }
+
+// u_t = b_c + sum_j w[j] x_{t-j}: one thread per (sequence, chunk, channel), forward in time.  grid (D/256, nchunk, B)
+__global__ void __launch_bounds__(256) conv_forward_kernel(EwArgs a) {
+    const int d = blockIdx.x * 256 + threadIdx.x, c = blockIdx.y, b = blockIdx.z;
+    const int T = a.T, D = a.D;
+    const int t0 = c * CHUNK, t1 = min(T, t0 + CHUNK);
+    float w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) w[j] = bf2f(a.conv_w[(size_t)j * D + d]);
+    const float cb = a.conv_b ? a.conv_b[d] : 0.0f;
+    auto xat = [&](int t) -> float {
+        if (t >= 0) return bf2f(a.x[((size_t)b * T + t) * D + d]);
+        return a.cs_in ? bf2f(a.cs_in[((size_t)b * 3 + (3 + t)) * D + d]) : 0.0f;
+    };
+    float x3 = xat(t0 - 3), x2 = xat(t0 - 2), x1 = xat(t0 - 1);
+    for (int t = t0; t < t1; t += 8) {
+        float xs[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) xs[k] = bf2f(a.x[((size_t)b * T + t + k) * D + d]);
+        uint32_t packed[4];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const float uv = fmaf(w[3], x3, fmaf(w[2], x2, fmaf(w[1], x1, fmaf(w[0], xs[k], cb))));
+            const __half ub = to_half_sat(uv);
+            a.u[((size_t)b * T + t + k) * D + d] = ub;
+            const uint32_t bits = (uint32_t)__half_as_ushort(ub);
+            if (k & 1) packed[k >> 1] |= bits << 16; else packed[k >> 1] = bits;
+            x3 = x2; x2 = x1; x1 = xs[k];
+        }
+        *(uint4 *)(a.uT + (size_t)d * a.BTp + (size_t)b * T + t) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+    }
+}
+
+// a_t = exp(-s sigmoid(z_a + b_a)) from the stored pre-activation
+__device__ __forceinline__ float decay_from_z(const EwArgs &a, size_t tok, int h, int n, float s, float ba) {
+    const float za = __half2float(a.z[((tok * a.H + h) * 2 + 0) * DH + n]);
+    return expf(-s * sigmoid_acc(za + ba));
+}
+
+// Reverse scan, pass 1: per chunk the product of a_t and the carry a_first g_first it hands to earlier tokens when
+// nothing comes in from later ones.  grid (D/256, nchunk, B)
+__global__ void __launch_bounds__(256) scan_fold_kernel(EwArgs a) {
+    const int d = blockIdx.x * 256 + threadIdx.x, c = blockIdx.y, b = blockIdx.z;
+    const int T = a.T, D = a.D, h = d / DH, n = d % DH;
+    const int t0 = c * CHUNK, t1 = min(T, t0 + CHUNK);
+    const float s = decay_rate(a.lambda[d], a.c), ba = a.b_a[d];
+    float carry = 0.0f, Q = 1.0f;
+    for (int t = t1 - 1; t >= t0; --t) {
+        const size_t tok = (size_t)b * T + t;
+        const float at = decay_from_z(a, tok, h, n, s, ba);
+        const float g = bf2f(a.dy[tok * D + d]) + carry;
+        carry = at * g;
+        Q *= at;
+    }
+    a.fold[((size_t)b * a.nchunk + c) * D + d] = make_float2(Q, carry);
+}
+
+// pass 2: carries across chunks, last chunk first.  grid (D/256, B)
+__global__ void __launch_bounds__(256) scan_carry_kernel(EwArgs a) {
+    const int d = blockIdx.x * 256 + threadIdx.x, b = blockIdx.y;
+    float X = 0.0f;
+    for (int c = a.nchunk - 1; c >= 0; --c) {
+        const size_t i = ((size_t)b * a.nchunk + c) * a.D + d;
+        a.xin[i] = X;
+        const float2 f = a.fold[i];
+        X = fmaf(f.x, X, f.y);
+    }
+}
+
+// pass 3: the scan with its carry and every element-wise adjoint (derived from Eq. 1-4):
+//   g_t = dy_t + a_{t+1} g_{t+1};  dL = g a (h_{t-1} - a v / m);  dv = g m;  di = dv u;  du = dv i;
+//   dr = -s dL;  dz_a = dr r (1-r);  dz_x = di i (1-i);  dLambda += dL c r sigmoid(-Lambda).   grid (D/256, nchunk, B)
+__global__ void __launch_bounds__(256) scan_apply_kernel(EwArgs a) {
+    const int d = blockIdx.x * 256 + threadIdx.x, c = blockIdx.y, b = blockIdx.z;
+    const int T = a.T, D = a.D, h = d / DH, n = d % DH;
+    const int t0 = c * CHUNK, t1 = min(T, t0 + CHUNK);
+    const float lam = a.lambda[d];
+    const float s = decay_rate(lam, a.c), ba = a.b_a[d], bx = a.b_x[d];
+    const float dsdlam_neg = a.c * sigmoid_acc(-lam);
+    float carry = a.xin[((size_t)b * a.nchunk + c) * D + d];
+    float s_lam = 0.0f, s_ba = 0.0f, s_bx = 0.0f;
+    for (int tb = t1 - 8; tb >= t0; tb -= 8) {
+        float dyv[8], hpv[8], zav[8], zxv[8], uv[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int t = tb + k;
+            const size_t tok = (size_t)b * T + t;
+            dyv[k] = bf2f(a.dy[tok * D + d]);
+            hpv[k] = t > 0 ? bf2f(a.y[(tok - 1) * D + d]) : (a.h0 ? a.h0[(size_t)b * D + d] : 0.0f);
+            zav[k] = __half2float(a.z[((tok * a.H + h) * 2 + 0) * DH + n]);
+            zxv[k] = __half2float(a.z[((tok * a.H + h) * 2 + 1) * DH + n]);
+            uv[k] = __half2float(a.u[tok * D + d]);
+        }
+        uint32_t pa[4], px[4];
+#pragma unroll
+        for (int k = 7; k >= 0; --k) {
+            const size_t tok = (size_t)b * T + tb + k;
+            const float r = sigmoid_acc(zav[k] + ba), gi = sigmoid_acc(zxv[k] + bx);
+            const float L = -s * r, at = expf(L), mt = sqrtf(fmaxf(0.0f, -expm1f(2.0f * L)));
+            const float g = dyv[k] + carry;
+            carry = at * g;
+            const float v = gi * uv[k];
+            const float dm_term = mt > 0.0f ? at * at * v / mt : 0.0f;
+            const float dL = g * (at * hpv[k] - dm_term);
+            const float dv = g * mt;
+            const float dza = -s * dL * r * (1.0f - r), dzx = dv * uv[k] * gi * (1.0f - gi);
+            s_lam = fmaf(dL * r, dsdlam_neg, s_lam);
+            s_ba += dza; s_bx += dzx;
+            a.du[tok * D + d] = dv * gi;
+            const __half ha = to_half_sat(dza), hx = to_half_sat(dzx);
+            a.dz[((tok * a.H + h) * 2 + 0) * DH + n] = ha;
+            a.dz[((tok * a.H + h) * 2 + 1) * DH + n] = hx;
+            const uint32_t ba16 = (uint32_t)__half_as_ushort(ha), bx16 = (uint32_t)__half_as_ushort(hx);
+            if (k & 1) { pa[k >> 1] = ba16 << 16; px[k >> 1] = bx16 << 16; } else { pa[k >> 1] |= ba16; px[k >> 1] |= bx16; }
+        }
+        const size_t col = (size_t)b * T + tb;
+        *(uint4 *)(a.dzT + ((size_t)h * 2 * DH + n) * a.BTp + col) = make_uint4(pa[0], pa[1], pa[2], pa[3]);
+        *(uint4 *)(a.dzT + ((size_t)h * 2 * DH + DH + n) * a.BTp + col) = make_uint4(px[0], px[1], px[2], px[3]);
+    }
+    float *pv = a.part_vec + ((size_t)b * a.nchunk + c) * 3 * D + d;
+    pv[0] = s_lam; pv[(size_t)D] = s_ba; pv[(size_t)2 * D] = s_bx;
+}
+
+inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+struct BwdLayout {
+    size_t BT, BTp, off_u, off_uT, off_z, off_dz, off_dzT, off_du, off_y, off_hT, off_cs, off_fold, off_xin, off_pvec, off_pconv, off_pdw,
+        off_wt, off_w16, off_fws, total;
+    int nchunk, nchunk_conv, S, kb_per_split;
+};
+
+BwdLayout bwd_layout(int B, int T, int D, int H) {
+    BwdLayout L{};
+    L.BT = (size_t)B * T;
+    L.BTp = (L.BT + 63) & ~(size_t)63;
+    L.nchunk = (T + CHUNK - 1) / CHUNK;
+    L.nchunk_conv = (T + GENERIC_BWD_CHUNK - 1) / GENERIC_BWD_CHUNK;
+    const int kblocks = (int)(L.BTp / 64);
+    L.S = kblocks < 8 ? kblocks : 8;
+    L.kb_per_split = (kblocks + L.S - 1) / L.S;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { const size_t at = o; o += up256(bytes); return at; };
+    L.off_u = take(L.BT * D * 2);
+    L.off_uT = take((size_t)D * L.BTp * 2);
+    L.off_z = take(L.BT * D * 2 * 2);
+    L.off_dz = take(L.BT * D * 2 * 2);
+    L.off_dzT = take((size_t)D * 2 * L.BTp * 2);
+    L.off_du = take(L.BT * D * 4);
+    L.off_y = take(L.BT * D * 2);
+    L.off_hT = take((size_t)B * D * 4);
+    L.off_cs = take((size_t)B * 3 * D * 2);
+    L.off_fold = take((size_t)B * L.nchunk * D * 8);
+    L.off_xin = take((size_t)B * L.nchunk * D * 4);
+    L.off_pvec = take((size_t)B * L.nchunk * 3 * D * 4);
+    L.off_pconv = take((size_t)B * L.nchunk_conv * 5 * D * 4);
+    L.off_pdw = take((size_t)L.S * 2 * H * DH * DH * 4);
+    L.off_wt = take((size_t)H * DH * 2 * DH * 2);
+    L.off_w16 = take((size_t)H * DH * 2 * DH * 2);
+    L.off_fws = take(WS_HEADER_BYTES + sm100_prefill_workspace_bytes(B, T, D, H));
+    L.total = o;
+    return L;
+}
+
+}  // namespace
+
+bool sm100_backward_supported(int B, int T, int D, int H, int io) {
+    return io == RGLRU_BF16 && B > 0 && T > 0 && H > 0 && D == H * DH && T % 8 == 0;
+}
+
+size_t sm100_backward_workspace_bytes(int B, int T, int D, int H) { return bwd_layout(B, T, D, H).total; }
+
+cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, void *ws_body, size_t ws_body_bytes, uint32_t *status,
+                           cudaStream_t st) {
+    const int B = q.B, T = q.T, D = q.D, H = q.H;
+    const BwdLayout L = bwd_layout(B, T, D, H);
+    if (ws_body_bytes < L.total) return cudaErrorInvalidValue;
+    static bool attr_set = false;
+    cudaError_t e;
+    if (!attr_set) {
+        e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_ALLOC);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    char *ws = (char *)ws_body;
+    __half *u = (__half *)(ws + L.off_u), *uT = (__half *)(ws + L.off_uT), *z = (__half *)(ws + L.off_z);
+    __half *dz = (__half *)(ws + L.off_dz), *dzT = (__half *)(ws + L.off_dzT), *WT = (__half *)(ws + L.off_wt), *W16 = (__half *)(ws + L.off_w16);
+    float *du = (float *)(ws + L.off_du);
+
+    // 0. h_{t-1} comes from the forward output; run the forward when the caller kept none
+    const void *y = y_saved;
+    if (y == nullptr) {
+        FwdArgs f = fwd;
+        f.y = ws + L.off_y; f.h_T = (float *)(ws + L.off_hT); f.cs_out = ws + L.off_cs;
+        f.status = status;
+        char *fws = ws + L.off_fws;
+        e = sm100_prefill(f, fws + WS_HEADER_BYTES, sm100_prefill_workspace_bytes(B, T, D, H), st);
+        if (e != cudaSuccess) return e;
+        y = f.y;
+    }
+    if (L.BTp != L.BT) {   // the padded token columns enter the dW contraction and must be zero
+        if ((e = cudaMemsetAsync(uT, 0, (size_t)D * L.BTp * 2, st)) != cudaSuccess) return e;
+        if ((e = cudaMemsetAsync(dzT, 0, (size_t)D * 2 * L.BTp * 2, st)) != cudaSuccess) return e;
+    }
+
+    EwArgs a{};
+    a.B = B; a.T = T; a.D = D; a.H = H; a.nchunk = L.nchunk; a.BTp = L.BTp; a.c = q.c;
+    a.x = (const __nv_bfloat16 *)q.x; a.conv_w = (const __nv_bfloat16 *)q.conv_w; a.cs_in = (const __nv_bfloat16 *)q.cs_in;
+    a.dy = (const __nv_bfloat16 *)q.dy; a.y = (const __nv_bfloat16 *)y;
+    a.conv_b = fwd.conv_b; a.b_a = fwd.b_a; a.b_x = fwd.b_x; a.lambda = q.lambda; a.h0 = fwd.h0;
+    a.u = u; a.uT = uT; a.dz = dz; a.dzT = dzT; a.z = z; a.du = du;
+    a.fold = (float2 *)(ws + L.off_fold); a.xin = (float *)(ws + L.off_xin); a.part_vec = (float *)(ws + L.off_pvec);
+
+    // 1. W^T for the du contraction, conv output
+    const size_t nW = (size_t)H * 2 * DH * DH;
+    convert_w_kernel<<<(unsigned)((nW + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)q.W_a, (const __nv_bfloat16 *)q.W_x, W16, WT, H);
+    const dim3 grid_ew(D / 256, L.nchunk, B);
+    conv_forward_kernel<<<grid_ew, 256, 0, st>>>(a);
+
+    GemmArgs g{};
+    g.H = H; g.D = D; g.status = status; g.spin_ns = g_spin_limit_ns;
+    const unsigned mtiles = (unsigned)((L.BT + 127) / 128);
+    const uint64_t BT = L.BT, BTp = L.BTp;
+    // 2. z = u W^T per head and gate
+    {
+        const uint64_t da[3] = {DH, (uint64_t)H, BT}, sa[2] = {DH * 2, (uint64_t)D * 2};
+        const uint32_t ba[3] = {64, 1, 128};
+        const uint64_t db[3] = {DH, DH, (uint64_t)H}, sb[2] = {DH * 2, (uint64_t)DH * DH * 2};
+        const uint32_t bb[3] = {64, 256, 1};
+        if (!encode_map16_3d(&g.tm_a, u, da, sa, ba, true) || !encode_map16_3d(&g.tm_b0, W16, db, sb, bb, true) ||
+            !encode_map16_3d(&g.tm_b1, W16 + (size_t)H * DH * DH, db, sb, bb, true))
+            return cudaErrorNotSupported;
+        g.mode = MODE_Z; g.kblocks = DH / 64; g.rows_valid = (int)BT; g.out = z;
+        tc_gemm_kernel<<<dim3(mtiles, 2, H), GEMM_THREADS, GEMM_SMEM_ALLOC, st>>>(g);
+    }
+    // 3. reverse scan and element-wise adjoints
+    scan_fold_kernel<<<grid_ew, 256, 0, st>>>(a);
+    scan_carry_kernel<<<dim3(D / 256, B), 256, 0, st>>>(a);
+    scan_apply_kernel<<<grid_ew, 256, 0, st>>>(a);
+    // 4. du += dz W
+    {
+        const uint64_t da[3] = {2 * DH, (uint64_t)H, BT}, sa[2] = {2 * DH * 2, (uint64_t)H * 2 * DH * 2};
+        const uint32_t ba[3] = {64, 1, 128};
+        const uint64_t db[3] = {2 * DH, DH, (uint64_t)H}, sb[2] = {2 * DH * 2, (uint64_t)DH * 2 * DH * 2};
+        const uint32_t bb[3] = {64, 256, 1};
+        if (!encode_map16_3d(&g.tm_a, dz, da, sa, ba, true) || !encode_map16_3d(&g.tm_b0, WT, db, sb, bb, true)) return cudaErrorNotSupported;
+        g.tm_b1 = g.tm_b0;
+        g.mode = MODE_DU; g.kblocks = 2 * DH / 64; g.rows_valid = (int)BT; g.out = du;
+        tc_gemm_kernel<<<dim3(mtiles, 1, H), GEMM_THREADS, GEMM_SMEM_ALLOC, st>>>(g);
+    }
+    // 5. dW = dz^T u, split over the tokens, then a fixed-order sum of the splits
+    {
+        const uint64_t da[3] = {BTp, 2 * DH, (uint64_t)H}, sa[2] = {BTp * 2, (uint64_t)2 * DH * BTp * 2};
+        const uint32_t ba[3] = {64, 128, 1};
+        const uint64_t db[3] = {BTp, DH, (uint64_t)H}, sb[2] = {BTp * 2, (uint64_t)DH * BTp * 2};
+        const uint32_t bb[3] = {64, 256, 1};
+        if (!encode_map16_3d(&g.tm_a, dzT, da, sa, ba, true) || !encode_map16_3d(&g.tm_b0, uT, db, sb, bb, true)) return cudaErrorNotSupported;
+        g.tm_b1 = g.tm_b0;
+        float *part = (float *)(ws + L.off_pdw);
+        g.mode = MODE_DW; g.kblocks = L.kb_per_split; g.rows_valid = 2 * DH; g.out = part;
+        tc_gemm_kernel<<<dim3(4, L.S, H), GEMM_THREADS, GEMM_SMEM_ALLOC, st>>>(g);
+        const size_t wsz = (size_t)H * DH * DH;
+        if ((e = reduce_partials(part, L.S, 2 * wsz, q.dW_a, wsz, st)) != cudaSuccess) return e;
+        if ((e = reduce_partials(part + wsz, L.S, 2 * wsz, q.dW_x, wsz, st)) != cudaSuccess) return e;
+    }
+    // 6. per-channel sums, Conv1D adjoint
+    const int nparts = B * L.nchunk;
+    if ((e = reduce_partials(a.part_vec, nparts, (size_t)3 * D, q.dlambda, D, st)) != cudaSuccess) return e;
+    if ((e = reduce_partials(a.part_vec + D, nparts, (size_t)3 * D, q.db_a, D, st)) != cudaSuccess) return e;
+    if ((e = reduce_partials(a.part_vec + 2 * (size_t)D, nparts, (size_t)3 * D, q.db_x, D, st)) != cudaSuccess) return e;
+    q.hp = du;
+    q.part_conv = (float *)(ws + L.off_pconv);
+    if ((e = generic_bwd_conv_and_reduce(q, RGLRU_BF16, st)) != cudaSuccess) return e;
+    return cudaGetLastError();
+}
+
+}  // namespace rglru

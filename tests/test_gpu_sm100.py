@@ -128,3 +128,27 @@ def test_decode_agrees_with_generic_decode_and_status():
     assert_close("y", to_np(outs[0][0]), to_np(outs[1][0]), "bf16")
     assert_close("h", to_np(outs[0][1]), to_np(outs[1][1]), "bf16")
     assert torch.equal(outs[0][2], outs[1][2])
+
+
+@pytest.mark.parametrize("B,T,H,with_y", [(3, 8, 1, True), (2, 136, 1, True), (1, 264, 2, False), (2, 1000, 1, True)])
+def test_backward_tensor_core_path(oracle, B, T, H, with_y):
+    """Tensor-core backward (GEMMs for z, du and dW around the chunked reverse scan) against the oracle's analytic
+    gradients; with and without the saved forward output."""
+    import torch
+    from paper_2402_19427_b200 import binding
+    D = 256 * H
+    inp = synth.make_inputs(B, T, D, H, io="bf16", seed=900 + T, with_dy=True, with_state=True, bias_scale=0.2)
+    params = binding.Params.from_numpy(inp["params"], "bf16")
+    x = to_dev(inp["x"], "bf16"); dy = to_dev(inp["dy"], "bf16")
+    h0 = to_dev(inp["h0"]); cs = to_dev(inp["conv_state"], "bf16")
+    shape = binding.make_shape(B, T, D, H, torch.bfloat16)
+    assert binding.workspace_bytes(shape, binding.OP_BACKWARD) != binding.workspace_bytes(
+        binding.make_shape(B, T, D, H, torch.bfloat16, flags=1), binding.OP_BACKWARD)      # not the generic path
+    y = binding.prefill(x, params, h0=h0, conv_state_in=cs)[0] if with_y else None
+    ws = binding.alloc_workspace(shape, binding.OP_BACKWARD, x.device)
+    g = binding.backward(x, params, dy, h0=h0, conv_state_in=cs, y=y, workspace=ws)
+    assert binding.query_status(ws) == binding.OK
+    gr = oracle.backward(inp["x"].astype(np.float64), f64(inp["params"]), H, inp["dy"].astype(np.float64),
+                         h0=inp["h0"].astype(np.float64), conv_state_in=inp["conv_state"].astype(np.float64))
+    for k in gr:
+        assert_close("d" + k, to_np(g[k]), gr[k], "bf16")

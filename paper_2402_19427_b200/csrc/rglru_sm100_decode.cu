@@ -139,20 +139,31 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
         __nv_bfloat16 *cs = (__nv_bfloat16 *)f.cs_out;   // in/out
         const uint32_t u_kb = SMEM_U + (uint32_t)(dl >> 6) * KBLOCK_BYTES;
         const uint32_t chunk = (uint32_t)(dl & 63) >> 3;
+        // all global loads of the phase are issued before anything waits on them
+        constexpr int NIT = NB_MAX / 16;
+        uint4 xv[NIT], r0[NIT], r1[NIT], r2[NIT];   // x_t and x_{t-3}, x_{t-2}, x_{t-1} per sequence
+#pragma unroll
+        for (int i = 0; i < NIT; ++i) {
+            const int n = (tid >> 4) + 16 * i, b = b0 + n;
+            if (n < NB && b < B) {
+                xv[i] = *(const uint4 *)(x + (size_t)b * D + d);
+                r0[i] = *(const uint4 *)(cs + ((size_t)b * 3 + 0) * D + d);
+                r1[i] = *(const uint4 *)(cs + ((size_t)b * 3 + 1) * D + d);
+                r2[i] = *(const uint4 *)(cs + ((size_t)b * 3 + 2) * D + d);
+            }
+        }
         cluster_wait();
         const uint32_t peer_base = map_to_cta(base, rank ^ 1u);
-        for (int n = tid >> 4; n < NB; n += 16) {
-            const int b = b0 + n;
+        const uint32_t w0[4] = {w[0].x, w[0].y, w[0].z, w[0].w}, w1[4] = {w[1].x, w[1].y, w[1].z, w[1].w},
+                       w2[4] = {w[2].x, w[2].y, w[2].z, w[2].w}, w3[4] = {w[3].x, w[3].y, w[3].z, w[3].w};
+#pragma unroll
+        for (int i = 0; i < NIT; ++i) {
+            const int n = (tid >> 4) + 16 * i, b = b0 + n;
+            if (n >= NB) break;
             uint4 uo = make_uint4(0u, 0u, 0u, 0u);
             if (b < B) {
-                const uint4 xv = *(const uint4 *)(x + (size_t)b * D + d);
-                uint4 *c0p = (uint4 *)(cs + ((size_t)b * 3 + 0) * D + d), *c1p = (uint4 *)(cs + ((size_t)b * 3 + 1) * D + d),
-                      *c2p = (uint4 *)(cs + ((size_t)b * 3 + 2) * D + d);
-                const uint4 r0 = *c0p, r1 = *c1p, r2 = *c2p;   // x_{t-3}, x_{t-2}, x_{t-1}
-                const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w}, a0[4] = {r0.x, r0.y, r0.z, r0.w}, a1[4] = {r1.x, r1.y, r1.z, r1.w},
-                               a2[4] = {r2.x, r2.y, r2.z, r2.w};
-                const uint32_t w0[4] = {w[0].x, w[0].y, w[0].z, w[0].w}, w1[4] = {w[1].x, w[1].y, w[1].z, w[1].w},
-                               w2[4] = {w[2].x, w[2].y, w[2].z, w[2].w}, w3[4] = {w[3].x, w[3].y, w[3].z, w[3].w};
+                const uint32_t xw[4] = {xv[i].x, xv[i].y, xv[i].z, xv[i].w}, a0[4] = {r0[i].x, r0[i].y, r0[i].z, r0[i].w},
+                               a1[4] = {r1[i].x, r1[i].y, r1[i].z, r1[i].w}, a2[4] = {r2[i].x, r2[i].y, r2[i].z, r2[i].w};
                 uint32_t o[4], rem[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
@@ -166,7 +177,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
                 }
                 uo = make_uint4(o[0], o[1], o[2], o[3]);
                 *(uint4 *)(smem + SMEM_R + (uint32_t)n * (CH * 2) + (uint32_t)c * 16u) = make_uint4(rem[0], rem[1], rem[2], rem[3]);
-                *c0p = r1; *c1p = r2; *c2p = xv;   // the conv state moves up by one row: bit-exact copies
+                // the conv state moves up by one row: bit-exact copies
+                *(uint4 *)(cs + ((size_t)b * 3 + 0) * D + d) = r1[i];
+                *(uint4 *)(cs + ((size_t)b * 3 + 1) * D + d) = r2[i];
+                *(uint4 *)(cs + ((size_t)b * 3 + 2) * D + d) = xv[i];
             }
             const uint32_t off = u_kb + (uint32_t)n * 128u + ((chunk ^ (uint32_t)(n & 7)) << 4);
             *(uint4 *)(smem + off) = uo;
@@ -215,17 +229,21 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
         __nv_bfloat16 *y = (__nv_bfloat16 *)f.y;
         const int nh = NB >> 1;                           // multiple of 8
         const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16);
+        // the recurrent state of this warp's sequences is fetched while the tensor core works
+        float hv[NB_MAX / 2];
+#pragma unroll
+        for (int j = 0; j < NB_MAX / 2; ++j) {
+            const int b = b0 + k * nh + j;
+            hv[j] = (j < nh && b < B) ? h[(size_t)b * D + d] : 0.0f;
+        }
         if (!warp_wait(BAR_ACC, 0, spin, &no_abort)) {
             timed_out = 1;
         } else {
             tc_fence_after();
-            for (int n0 = k * nh; n0 < (k + 1) * nh; n0 += 8) {
-                float hv[8];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int b = b0 + n0 + j;
-                    hv[j] = b < B ? h[(size_t)b * D + d] : 0.0f;
-                }
+            for (int j0 = 0; j0 < NB_MAX / 2; j0 += 8) {
+                if (j0 >= nh) break;
+                const int n0 = k * nh + j0;
                 float za[8], zx[8];
                 tmem_ld8(tm_lane + n0, za);
                 tmem_ld8(tm_lane + 128 + n0, zx);
@@ -237,7 +255,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
                     const uint32_t rb = *(const uint16_t *)(r_col + (uint32_t)n * (CH * 2));
                     float a, v;
                     gate(za[j], zx[j], __uint_as_float(ub << 16) + __uint_as_float(rb << 16), hba, hbx, s, poly, a, v);
-                    const float hn = fmaf(a, hv[j], v);
+                    const float hn = fmaf(a, hv[j0 + j], v);
                     if (b < B) {
                         h[(size_t)b * D + d] = hn;
                         y[(size_t)b * D + d] = __float2bfloat16_rn(hn);

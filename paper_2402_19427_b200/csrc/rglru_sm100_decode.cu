@@ -22,6 +22,7 @@
 
 #include "rglru_internal.h"
 #include "sm100_ptx.cuh"
+#include "sm100_gates.cuh"
 
 namespace rglru {
 namespace {
@@ -42,7 +43,6 @@ constexpr uint32_t SMEM_MISC = SMEM_BAR + 16;             // tmem base
 constexpr uint32_t SMEM_TOTAL = SMEM_MISC + 16;
 constexpr uint32_t SMEM_ALLOC = SMEM_TOTAL + 1024;
 constexpr uint32_t TMEM_COLS = 256;                        // z_a in columns [0, NB), z_x in [128, 128 + NB)
-constexpr float S_POLY = 0.25f;                            // decay rates up to here use the polynomial for 1 - a_t
 
 struct DecArgs {
     alignas(64) CUtensorMap tm_wa;   // W_a as [H][256 out][256 in], box 128 out x 64 in, 128-byte swizzle
@@ -58,29 +58,6 @@ __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *(const uint32_t *)&v;
-}
-
-// (z_a, z_x, u) -> (a_t, v_t) of Eq. 3-4 with the same formulation as the prefill kernel:
-//   r = 1/2 + 1/2 tanh((z_a + b_a)/2), x = 2 s r, f = 1 - a_t = -expm1(-x/2), sqrt(1 - a_t^2)/2 = sqrt(f (1/2 - f/4)),
-//   v = (sqrt(1 - a_t^2)/2 u)(1 + tanh((z_x + b_x)/2)).
-__device__ __forceinline__ void gate(float za, float zx, float u, float hba, float hbx, float s, bool poly, float &a, float &v) {
-    const float ta = tanh_approx(fmaf(za, 0.5f, hba));
-    const float x = fmaf(ta, s, s);
-    float f;
-    if (poly) {
-        float pl = fmaf(x, -1.0f / 384.0f, 1.0f / 48.0f);
-        pl = fmaf(pl, x, -0.125f);
-        pl = fmaf(pl, x, 0.5f);
-        f = pl * x;
-        a = 1.0f - f;
-    } else {
-        a = ex2_approx(x * -0.72134752f);
-        f = 1.0f - a;
-    }
-    const float mh = sqrt_approx(fmaxf(f * fmaf(f, -0.25f, 0.5f), 0.0f));
-    const float tx = tanh_approx(fmaf(zx, 0.5f, hbx));
-    const float g = mh * u;
-    v = fmaf(g, tx, g);
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_decode_kernel(const __grid_constant__ DecArgs p) {
@@ -113,8 +90,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     const uint32_t tmem = *tmem_base_s;
     cluster_arrive();   // the peer must be running before anything is stored into its shared memory
 
-    // ---- this CTA's gate weights: 2 gates x 4 K blocks of [128 out rows x 64 in channels]
-    if (tid == 0) {
+    // ---- this CTA's gate weights: 2 gates x 4 K blocks of [128 out rows x 64 in channels], issued by the last warp so
+    //      that the descriptor fetch of the first tiled copy delays nobody's global loads; they are the longest latency
+    //      of the step (128 KB per CTA out of L2) and overlap the whole conv phase
+    if (tid == NTHREADS - 32) {
         mbar_expect_tx(BAR_W, 8 * KBLOCK_BYTES);
 #pragma unroll
         for (int kb = 0; kb < 4; ++kb) {
@@ -122,6 +101,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
             tma_load_3d(base + SMEM_WX + kb * KBLOCK_BYTES, &p.tm_wx, kb * 64, (int)rank * CH, head, BAR_W);
         }
     }
+    __syncwarp();
 
     // ---- conv phase: thread = (8-channel chunk c, sequences n = tid/16, tid/16 + 16, ...)
     {
@@ -191,6 +171,30 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     cluster_arrive();
     cluster_wait();      // both halves of the U tile are in place in both CTAs
 
+    // ---- epilogue: warp (q, k) owns channels 32 q .. 32 q + 31 and half k of the tile's sequences
+    const int q = warp & 3, k = warp >> 2;
+        const int c_own = q * 32 + lane;
+        const int dl = (int)rank * CH + c_own;
+        const size_t d = (size_t)head * DH + dl;
+        const float lam = f.lambda[d];
+        const float zl = -lam;
+        const float s = f.c * (zl > 0.0f ? zl + log1pf(expf(-zl)) : log1pf(expf(zl)));
+        const bool poly = __all_sync(0xffffffffu, s <= S_POLY);
+        const f32x2 hba2 = pack2(0.5f * f.b_a[d], 0.5f * f.b_a[d]), hbx2 = pack2(0.5f * f.b_x[d], 0.5f * f.b_x[d]), s2 = pack2(s, s);
+        const uint8_t *u_col = smem + SMEM_U + (uint32_t)(dl >> 6) * KBLOCK_BYTES + (uint32_t)(dl & 7) * 2u;
+        const uint32_t u_chunk = (uint32_t)(dl & 63) >> 3;
+        const uint8_t *r_col = smem + SMEM_R + (uint32_t)c_own * 2u;
+        float *h = f.h_T;                                 // in/out
+        __nv_bfloat16 *y = (__nv_bfloat16 *)f.y;
+        const int nh = NB >> 1;                           // multiple of 8
+        const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16);
+        // the recurrent state of this warp's sequences is fetched while the tensor core works
+        float hv[NB_MAX / 2];
+#pragma unroll
+        for (int j = 0; j < NB_MAX / 2; ++j) {
+            const int b = b0 + k * nh + j;
+            hv[j] = (j < nh && b < B) ? h[(size_t)b * D + d] : 0.0f;
+        }
     // ---- gate products
     if (tid == 0) {
         if (mbar_wait(BAR_W, 0, spin, &no_abort)) {
@@ -211,31 +215,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     }
     __syncwarp();
 
-    // ---- epilogue: warp (q, k) owns channels 32 q .. 32 q + 31 and half k of the tile's sequences
     {
-        const int q = warp & 3, k = warp >> 2;
-        const int c_own = q * 32 + lane;
-        const int dl = (int)rank * CH + c_own;
-        const size_t d = (size_t)head * DH + dl;
-        const float lam = f.lambda[d];
-        const float zl = -lam;
-        const float s = f.c * (zl > 0.0f ? zl + log1pf(expf(-zl)) : log1pf(expf(zl)));
-        const bool poly = __all_sync(0xffffffffu, s <= S_POLY);
-        const float hba = 0.5f * f.b_a[d], hbx = 0.5f * f.b_x[d];
-        const uint8_t *u_col = smem + SMEM_U + (uint32_t)(dl >> 6) * KBLOCK_BYTES + (uint32_t)(dl & 7) * 2u;
-        const uint32_t u_chunk = (uint32_t)(dl & 63) >> 3;
-        const uint8_t *r_col = smem + SMEM_R + (uint32_t)c_own * 2u;
-        float *h = f.h_T;                                 // in/out
-        __nv_bfloat16 *y = (__nv_bfloat16 *)f.y;
-        const int nh = NB >> 1;                           // multiple of 8
-        const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16);
-        // the recurrent state of this warp's sequences is fetched while the tensor core works
-        float hv[NB_MAX / 2];
-#pragma unroll
-        for (int j = 0; j < NB_MAX / 2; ++j) {
-            const int b = b0 + k * nh + j;
-            hv[j] = (j < nh && b < B) ? h[(size_t)b * D + d] : 0.0f;
-        }
         if (!warp_wait(BAR_ACC, 0, spin, &no_abort)) {
             timed_out = 1;
         } else {
@@ -248,17 +228,31 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
                 tmem_ld8(tm_lane + n0, za);
                 tmem_ld8(tm_lane + 128 + n0, zx);
                 tmem_ld_wait();
+                // two sequences per register pair, four pairs side by side
+                f32x2 A2[4], V2[4];
+                float u[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    const int n = n0 + j, b = b0 + n;
+                    const int n = n0 + j;
                     const uint32_t ub = *(const uint16_t *)(u_col + (uint32_t)n * 128u + ((u_chunk ^ (uint32_t)(n & 7)) << 4));
                     const uint32_t rb = *(const uint16_t *)(r_col + (uint32_t)n * (CH * 2));
-                    float a, v;
-                    gate(za[j], zx[j], __uint_as_float(ub << 16) + __uint_as_float(rb << 16), hba, hbx, s, poly, a, v);
-                    const float hn = fmaf(a, hv[j0 + j], v);
-                    if (b < B) {
-                        h[(size_t)b * D + d] = hn;
-                        y[(size_t)b * D + d] = __float2bfloat16_rn(hn);
+                    u[j] = __uint_as_float(ub << 16) + __uint_as_float(rb << 16);
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { A2[j] = pack2(za[2 * j], za[2 * j + 1]); V2[j] = pack2(zx[2 * j], zx[2 * j + 1]); }
+                if (poly) gate_group<true, 4>(A2, V2, u, hba2, hbx2, s2);
+                else gate_group<false, 4>(A2, V2, u, hba2, hbx2, s2);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const f32x2 H2 = fma2(A2[j], pack2(hv[j0 + 2 * j], hv[j0 + 2 * j + 1]), V2[j]);
+                    const float hn[2] = {lo2(H2), hi2(H2)};
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int b = b0 + n0 + 2 * j + e;
+                        if (b < B) {
+                            h[(size_t)b * D + d] = hn[e];
+                            y[(size_t)b * D + d] = __float2bfloat16_rn(hn[e]);
+                        }
                     }
                 }
             }

@@ -239,7 +239,10 @@ def run_ours(args):
     k = (e2e_steps - 1) % 2
     ref_y, _, _ = binding.prefill(xs[k], params, workspace=ws)
     torch.cuda.synchronize()
-    if not torch.equal(ref_y.cpu(), y_pin[k]):
+    # chunks of sequences run with their own time split, so sums associate differently: compare within the parity tolerance
+    a64, b64 = y_pin[k].double(), ref_y.cpu().double()
+    rms = float(b64.pow(2).mean().sqrt())
+    if not bool(((a64 - b64).abs() <= 2e-2 * torch.clamp(b64.abs(), min=rms)).all()):
         raise RuntimeError("host-buffer entry point disagrees with the device entry point")
     io_b = 2
     h2d = B * T * D * io_b

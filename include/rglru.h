@@ -137,8 +137,11 @@ int32_t rglru_backward(const rglru_shape_t *shape, const rglru_params_t *params,
 /*
  * rglru_prefill for callers whose activations live in HOST memory (pinned memory makes the
  * copies asynchronous).  x_host is copied to `staging`, the forward runs there, and y, h_T and
- * conv_state_out are copied back to the host pointers, all on `cuda_stream`; the call returns
- * without synchronising.  params, h0, conv_state_in, staging and workspace are device pointers.
+ * conv_state_out are copied back to the host pointers; the call returns without synchronising and work
+ * enqueued on `cuda_stream` afterwards sees the results.  The batch is cut into chunks of sequences whose
+ * host-to-device copy, forward and device-to-host copy overlap on two internal streams (created on first use
+ * per device); calls on one device must not be made from several host threads at once.
+ * params, h0, conv_state_in, staging and workspace are device pointers.
  *   staging : device scratch of at least rglru_host_staging_bytes(shape) bytes, 256-byte aligned.
  */
 size_t rglru_host_staging_bytes(const rglru_shape_t *shape);

@@ -2,6 +2,8 @@
 // kernel selection.  Every error is a return code; nothing here allocates device memory.
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 #include "rglru_internal.h"
 
 using namespace rglru;
@@ -38,6 +40,37 @@ inline bool overlap(const void *a, size_t na, const void *b, size_t nb) {
 
 bool use_sm100_prefill(const rglru_shape_t *s) {
     return !(s->flags & RGLRU_FLAG_FORCE_GENERIC) && sm100_prefill_supported(s->B, s->T, s->D, s->H, s->io);
+}
+
+// Two helper streams and the events that tie them to the caller's stream for rglru_prefill_host, one set per device,
+// created on first use (streams and events are not device memory).  Calls on one device are serialised by the mutex.
+struct HostPipe {
+    static constexpr int MAX_CHUNKS = 16;
+    std::mutex mutex;
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, done = nullptr, copied[MAX_CHUNKS] = {}, computed[MAX_CHUNKS] = {};
+    bool ready = false;
+};
+
+HostPipe *host_pipe() {
+    static HostPipe pipes[64];
+    static std::mutex setup;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(setup);
+    HostPipe &hp = pipes[dev];
+    if (!hp.ready) {
+        bool ok = cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.done, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; ok && i < HostPipe::MAX_CHUNKS; ++i)
+            ok = cudaEventCreateWithFlags(&hp.copied[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&hp.computed[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return nullptr;
+        hp.ready = true;
+    }
+    return &hp;
 }
 
 bool use_sm100_backward(const rglru_shape_t *s) {
@@ -191,18 +224,54 @@ int32_t rglru_prefill_host(const rglru_shape_t *s, const rglru_params_t *p, cons
     if (!x_host || !y_host || !h_T_host || !conv_state_out_host || !staging) return RGLRU_ERR_NULL;
     if (!aligned(staging, 256)) return RGLRU_ERR_ALIGN;
     if (staging_bytes < rglru_host_staging_bytes(s)) return RGLRU_ERR_WORKSPACE;
-    const size_t xbytes = (size_t)s->B * s->T * s->D * io_bytes(s->io);
-    const size_t hbytes = (size_t)s->B * s->D * sizeof(float);
-    const size_t cbytes = (size_t)s->B * 3 * s->D * io_bytes(s->io);
+    const size_t io = io_bytes(s->io);
+    const size_t seq_x = (size_t)s->T * s->D * io, seq_h = (size_t)s->D * sizeof(float), seq_c = (size_t)3 * s->D * io;
+    const size_t xbytes = (size_t)s->B * seq_x, hbytes = (size_t)s->B * seq_h, cbytes = (size_t)s->B * seq_c;
     const size_t xb = (xbytes + 255) & ~(size_t)255, hb = (hbytes + 255) & ~(size_t)255;
     char *sx = (char *)staging, *sy = sx + xb, *sh = sy + xb, *sc = sh + hb;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    if (cudaMemcpyAsync(sx, x_host, xbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return RGLRU_ERR_CUDA;
-    rc = rglru_prefill(s, p, sx, h0, conv_state_in, sy, (float *)sh, sc, workspace, workspace_bytes, cuda_stream);
-    if (rc != RGLRU_OK) return rc;
-    if (cudaMemcpyAsync(y_host, sy, xbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return RGLRU_ERR_CUDA;
-    if (cudaMemcpyAsync(h_T_host, sh, hbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return RGLRU_ERR_CUDA;
-    if (cudaMemcpyAsync(conv_state_out_host, sc, cbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return RGLRU_ERR_CUDA;
+
+    // Sequences are independent, so the batch is cut into chunks that move through three stages at once: host-to-device
+    // copy of chunk c+1, forward of chunk c, device-to-host copy of chunk c-1 (PCIe carries both directions at the same
+    // time).  Chunk boundaries must keep every pointer 16-byte aligned; otherwise the whole batch is one chunk.
+    HostPipe *hp = host_pipe();
+    const bool splittable = hp != nullptr && s->B > 1 && seq_x % 16 == 0 && seq_h % 16 == 0 && seq_c % 16 == 0;
+    const int nchunks = splittable ? (s->B < HostPipe::MAX_CHUNKS ? s->B : HostPipe::MAX_CHUNKS) : 1;
+    if (nchunks == 1) {
+        if (cudaMemcpyAsync(sx, x_host, xbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return RGLRU_ERR_CUDA;
+        rc = rglru_prefill(s, p, sx, h0, conv_state_in, sy, (float *)sh, sc, workspace, workspace_bytes, cuda_stream);
+        if (rc != RGLRU_OK) return rc;
+        if (cudaMemcpyAsync(y_host, sy, xbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return RGLRU_ERR_CUDA;
+        if (cudaMemcpyAsync(h_T_host, sh, hbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return RGLRU_ERR_CUDA;
+        if (cudaMemcpyAsync(conv_state_out_host, sc, cbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return RGLRU_ERR_CUDA;
+        return RGLRU_OK;
+    }
+    std::lock_guard<std::mutex> lock(hp->mutex);
+#define CK(call) do { if ((call) != cudaSuccess) return RGLRU_ERR_CUDA; } while (0)
+    CK(cudaEventRecord(hp->start, st));                      // everything below follows the work already on the stream
+    CK(cudaStreamWaitEvent(hp->in, hp->start, 0));
+    CK(cudaStreamWaitEvent(hp->out, hp->start, 0));
+    for (int c = 0; c < nchunks; ++c) {
+        const int b0 = (int)((long long)s->B * c / nchunks), b1 = (int)((long long)s->B * (c + 1) / nchunks);
+        rglru_shape_t sc_shape = *s;
+        sc_shape.B = b1 - b0;
+        const size_t xo = (size_t)b0 * seq_x, ho = (size_t)b0 * seq_h, co = (size_t)b0 * seq_c, xn = (size_t)(b1 - b0) * seq_x;
+        CK(cudaMemcpyAsync(sx + xo, (const char *)x_host + xo, xn, cudaMemcpyHostToDevice, hp->in));
+        CK(cudaEventRecord(hp->copied[c], hp->in));
+        CK(cudaStreamWaitEvent(st, hp->copied[c], 0));
+        rc = rglru_prefill(&sc_shape, p, sx + xo, h0 ? (const float *)((const char *)h0 + ho) : nullptr,
+                           conv_state_in ? (const char *)conv_state_in + co : nullptr, sy + xo, (float *)(sh + ho), sc + co, workspace,
+                           workspace_bytes, cuda_stream);
+        if (rc != RGLRU_OK) return rc;
+        CK(cudaEventRecord(hp->computed[c], st));
+        CK(cudaStreamWaitEvent(hp->out, hp->computed[c], 0));
+        CK(cudaMemcpyAsync((char *)y_host + xo, sy + xo, xn, cudaMemcpyDeviceToHost, hp->out));
+    }
+    CK(cudaMemcpyAsync(h_T_host, sh, hbytes, cudaMemcpyDeviceToHost, hp->out));
+    CK(cudaMemcpyAsync(conv_state_out_host, sc, cbytes, cudaMemcpyDeviceToHost, hp->out));
+    CK(cudaEventRecord(hp->done, hp->out));
+    CK(cudaStreamWaitEvent(st, hp->done, 0));                // later work on the caller's stream sees the results
+#undef CK
     return RGLRU_OK;
 }
 

@@ -152,3 +152,30 @@ def test_backward_tensor_core_path(oracle, B, T, H, with_y):
                          h0=inp["h0"].astype(np.float64), conv_state_in=inp["conv_state"].astype(np.float64))
     for k in gr:
         assert_close("d" + k, to_np(g[k]), gr[k], "bf16")
+
+
+def test_prefill_host_pipelined_chunks_match_device_prefill(oracle):
+    """rglru_prefill_host cuts the batch into chunks of sequences that are copied in, run and copied out concurrently;
+    the result must be the forward of the whole batch."""
+    import torch
+    from paper_2402_19427_b200 import binding
+    B, T, H = 5, 300, 2
+    D = 256 * H
+    inp = synth.make_inputs(B, T, D, H, io="bf16", seed=77, with_state=True, bias_scale=0.2)
+    params = binding.Params.from_numpy(inp["params"], "bf16")
+    h0 = to_dev(inp["h0"]); cs = to_dev(inp["conv_state"], "bf16")
+    x_pin = torch.from_numpy(inp["x"]).to(torch.bfloat16).pin_memory()
+    y_pin = torch.empty(B, T, D, dtype=torch.bfloat16).pin_memory()
+    hT_pin = torch.empty(B, D, dtype=torch.float32).pin_memory()
+    cs_pin = torch.empty(B, 3, D, dtype=torch.bfloat16).pin_memory()
+    shape = binding.make_shape(B, T, D, H, torch.bfloat16)
+    ws = binding.alloc_workspace(shape, binding.OP_PREFILL, h0.device)
+    staging = torch.empty(binding.host_staging_bytes(shape), dtype=torch.uint8, device=h0.device)
+    for _ in range(2):   # twice: the helper streams and events are reused
+        binding.prefill_host(x_pin, params, y_pin, hT_pin, cs_pin, staging, ws, h0=h0, conv_state_in=cs)
+        torch.cuda.synchronize()
+        assert binding.query_status(ws) == binding.OK
+        yr, hr, cr = oracle_prefill(oracle, inp, h0=inp["h0"].astype(np.float64), cs=inp["conv_state"].astype(np.float64))
+        assert_close("y", to_np(y_pin), yr, "bf16"); assert_close("h_T", to_np(hT_pin), hr, "bf16")
+        assert np.array_equal(to_np(cs_pin), cr)
+        y_pin.zero_()

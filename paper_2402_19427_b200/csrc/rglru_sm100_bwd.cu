@@ -176,6 +176,17 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
 // ------------------------------------------------------------------ element-wise kernels
 __device__ __forceinline__ float bf2f(__nv_bfloat16 v) { return __bfloat162float(v); }
 __device__ __forceinline__ float sigmoid_acc(float z) { return 1.0f / (1.0f + expf(-z)); }
+// Hardware-approximate versions for the per-element work (relative error ~1e-6, far inside the gradient tolerance)
+__device__ __forceinline__ float sigmoid_fast(float z) { return __frcp_rn(1.0f + __expf(-z)); }
+// 1 - exp(x) for x <= 0 without cancellation near 0
+__device__ __forceinline__ float one_minus_exp(float x) {
+    if (x > -0.25f) {   // -x (1 + x/2 + x^2/6 + x^3/24 + x^4/120 + x^5/720): relative truncation error < 2e-7
+        float pl = fmaf(x, 1.0f / 720.0f, 1.0f / 120.0f);
+        pl = fmaf(pl, x, 1.0f / 24.0f); pl = fmaf(pl, x, 1.0f / 6.0f); pl = fmaf(pl, x, 0.5f); pl = fmaf(pl, x, 1.0f);
+        return -x * pl;
+    }
+    return 1.0f - __expf(x);
+}
 // s = c softplus(-Lambda)   (Appendix A, with a = sigmoid(Lambda))
 __device__ __forceinline__ float decay_rate(float lambda, float c) {
     const float z = -lambda;
@@ -244,7 +255,7 @@ __global__ void __launch_bounds__(256) conv_forward_kernel(EwArgs a) {
 // a_t = exp(-s sigmoid(z_a + b_a)) from the stored pre-activation
 __device__ __forceinline__ float decay_from_z(const EwArgs &a, size_t tok, int h, int n, float s, float ba) {
     const float za = __half2float(a.z[((tok * a.H + h) * 2 + 0) * DH + n]);
-    return expf(-s * sigmoid_acc(za + ba));
+    return __expf(-s * sigmoid_fast(za + ba));
 }
 
 // Reverse scan, pass 1: per chunk the product of a_t and the carry a_first g_first it hands to earlier tokens when
@@ -255,12 +266,22 @@ __global__ void __launch_bounds__(256) scan_fold_kernel(EwArgs a) {
     const int t0 = c * CHUNK, t1 = min(T, t0 + CHUNK);
     const float s = decay_rate(a.lambda[d], a.c), ba = a.b_a[d];
     float carry = 0.0f, Q = 1.0f;
-    for (int t = t1 - 1; t >= t0; --t) {
-        const size_t tok = (size_t)b * T + t;
-        const float at = decay_from_z(a, tok, h, n, s, ba);
-        const float g = bf2f(a.dy[tok * D + d]) + carry;
-        carry = at * g;
-        Q *= at;
+    const size_t tokb = (size_t)b * T + (t1 - 8);
+    const size_t sD = (size_t)D, sZ = (size_t)a.H * 2 * DH;
+    const __nv_bfloat16 *p_dy = a.dy + tokb * sD + d;
+    const __half *p_z = a.z + tokb * sZ + (size_t)h * 2 * DH + n;
+    for (int tb = t1 - 8; tb >= t0; tb -= 8) {
+        float dyv[8], zav[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { dyv[k] = bf2f(p_dy[k * sD]); zav[k] = __half2float(p_z[k * sZ]); }
+#pragma unroll
+        for (int k = 7; k >= 0; --k) {
+            const float at = __expf(-s * sigmoid_fast(zav[k] + ba));
+            const float g = dyv[k] + carry;
+            carry = at * g;
+            Q *= at;
+        }
+        p_dy -= 8 * sD; p_z -= 8 * sZ;
     }
     a.fold[((size_t)b * a.nchunk + c) * D + d] = make_float2(Q, carry);
 }
@@ -289,43 +310,49 @@ __global__ void __launch_bounds__(256) scan_apply_kernel(EwArgs a) {
     const float dsdlam_neg = a.c * sigmoid_acc(-lam);
     float carry = a.xin[((size_t)b * a.nchunk + c) * D + d];
     float s_lam = 0.0f, s_ba = 0.0f, s_bx = 0.0f;
+    // running pointers at token t1 - 8 (the loop walks backwards in steps of eight tokens)
+    const size_t tokb = (size_t)b * T + (t1 - 8);
+    const size_t sD = (size_t)D, sZ = (size_t)a.H * 2 * DH;          // token strides of [tok][D] and [tok][H][2][256] arrays
+    const __nv_bfloat16 *p_dy = a.dy + tokb * sD + d, *p_y = a.y + (tokb - 1) * sD + d;
+    const __half *p_z = a.z + tokb * sZ + (size_t)h * 2 * DH + n, *p_u = a.u + tokb * sD + d;
+    __half *p_dz = a.dz + tokb * sZ + (size_t)h * 2 * DH + n;
+    float *p_du = a.du + tokb * sD + d;
+    __half *p_ta = a.dzT + ((size_t)h * 2 * DH + n) * a.BTp + tokb, *p_tx = p_ta + (size_t)DH * a.BTp;
+    const float h0v = a.h0 ? a.h0[(size_t)b * D + d] : 0.0f;
     for (int tb = t1 - 8; tb >= t0; tb -= 8) {
         float dyv[8], hpv[8], zav[8], zxv[8], uv[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-            const int t = tb + k;
-            const size_t tok = (size_t)b * T + t;
-            dyv[k] = bf2f(a.dy[tok * D + d]);
-            hpv[k] = t > 0 ? bf2f(a.y[(tok - 1) * D + d]) : (a.h0 ? a.h0[(size_t)b * D + d] : 0.0f);
-            zav[k] = __half2float(a.z[((tok * a.H + h) * 2 + 0) * DH + n]);
-            zxv[k] = __half2float(a.z[((tok * a.H + h) * 2 + 1) * DH + n]);
-            uv[k] = __half2float(a.u[tok * D + d]);
+            dyv[k] = bf2f(p_dy[k * sD]);
+            hpv[k] = (tb + k) > 0 ? bf2f(p_y[k * sD]) : h0v;
+            zav[k] = __half2float(p_z[k * sZ]);
+            zxv[k] = __half2float(p_z[k * sZ + DH]);
+            uv[k] = __half2float(p_u[k * sD]);
         }
         uint32_t pa[4], px[4];
 #pragma unroll
         for (int k = 7; k >= 0; --k) {
-            const size_t tok = (size_t)b * T + tb + k;
-            const float r = sigmoid_acc(zav[k] + ba), gi = sigmoid_acc(zxv[k] + bx);
-            const float L = -s * r, at = expf(L), mt = sqrtf(fmaxf(0.0f, -expm1f(2.0f * L)));
+            const float r = sigmoid_fast(zav[k] + ba), gi = sigmoid_fast(zxv[k] + bx);
+            const float L = -s * r, at = __expf(L), m2 = one_minus_exp(2.0f * L);
+            const float mt = sqrtf(m2), rm = m2 > 0.0f ? rsqrtf(m2) : 0.0f;
             const float g = dyv[k] + carry;
             carry = at * g;
             const float v = gi * uv[k];
-            const float dm_term = mt > 0.0f ? at * at * v / mt : 0.0f;
-            const float dL = g * (at * hpv[k] - dm_term);
+            const float dL = g * (at * hpv[k] - at * at * v * rm);
             const float dv = g * mt;
             const float dza = -s * dL * r * (1.0f - r), dzx = dv * uv[k] * gi * (1.0f - gi);
             s_lam = fmaf(dL * r, dsdlam_neg, s_lam);
             s_ba += dza; s_bx += dzx;
-            a.du[tok * D + d] = dv * gi;
+            p_du[k * sD] = dv * gi;
             const __half ha = to_half_sat(dza), hx = to_half_sat(dzx);
-            a.dz[((tok * a.H + h) * 2 + 0) * DH + n] = ha;
-            a.dz[((tok * a.H + h) * 2 + 1) * DH + n] = hx;
+            p_dz[k * sZ] = ha;
+            p_dz[k * sZ + DH] = hx;
             const uint32_t ba16 = (uint32_t)__half_as_ushort(ha), bx16 = (uint32_t)__half_as_ushort(hx);
             if (k & 1) { pa[k >> 1] = ba16 << 16; px[k >> 1] = bx16 << 16; } else { pa[k >> 1] |= ba16; px[k >> 1] |= bx16; }
         }
-        const size_t col = (size_t)b * T + tb;
-        *(uint4 *)(a.dzT + ((size_t)h * 2 * DH + n) * a.BTp + col) = make_uint4(pa[0], pa[1], pa[2], pa[3]);
-        *(uint4 *)(a.dzT + ((size_t)h * 2 * DH + DH + n) * a.BTp + col) = make_uint4(px[0], px[1], px[2], px[3]);
+        *(uint4 *)p_ta = make_uint4(pa[0], pa[1], pa[2], pa[3]);
+        *(uint4 *)p_tx = make_uint4(px[0], px[1], px[2], px[3]);
+        p_dy -= 8 * sD; p_y -= 8 * sD; p_z -= 8 * sZ; p_u -= 8 * sD; p_dz -= 8 * sZ; p_du -= 8 * sD; p_ta -= 8; p_tx -= 8;
     }
     float *pv = a.part_vec + ((size_t)b * a.nchunk + c) * 3 * D + d;
     pv[0] = s_lam; pv[(size_t)D] = s_ba; pv[(size_t)2 * D] = s_bx;

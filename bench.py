@@ -352,13 +352,14 @@ def measure_extras(binding, dev, peaks):
     dy = torch.randn(B, T, D, device=dev, generator=g).to(dt)
     shape = binding.make_shape(B, T, D, H, dt)
     ws = binding.alloc_workspace(shape, binding.OP_BACKWARD, dev)
-    binding.backward(x, params, dy, workspace=ws); torch.cuda.synchronize()
+    y_saved, _, _ = binding.prefill(x, params)          # a training step keeps the forward output for the backward
+    binding.backward(x, params, dy, y=y_saved, workspace=ws); torch.cuda.synchronize()
     e0.record()
-    binding.backward(x, params, dy, workspace=ws)
+    binding.backward(x, params, dy, y=y_saved, workspace=ws)
     e1.record(); torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
     bwd_flops = B * T * D * 12 * Dh
-    out["backward"] = {"workload": f"B={B} T={T} D_RNN={D} H={H} bf16 io", "tokens_per_s": B * T / (ms * 1e-3), "ms": ms,
+    out["backward"] = {"workload": f"B={B} T={T} D_RNN={D} H={H} bf16 io, forward output saved", "tokens_per_s": B * T / (ms * 1e-3), "ms": ms,
                        "gate_tflops_achieved": bwd_flops / (ms * 1e-3) / 1e12,
                        "roofline_frac": bwd_flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
     return out

@@ -12,7 +12,7 @@
 //                        and channel-major), the direct part of du (fp32), partial sums of dLambda, db_a, db_x
 //   4. GEMM              du += dz_a W_a + dz_x W_x
 //   5. GEMM (split K)    dW_a | dW_x = dz^T u over all tokens, fp32 partial sums per split, reduced in fixed order
-//   6. Conv1D adjoint    dx, dconv_w, dconv_b (shared with the shape-generic backward), fixed-order reductions
+//   6. Conv1D adjoint    dx, dconv_w, dconv_b with sliding windows, fixed-order reductions
 // h_{t-1} comes from the forward output y (bf16); when the caller has none the forward is run first.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -358,6 +358,51 @@ __global__ void __launch_bounds__(256) scan_apply_kernel(EwArgs a) {
     pv[0] = s_lam; pv[(size_t)D] = s_ba; pv[(size_t)2 * D] = s_bx;
 }
 
+// Conv1D adjoint: dx_t = sum_j w[j] du_{t+j} (t + j < T); per-chunk partial sums of dw[j] = sum_t du_t x_{t-j} and
+// db_c = sum_t du_t.  One thread per (sequence, chunk, channel) walks forward with sliding windows, so that every du and
+// every x is loaded once.  grid (D/256, nchunk, B)
+struct ConvBwdArgs {
+    int B, T, D, nchunk;
+    const __nv_bfloat16 *x, *conv_w, *cs_in;
+    const float *du;
+    __nv_bfloat16 *dx;
+    float *part_conv;   // [B*nchunk][5][D]
+};
+
+__global__ void __launch_bounds__(256) conv_backward_kernel(ConvBwdArgs a) {
+    const int d = blockIdx.x * 256 + threadIdx.x, c = blockIdx.y, b = blockIdx.z;
+    const int T = a.T, D = a.D;
+    const int t0 = c * CHUNK, t1 = min(T, t0 + CHUNK);
+    float w[4], sw[4] = {0.f, 0.f, 0.f, 0.f}, sb = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) w[j] = bf2f(a.conv_w[(size_t)j * D + d]);
+    auto xat = [&](int t) -> float {
+        if (t >= 0) return bf2f(a.x[((size_t)b * T + t) * D + d]);
+        return a.cs_in ? bf2f(a.cs_in[((size_t)b * 3 + (3 + t)) * D + d]) : 0.0f;
+    };
+    auto duat = [&](int t) -> float { return t < T ? a.du[((size_t)b * T + t) * D + d] : 0.0f; };
+    float x1 = xat(t0 - 1), x2 = xat(t0 - 2), x3 = xat(t0 - 3);     // x_{t-1}, x_{t-2}, x_{t-3}
+    float g0 = duat(t0), g1 = duat(t0 + 1), g2 = duat(t0 + 2);     // du_t, du_{t+1}, du_{t+2}
+    for (int tb = t0; tb < t1; tb += 8) {
+        float xs[8], gs[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { xs[k] = bf2f(a.x[((size_t)b * T + tb + k) * D + d]); gs[k] = duat(tb + k + 3); }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const float g3 = gs[k], x0 = xs[k];
+            a.dx[((size_t)b * T + tb + k) * D + d] = __float2bfloat16_rn(fmaf(w[3], g3, fmaf(w[2], g2, fmaf(w[1], g1, w[0] * g0))));
+            sw[0] = fmaf(g0, x0, sw[0]); sw[1] = fmaf(g0, x1, sw[1]); sw[2] = fmaf(g0, x2, sw[2]); sw[3] = fmaf(g0, x3, sw[3]);
+            sb += g0;
+            g0 = g1; g1 = g2; g2 = g3;
+            x3 = x2; x2 = x1; x1 = x0;
+        }
+    }
+    float *pc = a.part_conv + ((size_t)(b * a.nchunk + c) * 5) * D + d;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) pc[(size_t)j * D] = sw[j];
+    pc[(size_t)4 * D] = sb;
+}
+
 inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 struct BwdLayout {
@@ -389,7 +434,7 @@ BwdLayout bwd_layout(int B, int T, int D, int H) {
     L.off_fold = take((size_t)B * L.nchunk * D * 8);
     L.off_xin = take((size_t)B * L.nchunk * D * 4);
     L.off_pvec = take((size_t)B * L.nchunk * 3 * D * 4);
-    L.off_pconv = take((size_t)B * L.nchunk_conv * 5 * D * 4);
+    L.off_pconv = take((size_t)B * L.nchunk * 5 * D * 4);
     L.off_pdw = take((size_t)L.S * 2 * H * DH * DH * 4);
     L.off_wt = take((size_t)H * DH * 2 * DH * 2);
     L.off_w16 = take((size_t)H * DH * 2 * DH * 2);
@@ -504,9 +549,13 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
     if ((e = reduce_partials(a.part_vec, nparts, (size_t)3 * D, q.dlambda, D, st)) != cudaSuccess) return e;
     if ((e = reduce_partials(a.part_vec + D, nparts, (size_t)3 * D, q.db_a, D, st)) != cudaSuccess) return e;
     if ((e = reduce_partials(a.part_vec + 2 * (size_t)D, nparts, (size_t)3 * D, q.db_x, D, st)) != cudaSuccess) return e;
-    q.hp = du;
-    q.part_conv = (float *)(ws + L.off_pconv);
-    if ((e = generic_bwd_conv_and_reduce(q, RGLRU_BF16, st)) != cudaSuccess) return e;
+    ConvBwdArgs cb{};
+    cb.B = B; cb.T = T; cb.D = D; cb.nchunk = L.nchunk;
+    cb.x = a.x; cb.conv_w = a.conv_w; cb.cs_in = a.cs_in; cb.du = du; cb.dx = (__nv_bfloat16 *)q.dx;
+    cb.part_conv = (float *)(ws + L.off_pconv);
+    conv_backward_kernel<<<grid_ew, 256, 0, st>>>(cb);
+    if ((e = reduce_partials(cb.part_conv, nparts, (size_t)5 * D, q.dconv_w, (size_t)4 * D, st)) != cudaSuccess) return e;
+    if ((e = reduce_partials(cb.part_conv + 4 * (size_t)D, nparts, (size_t)5 * D, q.dconv_b, D, st)) != cudaSuccess) return e;
     return cudaGetLastError();
 }
 

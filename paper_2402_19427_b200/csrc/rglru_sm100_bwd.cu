@@ -34,7 +34,7 @@ constexpr uint32_t A_STAGE_BYTES = 128 * 128;   // 128 rows x 64 bf16
 constexpr uint32_t B_STAGE_BYTES = 256 * 128;   // 256 rows x 64 bf16
 constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr uint32_t GEMM_SMEM_BAR = GEMM_STAGES * STAGE_BYTES;
-constexpr uint32_t GEMM_SMEM_TOTAL = GEMM_SMEM_BAR + (2 * GEMM_STAGES + 1) * 8 + 16;
+constexpr uint32_t GEMM_SMEM_TOTAL = GEMM_SMEM_BAR + (2 * GEMM_STAGES + 4) * 8 + 16;
 constexpr uint32_t GEMM_SMEM_ALLOC = GEMM_SMEM_TOTAL + 1024;
 
 enum { MODE_Z = 0, MODE_DU = 1, MODE_DW = 2 };
@@ -44,6 +44,7 @@ struct GemmArgs {
     alignas(64) CUtensorMap tm_b0;   // B rows (N side), K innermost
     alignas(64) CUtensorMap tm_b1;   // MODE_Z: the second gate's weights (grid.y selects)
     int mode, H, D;
+    int nx, ny;        // tile grid: nx x ny x H
     int kblocks;       // 64-wide K blocks per CTA
     int rows_valid;    // MODE_Z / MODE_DU: number of tokens; MODE_DW: 512
     void *out;         // MODE_Z: __half z[tok][H][2][256]; MODE_DU: float du[tok][D] (+=); MODE_DW: float part[split][2][H][256][256]
@@ -51,11 +52,13 @@ struct GemmArgs {
     unsigned long long spin_ns;
 };
 
-// C[128 x 256] = A[128 x K] B[256 x K]^T for one tile; A and B tiles arrive by tiled TMA in the 128-byte-swizzled
-// K-major layout, accumulate in tensor memory (fp32), and leave through the four epilogue warps.
-//   MODE_Z : grid (token tiles, 2 gates, H)   A = u[tok][h][k]        B = W_gate[h][out][k]
-//   MODE_DU: grid (token tiles, 1, H)         A = dz[tok][h][k=512]   B = W^T[h][in][k=512]
-//   MODE_DW: grid (4 row tiles, splits, H)    A = dz^T[h][row][tok]   B = u^T[h][in][tok], K = this split's tokens
+// C[128 x 256] = A[128 x K] B[256 x K]^T per tile; A and B tiles arrive by tiled TMA in the 128-byte-swizzled K-major
+// layout, accumulate in tensor memory (fp32), and leave through the four epilogue warps.  CTAs are persistent: each
+// walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... with two accumulators, so that the epilogue of one tile overlaps
+// the loads and MMAs of the next.  Tile number -> (x, y, z) with x fastest:
+//   MODE_Z : (token tiles, 2 gates, H)   A = u[tok][h][k]        B = W_gate[h][out][k]
+//   MODE_DU: (token tiles, 1, H)         A = dz[tok][h][k=512]   B = W^T[h][in][k=512]
+//   MODE_DW: (4 row tiles, splits, H)    A = dz^T[h][row][tok]   B = u^T[h][in][tok], K = this split's tokens
 __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_constant__ GemmArgs p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -64,20 +67,21 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
     const uint32_t bar0 = base + GEMM_SMEM_BAR;
     auto BAR_FULL = [&](int s) { return bar0 + 8u * s; };
     auto BAR_EMPTY = [&](int s) { return bar0 + 8u * (GEMM_STAGES + s); };
-    const uint32_t BAR_ACC = bar0 + 8u * (2 * GEMM_STAGES);
-    uint32_t *tmem_base_s = (uint32_t *)(smem + GEMM_SMEM_BAR + (2 * GEMM_STAGES + 1) * 8);
+    auto BAR_ACCFULL = [&](int a) { return bar0 + 8u * (2 * GEMM_STAGES + a); };
+    auto BAR_ACCEMPTY = [&](int a) { return bar0 + 8u * (2 * GEMM_STAGES + 2 + a); };
+    uint32_t *tmem_base_s = (uint32_t *)(smem + GEMM_SMEM_BAR + (2 * GEMM_STAGES + 4) * 8);
     volatile int *abort_flag = (volatile int *)(tmem_base_s + 1);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int h = blockIdx.z;
     const unsigned long long spin = p.spin_ns;
+    const int ntiles = p.nx * p.ny * p.H;
 
     if (tid == 0) {
         for (int s = 0; s < GEMM_STAGES; ++s) { mbar_init(BAR_FULL(s), 1); mbar_init(BAR_EMPTY(s), 1); }
-        mbar_init(BAR_ACC, 1);
+        for (int a = 0; a < 2; ++a) { mbar_init(BAR_ACCFULL(a), 1); mbar_init(BAR_ACCEMPTY(a), 4); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) { tmem_alloc(smem_u32(tmem_base_s), 256); tmem_relinquish(); }
+    if (warp == 1) { tmem_alloc(smem_u32(tmem_base_s), 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -87,20 +91,24 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
     if (warp == 0) {
         // ---- TMA producer
         if (lane == 0) {
-            const CUtensorMap *tb = (p.mode == MODE_Z && blockIdx.y == 1) ? &p.tm_b1 : &p.tm_b0;
-            for (int kb = 0; kb < p.kblocks; ++kb) {
-                const int s = kb % GEMM_STAGES;
-                ok = mbar_wait(BAR_EMPTY(s), ((kb / GEMM_STAGES) & 1) ^ 1, spin, abort_flag);
-                if (!ok) break;
-                mbar_expect_tx(BAR_FULL(s), STAGE_BYTES);
-                const uint32_t a_dst = base + s * STAGE_BYTES, b_dst = a_dst + A_STAGE_BYTES;
-                if (p.mode == MODE_DW) {
-                    const int k0 = ((int)blockIdx.y * p.kblocks + kb) * 64;
-                    tma_load_3d(a_dst, &p.tm_a, k0, (int)blockIdx.x * 128, h, BAR_FULL(s));
-                    tma_load_3d(b_dst, tb, k0, 0, h, BAR_FULL(s));
-                } else {
-                    tma_load_3d(a_dst, &p.tm_a, kb * 64, h, (int)blockIdx.x * 128, BAR_FULL(s));
-                    tma_load_3d(b_dst, tb, kb * 64, 0, h, BAR_FULL(s));
+            int kbg = 0;   // K blocks issued so far, over all tiles (ring position)
+            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+                const int tx = tile % p.nx, ty = (tile / p.nx) % p.ny, h = tile / (p.nx * p.ny);
+                const CUtensorMap *tb = (p.mode == MODE_Z && ty == 1) ? &p.tm_b1 : &p.tm_b0;
+                for (int kb = 0; kb < p.kblocks; ++kb, ++kbg) {
+                    const int s = kbg % GEMM_STAGES;
+                    ok = mbar_wait(BAR_EMPTY(s), ((kbg / GEMM_STAGES) & 1) ^ 1, spin, abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(BAR_FULL(s), STAGE_BYTES);
+                    const uint32_t a_dst = base + s * STAGE_BYTES, b_dst = a_dst + A_STAGE_BYTES;
+                    if (p.mode == MODE_DW) {
+                        const int k0 = (ty * p.kblocks + kb) * 64;
+                        tma_load_3d(a_dst, &p.tm_a, k0, tx * 128, h, BAR_FULL(s));
+                        tma_load_3d(b_dst, tb, k0, 0, h, BAR_FULL(s));
+                    } else {
+                        tma_load_3d(a_dst, &p.tm_a, kb * 64, h, tx * 128, BAR_FULL(s));
+                        tma_load_3d(b_dst, tb, kb * 64, 0, h, BAR_FULL(s));
+                    }
                 }
             }
             if (!ok) { *abort_flag = 1; atomicExch(p.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT); }
@@ -109,28 +117,38 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
         // ---- MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_f16(128, 256);
-            for (int kb = 0; kb < p.kblocks; ++kb) {
-                const int s = kb % GEMM_STAGES;
-                ok = mbar_wait(BAR_FULL(s), (kb / GEMM_STAGES) & 1, spin, abort_flag);
+            int kbg = 0, it = 0;
+            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
+                const int acc = it & 1;
+                ok = mbar_wait(BAR_ACCEMPTY(acc), ((it >> 1) & 1) ^ 1, spin, abort_flag);   // epilogue of tile it - 2 done
                 if (!ok) break;
-                tc_fence_after();
-                const uint32_t a_src = base + s * STAGE_BYTES, b_src = a_src + A_STAGE_BYTES;
+                for (int kb = 0; kb < p.kblocks; ++kb, ++kbg) {
+                    const int s = kbg % GEMM_STAGES;
+                    ok = mbar_wait(BAR_FULL(s), (kbg / GEMM_STAGES) & 1, spin, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_src = base + s * STAGE_BYTES, b_src = a_src + A_STAGE_BYTES;
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    mma_ss(tmem, make_desc_sw128(a_src + ks * 32), make_desc_sw128(b_src + ks * 32), idesc, (kb | ks) != 0);
-                tc_commit(BAR_EMPTY(s));
+                    for (int ks = 0; ks < 4; ++ks)
+                        mma_ss(tmem + acc * 256, make_desc_sw128(a_src + ks * 32), make_desc_sw128(b_src + ks * 32), idesc, (kb | ks) != 0);
+                    tc_commit(BAR_EMPTY(s));
+                }
+                if (ok) tc_commit(BAR_ACCFULL(acc));
             }
-            if (ok) tc_commit(BAR_ACC);
-            else { *abort_flag = 1; atomicExch(p.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT); }
+            if (!ok) { *abort_flag = 1; atomicExch(p.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT); }
         }
     } else {
         // ---- epilogue: warp owns TMEM lanes 32 (warp & 3) .. +31 = rows of the tile
         const int q = warp & 3;
-        const int row = (int)blockIdx.x * 128 + q * 32 + lane;
-        ok = warp_wait(BAR_ACC, 0, spin, abort_flag);
-        if (ok) {
+        int it = 0;
+        for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
+            const int tx = tile % p.nx, ty = (tile / p.nx) % p.ny, h = tile / (p.nx * p.ny);
+            const int acc = it & 1;
+            const int row = tx * 128 + q * 32 + lane;
+            ok = warp_wait(BAR_ACCFULL(acc), (it >> 1) & 1, spin, abort_flag);
+            if (!ok) break;
             tc_fence_after();
-            const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16);
+            const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16) + acc * 256;
             const bool valid = row < p.rows_valid;
 #pragma unroll 1
             for (int c0 = 0; c0 < 256; c0 += 32) {
@@ -139,7 +157,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                 tmem_ld_wait();
                 if (!valid) continue;
                 if (p.mode == MODE_Z) {
-                    __half *dst = (__half *)p.out + (((size_t)row * p.H + h) * 2 + blockIdx.y) * 256 + c0;
+                    __half *dst = (__half *)p.out + (((size_t)row * p.H + h) * 2 + ty) * 256 + c0;
                     uint32_t w[16];
 #pragma unroll
                     for (int j = 0; j < 16; ++j) { const __half2 hh = __floats2half2_rn(lo2(v[j]), hi2(v[j])); w[j] = *(const uint32_t *)&hh; }
@@ -155,14 +173,16 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                     }
                 } else {
                     const int g = row >> 8, o_row = row & 255;
-                    float4 *dst = (float4 *)((float *)p.out + ((((size_t)blockIdx.y * 2 + g) * p.H + h) * 256 + o_row) * 256 + c0);
+                    float4 *dst = (float4 *)((float *)p.out + ((((size_t)ty * 2 + g) * p.H + h) * 256 + o_row) * 256 + c0);
 #pragma unroll
                     for (int j = 0; j < 8; ++j) dst[j] = make_float4(lo2(v[2 * j]), hi2(v[2 * j]), lo2(v[2 * j + 1]), hi2(v[2 * j + 1]));
                 }
             }
-        } else if (lane == 0) {
-            *abort_flag = 1; atomicExch(p.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(BAR_ACCEMPTY(acc));   // this accumulator may be overwritten
         }
+        if (!ok && lane == 0) { *abort_flag = 1; atomicExch(p.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT); }
     }
     if (*abort_flag) {   // let copies and MMAs in flight land before shared and tensor memory are given back
         const uint64_t tw = gtimer();
@@ -170,7 +190,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, 256);
+    if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
 // ------------------------------------------------------------------ element-wise kernels
@@ -405,6 +425,13 @@ __global__ void __launch_bounds__(256) conv_backward_kernel(ConvBwdArgs a) {
 
 inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 
+unsigned gemm_grid(const GemmArgs &g) {
+    int dev = 0, nsm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&nsm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || nsm <= 0) nsm = 148;
+    const int ntiles = g.nx * g.ny * g.H;
+    return (unsigned)(ntiles < nsm ? ntiles : nsm);
+}
+
 struct BwdLayout {
     size_t BT, BTp, off_u, off_uT, off_z, off_dz, off_dzT, off_du, off_y, off_hT, off_cs, off_fold, off_xin, off_pvec, off_pconv, off_pdw,
         off_wt, off_w16, off_fws, total;
@@ -512,7 +539,8 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
             !encode_map16_3d(&g.tm_b1, W16 + (size_t)H * DH * DH, db, sb, bb, true))
             return cudaErrorNotSupported;
         g.mode = MODE_Z; g.kblocks = DH / 64; g.rows_valid = (int)BT; g.out = z;
-        tc_gemm_kernel<<<dim3(mtiles, 2, H), GEMM_THREADS, GEMM_SMEM_ALLOC, st>>>(g);
+        g.nx = (int)mtiles; g.ny = 2;
+        tc_gemm_kernel<<<gemm_grid(g), GEMM_THREADS, GEMM_SMEM_ALLOC, st>>>(g);
     }
     // 3. reverse scan and element-wise adjoints
     scan_fold_kernel<<<grid_ew, 256, 0, st>>>(a);
@@ -527,7 +555,8 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
         if (!encode_map16_3d(&g.tm_a, dz, da, sa, ba, true) || !encode_map16_3d(&g.tm_b0, WT, db, sb, bb, true)) return cudaErrorNotSupported;
         g.tm_b1 = g.tm_b0;
         g.mode = MODE_DU; g.kblocks = 2 * DH / 64; g.rows_valid = (int)BT; g.out = du;
-        tc_gemm_kernel<<<dim3(mtiles, 1, H), GEMM_THREADS, GEMM_SMEM_ALLOC, st>>>(g);
+        g.nx = (int)mtiles; g.ny = 1;
+        tc_gemm_kernel<<<gemm_grid(g), GEMM_THREADS, GEMM_SMEM_ALLOC, st>>>(g);
     }
     // 5. dW = dz^T u, split over the tokens, then a fixed-order sum of the splits
     {
@@ -539,7 +568,8 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
         g.tm_b1 = g.tm_b0;
         float *part = (float *)(ws + L.off_pdw);
         g.mode = MODE_DW; g.kblocks = L.kb_per_split; g.rows_valid = 2 * DH; g.out = part;
-        tc_gemm_kernel<<<dim3(4, L.S, H), GEMM_THREADS, GEMM_SMEM_ALLOC, st>>>(g);
+        g.nx = 4; g.ny = L.S;
+        tc_gemm_kernel<<<gemm_grid(g), GEMM_THREADS, GEMM_SMEM_ALLOC, st>>>(g);
         const size_t wsz = (size_t)H * DH * DH;
         if ((e = reduce_partials(part, L.S, 2 * wsz, q.dW_a, wsz, st)) != cudaSuccess) return e;
         if ((e = reduce_partials(part + wsz, L.S, 2 * wsz, q.dW_x, wsz, st)) != cudaSuccess) return e;

@@ -108,7 +108,25 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
     const int T = f.T, D = f.D, S = p.S;
     const int group = blockIdx.x / S, kcta = blockIdx.x % S;  // group = head * 2 + half
     const int head = group >> 1, half = group & 1;
-    const int n_my_tiles = (p.tiles_total - kcta + S - 1) / S;
+    // Work of this CTA.  Sequences are dealt out whole where that keeps the S CTAs of the half-head balanced: CTA kcta
+    // gets sequences kcta, kcta + S, ... of the first (B / S) * S ones and walks each from start to end, so a tile's
+    // incoming state is simply the state the CTA itself reached ("local" tiles: no record, no look-back).  The B % S
+    // sequences left over are split in time, tile g of them going to CTA g % S ("shared" tiles, decoupled look-back).
+    // Shared tiles come first, so that the S CTAs pass through them in step.
+    const int B_whole = (f.B / S) * S, shared_tiles = (f.B - B_whole) * p.tps;
+    const int n_shared = kcta < shared_tiles ? (shared_tiles - kcta + S - 1) / S : 0;
+    const int n_my_tiles = n_shared + (B_whole / S) * p.tps;
+    // tile number `it` of this CTA -> sequence b, tile ti within it; true when it is a shared tile
+    auto tile_of = [&](int it, int &b, int &ti) -> bool {
+        if (it < n_shared) {
+            const int g = kcta + it * S;
+            b = B_whole + g / p.tps; ti = g % p.tps;
+            return true;
+        }
+        const int j = it - n_shared;
+        b = kcta + (j / p.tps) * S; ti = j % p.tps;
+        return false;
+    };
     const unsigned long long spin = p.spin_ns;
 
     if (tid == 0) {
@@ -180,7 +198,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         int slab_n = 0;
         bool ok = true;
         for (int it = 0; it < n_my_tiles && ok; ++it) {
-            const int g = kcta + it * S, ti = g % p.tps;
+            int b, ti;
+            tile_of(it, b, ti);
             const int t0 = ti * TILE_N;
             const int st = it % US;
             ok = warp_wait(BAR_UEMPTY(st), ((it / US) & 1) ^ 1, spin, abort_flag);
@@ -267,7 +286,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         int slab_n = 0;
         bool ok = true;
         for (int it = 0; it < n_my_tiles && ok; ++it) {
-            const int g = kcta + it * S, b = g / p.tps, ti = g % p.tps;
+            int b, ti;
+            const bool shared = tile_of(it, b, ti);
+            const int g = b * p.tps + ti;   // tile number within the half-head: index of its carry record
             const int t0 = ti * TILE_N;
             const int nslab = min(TILE_N / SLAB, (T - t0 + SLAB - 1) / SLAB);
             for (int s = 0; s < nslab; ++s, ++slab_n) {
@@ -359,7 +380,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         float h_prev_own = 0.0f;  // state at the end of this CTA's previous tile
         bool ok = true;
         for (int it = 0; it < n_my_tiles && ok; ++it) {
-            const int g = kcta + it * S, b = g / p.tps, ti = g % p.tps;
+            int b, ti;
+            const bool shared = tile_of(it, b, ti);
+            const int g = b * p.tps + ti;   // tile number within the half-head: index of its carry record
             const int t0 = ti * TILE_N;
             const int st = it % US;
             const int nv = max(0, min(EPI_TOK, T - t0 - k * EPI_TOK));  // valid tokens of this warp
@@ -417,7 +440,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             const float P_0 = k ? other.x : P, hl_0 = k ? other.y : hl;     // tokens [0, 64)
             const float P_1 = k ? P : other.x, hl_1 = k ? hl : other.y;     // tokens [64, 128)
             const float P_t = P_0 * P_1, hl_t = fmaf(P_1, hl_0, hl_1);      // whole tile
-            if (S > 1 && k == 1) {
+            if (shared && S > 1 && k == 1) {
                 uint4 rec;
                 rec.x = __float_as_uint(P_t); rec.y = p.tag; rec.z = __float_as_uint(hl_t); rec.w = p.tag;
                 uint4 *dst = p.agg + ((size_t)group * p.tiles_total + g) * CH + c_own;
@@ -428,7 +451,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             //      the aggregates that the other CTAs published for the tiles in between (decoupled look-back)
             float h;
             int nback;
-            if (ti == 0 || (S > 1 && ti < S)) {
+            if (!shared) {
+                h = ti == 0 ? (f.h0 ? f.h0[(size_t)b * D + d] : 0.0f) : h_prev_own;
+                nback = 0;
+            } else if (ti == 0 || (S > 1 && ti < S)) {
                 h = f.h0 ? f.h0[(size_t)b * D + d] : 0.0f;
                 nback = ti;
             } else {

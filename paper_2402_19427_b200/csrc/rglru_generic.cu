@@ -429,18 +429,6 @@ cudaError_t reduce_partials(const float *in, int nparts, size_t stride, float *o
     return cudaGetLastError();
 }
 
-// Conv1D adjoint from du (fp32, in q.hp): dx, and dconv_w / dconv_b through per-chunk partial sums in q.part_conv.
-cudaError_t generic_bwd_conv_and_reduce(BwdArgs &q, int io, cudaStream_t st) {
-    const int B = q.B, T = q.T, D = q.D;
-    q.nchunk = (T + GENERIC_BWD_CHUNK - 1) / GENERIC_BWD_CHUNK;
-    dim3 g5((D + NT - 1) / NT, q.nchunk, B);
-    if (io == RGLRU_F32) generic_bwd_conv_kernel<float><<<g5, NT, 0, st>>>(q);
-    else generic_bwd_conv_kernel<__nv_bfloat16><<<g5, NT, 0, st>>>(q);
-    cudaError_t e = reduce_partials(q.part_conv, B * q.nchunk, (size_t)5 * D, q.dconv_w, (size_t)4 * D, st);
-    if (e != cudaSuccess) return e;
-    return reduce_partials(q.part_conv + 4 * (size_t)D, B * q.nchunk, (size_t)5 * D, q.dconv_b, D, st);
-}
-
 size_t generic_backward_workspace_bytes(int B, int T, int D, int H) {
     const size_t btd = (size_t)B * T * D, Dh = D / H;
     const int nchunk = (T + GENERIC_BWD_CHUNK - 1) / GENERIC_BWD_CHUNK;

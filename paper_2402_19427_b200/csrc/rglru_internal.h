@@ -78,8 +78,7 @@ bool sm100_backward_supported(int B, int T, int D, int H, int io);
 size_t sm100_backward_workspace_bytes(int B, int T, int D, int H);
 cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &b, const void *y_saved, void *ws_body, size_t ws_body_bytes, uint32_t *status,
                            cudaStream_t st);
-// pieces of the generic backward that the tensor-core backward reuses (du in b.hp -> dx and conv gradients; fixed-order sums)
-cudaError_t generic_bwd_conv_and_reduce(BwdArgs &q, int io, cudaStream_t st);
+// out[i] = sum over p of in[p * stride + i] in ascending p (fixed order: run-to-run identical results)
 cudaError_t reduce_partials(const float *in, int nparts, size_t stride, float *out, size_t n, cudaStream_t st);
 
 }  // namespace rglru

@@ -287,8 +287,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         bool ok = true;
         for (int it = 0; it < n_my_tiles && ok; ++it) {
             int b, ti;
-            const bool shared = tile_of(it, b, ti);
-            const int g = b * p.tps + ti;   // tile number within the half-head: index of its carry record
+            tile_of(it, b, ti);
             const int t0 = ti * TILE_N;
             const int nslab = min(TILE_N / SLAB, (T - t0 + SLAB - 1) / SLAB);
             for (int s = 0; s < nslab; ++s, ++slab_n) {
@@ -374,7 +373,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
                        (uint32_t)(k * EPI_TOK) * 128u;
         const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16);
         uint16_t *y_s = (uint16_t *)(smem + SMEM_Y + (uint32_t)k * Y_HALF_BYTES + (uint32_t)c_own * 2u);  // this thread's column of the y staging tile
-        __nv_bfloat16 *y = (__nv_bfloat16 *)f.y;
         const __nv_bfloat16 *x = (const __nv_bfloat16 *)f.x;
         const __nv_bfloat16 *cs_in = (const __nv_bfloat16 *)f.cs_in;
         float h_prev_own = 0.0f;  // state at the end of this CTA's previous tile

@@ -272,12 +272,6 @@ __global__ void __launch_bounds__(256) conv_forward_kernel(EwArgs a) {
     }
 }
 
-// a_t = exp(-s sigmoid(z_a + b_a)) from the stored pre-activation
-__device__ __forceinline__ float decay_from_z(const EwArgs &a, size_t tok, int h, int n, float s, float ba) {
-    const float za = __half2float(a.z[((tok * a.H + h) * 2 + 0) * DH + n]);
-    return __expf(-s * sigmoid_fast(za + ba));
-}
-
 // Reverse scan, pass 1: per chunk the product of a_t and the carry a_first g_first it hands to earlier tokens when
 // nothing comes in from later ones.  grid (D/256, nchunk, B)
 __global__ void __launch_bounds__(256) scan_fold_kernel(EwArgs a) {

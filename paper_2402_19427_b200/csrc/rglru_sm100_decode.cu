@@ -78,6 +78,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     int timed_out = 0;
     volatile int no_abort = 0;
 
+    // Programmatic dependent launch: the next kernel on the stream (typically the next decode step) may be scheduled
+    // as SMs free up, and runs its own prologue -- barrier set-up, tensor-memory allocation, the weight copies, the
+    // conv taps -- while this step is still finishing; it touches x, h and the conv state only after griddepcontrol.wait.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) {
         mbar_init(BAR_W, 1);
         mbar_init(BAR_ACC, 1);
@@ -119,6 +123,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
         __nv_bfloat16 *cs = (__nv_bfloat16 *)f.cs_out;   // in/out
         const uint32_t u_kb = SMEM_U + (uint32_t)(dl >> 6) * KBLOCK_BYTES;
         const uint32_t chunk = (uint32_t)(dl & 63) >> 3;
+        // everything above reads only parameters; x and the state may have been written by the kernel just before this
+        // one on the stream, whose completion (and visibility of its stores) is awaited here
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         // all global loads of the phase are issued before anything waits on them
         constexpr int NIT = NB_MAX / 16;
         uint4 xv[NIT], r0[NIT], r1[NIT], r2[NIT];   // x_t and x_{t-3}, x_{t-2}, x_{t-1} per sequence
@@ -299,8 +306,13 @@ cudaError_t sm100_decode(const FwdArgs &a, cudaStream_t st) {
     p.ntile = (a.B + NB - 1) / NB;
     p.spin_ns = g_spin_limit_ns;
     dim3 grid(2u * (unsigned)a.H * (unsigned)p.ntile), block(NTHREADS);
-    sm100_decode_kernel<<<grid, block, SMEM_ALLOC, st>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = SMEM_ALLOC; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see griddepcontrol in the kernel
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, sm100_decode_kernel, p);
 }
 
 }  // namespace rglru

@@ -14,7 +14,7 @@
 //     bf16 value, the term i_t * u_t of Eq. 4 takes bf16(u) + remainder, which is u to 16 mantissa bits;
 //   * one thread issues Z^T = W U^T for both gates (M = 128 channels, N = sequences of the tile, K = 256) with
 //     fp32 accumulators in tensor memory;
-//   * all eight warps run the epilogue: channel on the TMEM lane, sequences along the columns; gates, log-space
+//   * all sixteen warps run the epilogue: channel on the TMEM lane, sequences along the columns; gates, log-space
 //     decay and h <- a h + sqrt(1 - a^2) (i u) in fp32, h and y written with lane-contiguous stores.
 // Waits on the two mbarriers are bounded and end in RGLRU_ERR_TIMEOUT; the only cluster barriers come before them.
 #include <cuda.h>
@@ -32,7 +32,7 @@ using namespace ptx;
 constexpr int DH = 256;        // head width
 constexpr int CH = 128;        // channels per CTA
 constexpr int NB_MAX = 128;    // sequences per batch tile, at most
-constexpr int NTHREADS = 256;
+constexpr int NTHREADS = 512;
 constexpr uint32_t KBLOCK_BYTES = 128 * 128;               // 128 rows x 64 bf16: one K block of an operand tile
 constexpr uint32_t SMEM_WA = 0;
 constexpr uint32_t SMEM_WX = SMEM_WA + 4 * KBLOCK_BYTES;
@@ -107,7 +107,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     }
     __syncwarp();
 
-    // ---- conv phase: thread = (8-channel chunk c, sequences n = tid/16, tid/16 + 16, ...)
+    // ---- conv phase: thread = (8-channel chunk c, sequences n = tid/16, tid/16 + 32, ...)
     {
         const int c = tid & 15;
         const int dl = (int)rank * CH + c * 8;          // channel within the head
@@ -127,11 +127,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
         // one on the stream, whose completion (and visibility of its stores) is awaited here
         asm volatile("griddepcontrol.wait;" ::: "memory");
         // all global loads of the phase are issued before anything waits on them
-        constexpr int NIT = NB_MAX / 16;
+        constexpr int NIT = NB_MAX / 32;
         uint4 xv[NIT], r0[NIT], r1[NIT], r2[NIT];   // x_t and x_{t-3}, x_{t-2}, x_{t-1} per sequence
 #pragma unroll
         for (int i = 0; i < NIT; ++i) {
-            const int n = (tid >> 4) + 16 * i, b = b0 + n;
+            const int n = (tid >> 4) + 32 * i, b = b0 + n;
             if (n < NB && b < B) {
                 xv[i] = *(const uint4 *)(x + (size_t)b * D + d);
                 r0[i] = *(const uint4 *)(cs + ((size_t)b * 3 + 0) * D + d);
@@ -145,7 +145,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
                        w2[4] = {w[2].x, w[2].y, w[2].z, w[2].w}, w3[4] = {w[3].x, w[3].y, w[3].z, w[3].w};
 #pragma unroll
         for (int i = 0; i < NIT; ++i) {
-            const int n = (tid >> 4) + 16 * i, b = b0 + n;
+            const int n = (tid >> 4) + 32 * i, b = b0 + n;
             if (n >= NB) break;
             uint4 uo = make_uint4(0u, 0u, 0u, 0u);
             if (b < B) {
@@ -175,97 +175,107 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
         }
     }
     fence_async_all();   // generic-proxy writes (local and remote) before the tensor core reads them
-    cluster_arrive();
-    cluster_wait();      // both halves of the U tile are in place in both CTAs
+    __syncthreads();     // this CTA's half of the U tile is complete in its own shared memory
+    cluster_arrive();    // ... and, once the peer has waited, in the peer's
 
-    // ---- epilogue: warp (q, k) owns channels 32 q .. 32 q + 31 and half k of the tile's sequences
-    const int q = warp & 3, k = warp >> 2;
-        const int c_own = q * 32 + lane;
-        const int dl = (int)rank * CH + c_own;
-        const size_t d = (size_t)head * DH + dl;
-        const float lam = f.lambda[d];
-        const float zl = -lam;
-        const float s = f.c * (zl > 0.0f ? zl + log1pf(expf(-zl)) : log1pf(expf(zl)));
-        const bool poly = __all_sync(0xffffffffu, s <= S_POLY);
-        const f32x2 hba2 = pack2(0.5f * f.b_a[d], 0.5f * f.b_a[d]), hbx2 = pack2(0.5f * f.b_x[d], 0.5f * f.b_x[d]), s2 = pack2(s, s);
-        const uint8_t *u_col = smem + SMEM_U + (uint32_t)(dl >> 6) * KBLOCK_BYTES + (uint32_t)(dl & 7) * 2u;
-        const uint32_t u_chunk = (uint32_t)(dl & 63) >> 3;
-        const uint8_t *r_col = smem + SMEM_R + (uint32_t)c_own * 2u;
-        float *h = f.h_T;                                 // in/out
-        __nv_bfloat16 *y = (__nv_bfloat16 *)f.y;
-        const int nh = NB >> 1;                           // multiple of 8
-        const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16);
-        // the recurrent state of this warp's sequences is fetched while the tensor core works
-        float hv[NB_MAX / 2];
+    // ---- epilogue set-up: warp (q, kq) owns channels 32 q .. 32 q + 31 and quarter kq of the tile's sequences
+    const int q = warp & 3, kq = warp >> 2;
+    const int c_own = q * 32 + lane;
+    const int dl = (int)rank * CH + c_own;
+    const size_t d = (size_t)head * DH + dl;
+    const float lam = f.lambda[d];
+    const float zl = -lam;
+    const float s = f.c * (zl > 0.0f ? zl + log1pf(expf(-zl)) : log1pf(expf(zl)));
+    const bool poly = __all_sync(0xffffffffu, s <= S_POLY);
+    const f32x2 hba2 = pack2(0.5f * f.b_a[d], 0.5f * f.b_a[d]), hbx2 = pack2(0.5f * f.b_x[d], 0.5f * f.b_x[d]), s2 = pack2(s, s);
+    const uint8_t *u_col = smem + SMEM_U + (uint32_t)(dl >> 6) * KBLOCK_BYTES + (uint32_t)(dl & 7) * 2u;
+    const uint32_t u_chunk = (uint32_t)(dl & 63) >> 3;
+    const uint8_t *r_col = smem + SMEM_R + (uint32_t)c_own * 2u;
+    float *h = f.h_T;                                 // in/out
+    __nv_bfloat16 *y = (__nv_bfloat16 *)f.y;
+    const int nq = NB >> 2;                           // multiple of 4
+    const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16);
+    // the recurrent state of this warp's sequences is fetched while the tensor core works
+    float hv[NB_MAX / 4];
 #pragma unroll
-        for (int j = 0; j < NB_MAX / 2; ++j) {
-            const int b = b0 + k * nh + j;
-            hv[j] = (j < nh && b < B) ? h[(size_t)b * D + d] : 0.0f;
+    for (int j = 0; j < NB_MAX / 4; ++j) {
+        const int b = b0 + kq * nq + j;
+        hv[j] = (j < nq && b < B) ? h[(size_t)b * D + d] : 0.0f;
+    }
+
+    // ---- gate products: the K blocks this CTA convolved itself are multiplied while the peer's half is still on its way
+    const uint32_t idesc = make_idesc(128, NB);
+    auto issue_kblocks = [&](int kb_first, bool first) {   // two K blocks = 8 K steps of 16, both gates
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t koff = (uint32_t)(kb_first + (j >> 2)) * KBLOCK_BYTES + (uint32_t)(j & 3) * 32u;
+            const uint64_t bd = make_desc_sw128(base + SMEM_U + koff);
+            const uint32_t accum = (first && j == 0) ? 0u : 1u;
+            mma_ss(tmem, make_desc_sw128(base + SMEM_WA + koff), bd, idesc, accum);
+            mma_ss(tmem + 128, make_desc_sw128(base + SMEM_WX + koff), bd, idesc, accum);
         }
-    // ---- gate products
+    };
+    bool w_ok = true;
     if (tid == 0) {
-        if (mbar_wait(BAR_W, 0, spin, &no_abort)) {
-            fence_async_all();
+        w_ok = mbar_wait(BAR_W, 0, spin, &no_abort);
+        if (w_ok) {
             tc_fence_after();
-            const uint32_t idesc = make_idesc(128, NB);
-#pragma unroll
-            for (int ks = 0; ks < DH / 16; ++ks) {
-                const uint32_t koff = (uint32_t)(ks >> 2) * KBLOCK_BYTES + (uint32_t)(ks & 3) * 32u;
-                const uint64_t bd = make_desc_sw128(base + SMEM_U + koff);
-                mma_ss(tmem, make_desc_sw128(base + SMEM_WA + koff), bd, idesc, ks > 0);
-                mma_ss(tmem + 128, make_desc_sw128(base + SMEM_WX + koff), bd, idesc, ks > 0);
-            }
-            tc_commit(BAR_ACC);
+            issue_kblocks((int)rank * 2, true);
         } else {
             atomicExch(f.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
         }
     }
     __syncwarp();
+    cluster_wait();      // both halves of the U tile are in place in both CTAs
+    if (tid == 0 && w_ok) {
+        fence_async_all();
+        issue_kblocks((int)(rank ^ 1u) * 2, false);
+        tc_commit(BAR_ACC);
+    }
+    __syncwarp();
 
-    {
-        if (!warp_wait(BAR_ACC, 0, spin, &no_abort)) {
-            timed_out = 1;
-        } else {
-            tc_fence_after();
+    if (!warp_wait(BAR_ACC, 0, spin, &no_abort)) {
+        timed_out = 1;
+    } else {
+        tc_fence_after();
 #pragma unroll
-            for (int j0 = 0; j0 < NB_MAX / 2; j0 += 8) {
-                if (j0 >= nh) break;
-                const int n0 = k * nh + j0;
-                float za[8], zx[8];
-                tmem_ld8(tm_lane + n0, za);
-                tmem_ld8(tm_lane + 128 + n0, zx);
-                tmem_ld_wait();
-                // two sequences per register pair, four pairs side by side
-                f32x2 A2[4], V2[4];
-                float u[8];
+        for (int j0 = 0; j0 < NB_MAX / 4; j0 += 4) {
+            if (j0 >= nq) break;
+            const int n0 = kq * nq + j0;
+            float za[4], zx[4];
+            tmem_ld4(tm_lane + n0, za);
+            tmem_ld4(tm_lane + 128 + n0, zx);
+            tmem_ld_wait();
+            // two sequences per register pair, two pairs side by side
+            f32x2 A2[2], V2[2];
+            float u[4];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int n = n0 + j;
-                    const uint32_t ub = *(const uint16_t *)(u_col + (uint32_t)n * 128u + ((u_chunk ^ (uint32_t)(n & 7)) << 4));
-                    const uint32_t rb = *(const uint16_t *)(r_col + (uint32_t)n * (CH * 2));
-                    u[j] = __uint_as_float(ub << 16) + __uint_as_float(rb << 16);
-                }
+            for (int j = 0; j < 4; ++j) {
+                const int n = n0 + j;
+                const uint32_t ub = *(const uint16_t *)(u_col + (uint32_t)n * 128u + ((u_chunk ^ (uint32_t)(n & 7)) << 4));
+                const uint32_t rb = *(const uint16_t *)(r_col + (uint32_t)n * (CH * 2));
+                u[j] = __uint_as_float(ub << 16) + __uint_as_float(rb << 16);
+            }
 #pragma unroll
-                for (int j = 0; j < 4; ++j) { A2[j] = pack2(za[2 * j], za[2 * j + 1]); V2[j] = pack2(zx[2 * j], zx[2 * j + 1]); }
-                if (poly) gate_group<true, 4>(A2, V2, u, hba2, hbx2, s2);
-                else gate_group<false, 4>(A2, V2, u, hba2, hbx2, s2);
+            for (int j = 0; j < 2; ++j) { A2[j] = pack2(za[2 * j], za[2 * j + 1]); V2[j] = pack2(zx[2 * j], zx[2 * j + 1]); }
+            if (poly) gate_group<true, 2>(A2, V2, u, hba2, hbx2, s2);
+            else gate_group<false, 2>(A2, V2, u, hba2, hbx2, s2);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const f32x2 H2 = fma2(A2[j], pack2(hv[j0 + 2 * j], hv[j0 + 2 * j + 1]), V2[j]);
-                    const float hn[2] = {lo2(H2), hi2(H2)};
+            for (int j = 0; j < 2; ++j) {
+                const f32x2 H2 = fma2(A2[j], pack2(hv[j0 + 2 * j], hv[j0 + 2 * j + 1]), V2[j]);
+                const float hn[2] = {lo2(H2), hi2(H2)};
 #pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int b = b0 + n0 + 2 * j + e;
-                        if (b < B) {
-                            h[(size_t)b * D + d] = hn[e];
-                            y[(size_t)b * D + d] = __float2bfloat16_rn(hn[e]);
-                        }
+                for (int e = 0; e < 2; ++e) {
+                    const int b = b0 + n0 + 2 * j + e;
+                    if (b < B) {
+                        h[(size_t)b * D + d] = hn[e];
+                        y[(size_t)b * D + d] = __float2bfloat16_rn(hn[e]);
                     }
                 }
             }
         }
-        if (__any_sync(0xffffffffu, timed_out) && lane == 0) atomicExch(f.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
     }
+    if (__any_sync(0xffffffffu, timed_out) && lane == 0) atomicExch(f.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
 
     tc_fence_before();
     __syncthreads();

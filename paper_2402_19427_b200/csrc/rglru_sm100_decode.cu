@@ -107,22 +107,34 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     }
     __syncwarp();
 
+    // ---- epilogue constants (parameters only, fetched early): warp (q, kq) owns channels 32 q .. 32 q + 31 and quarter kq
+    //      of the tile's sequences
+    const int q = warp & 3, kq = warp >> 2;
+    const int c_own = q * 32 + lane;
+    const int dl = (int)rank * CH + c_own;
+    const size_t d = (size_t)head * DH + dl;
+    const float lam = f.lambda[d];
+    const float zl = -lam;
+    const float s = f.c * (zl > 0.0f ? zl + log1pf(expf(-zl)) : log1pf(expf(zl)));
+    const bool poly = __all_sync(0xffffffffu, s <= S_POLY);
+    const f32x2 hba2 = pack2(0.5f * f.b_a[d], 0.5f * f.b_a[d]), hbx2 = pack2(0.5f * f.b_x[d], 0.5f * f.b_x[d]), s2 = pack2(s, s);
+
     // ---- conv phase: thread = (8-channel chunk c, sequences n = tid/16, tid/16 + 32, ...)
     {
         const int c = tid & 15;
-        const int dl = (int)rank * CH + c * 8;          // channel within the head
-        const size_t d = (size_t)head * DH + dl;        // global channel
+        const int cdl = (int)rank * CH + c * 8;         // channel within the head
+        const size_t cd = (size_t)head * DH + cdl;      // global channel
         const __nv_bfloat16 *cw = (const __nv_bfloat16 *)f.conv_w;
         uint4 w[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) w[j] = *(const uint4 *)(cw + (size_t)j * D + d);
+        for (int j = 0; j < 4; ++j) w[j] = *(const uint4 *)(cw + (size_t)j * D + cd);
         float cb[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) cb[e] = f.conv_b ? f.conv_b[d + e] : 0.0f;
+        for (int e = 0; e < 8; ++e) cb[e] = f.conv_b ? f.conv_b[cd + e] : 0.0f;
         const __nv_bfloat16 *x = (const __nv_bfloat16 *)f.x;
         __nv_bfloat16 *cs = (__nv_bfloat16 *)f.cs_out;   // in/out
-        const uint32_t u_kb = SMEM_U + (uint32_t)(dl >> 6) * KBLOCK_BYTES;
-        const uint32_t chunk = (uint32_t)(dl & 63) >> 3;
+        const uint32_t u_kb = SMEM_U + (uint32_t)(cdl >> 6) * KBLOCK_BYTES;
+        const uint32_t chunk = (uint32_t)(cdl & 63) >> 3;
         // everything above reads only parameters; x and the state may have been written by the kernel just before this
         // one on the stream, whose completion (and visibility of its stores) is awaited here
         asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -133,10 +145,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
         for (int i = 0; i < NIT; ++i) {
             const int n = (tid >> 4) + 32 * i, b = b0 + n;
             if (n < NB && b < B) {
-                xv[i] = *(const uint4 *)(x + (size_t)b * D + d);
-                r0[i] = *(const uint4 *)(cs + ((size_t)b * 3 + 0) * D + d);
-                r1[i] = *(const uint4 *)(cs + ((size_t)b * 3 + 1) * D + d);
-                r2[i] = *(const uint4 *)(cs + ((size_t)b * 3 + 2) * D + d);
+                xv[i] = *(const uint4 *)(x + (size_t)b * D + cd);
+                r0[i] = *(const uint4 *)(cs + ((size_t)b * 3 + 0) * D + cd);
+                r1[i] = *(const uint4 *)(cs + ((size_t)b * 3 + 1) * D + cd);
+                r2[i] = *(const uint4 *)(cs + ((size_t)b * 3 + 2) * D + cd);
             }
         }
         cluster_wait();
@@ -165,9 +177,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
                 uo = make_uint4(o[0], o[1], o[2], o[3]);
                 *(uint4 *)(smem + SMEM_R + (uint32_t)n * (CH * 2) + (uint32_t)c * 16u) = make_uint4(rem[0], rem[1], rem[2], rem[3]);
                 // the conv state moves up by one row: bit-exact copies
-                *(uint4 *)(cs + ((size_t)b * 3 + 0) * D + d) = r1[i];
-                *(uint4 *)(cs + ((size_t)b * 3 + 1) * D + d) = r2[i];
-                *(uint4 *)(cs + ((size_t)b * 3 + 2) * D + d) = xv[i];
+                *(uint4 *)(cs + ((size_t)b * 3 + 0) * D + cd) = r1[i];
+                *(uint4 *)(cs + ((size_t)b * 3 + 1) * D + cd) = r2[i];
+                *(uint4 *)(cs + ((size_t)b * 3 + 2) * D + cd) = xv[i];
             }
             const uint32_t off = u_kb + (uint32_t)n * 128u + ((chunk ^ (uint32_t)(n & 7)) << 4);
             *(uint4 *)(smem + off) = uo;
@@ -178,16 +190,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     __syncthreads();     // this CTA's half of the U tile is complete in its own shared memory
     cluster_arrive();    // ... and, once the peer has waited, in the peer's
 
-    // ---- epilogue set-up: warp (q, kq) owns channels 32 q .. 32 q + 31 and quarter kq of the tile's sequences
-    const int q = warp & 3, kq = warp >> 2;
-    const int c_own = q * 32 + lane;
-    const int dl = (int)rank * CH + c_own;
-    const size_t d = (size_t)head * DH + dl;
-    const float lam = f.lambda[d];
-    const float zl = -lam;
-    const float s = f.c * (zl > 0.0f ? zl + log1pf(expf(-zl)) : log1pf(expf(zl)));
-    const bool poly = __all_sync(0xffffffffu, s <= S_POLY);
-    const f32x2 hba2 = pack2(0.5f * f.b_a[d], 0.5f * f.b_a[d]), hbx2 = pack2(0.5f * f.b_x[d], 0.5f * f.b_x[d]), s2 = pack2(s, s);
     const uint8_t *u_col = smem + SMEM_U + (uint32_t)(dl >> 6) * KBLOCK_BYTES + (uint32_t)(dl & 7) * 2u;
     const uint32_t u_chunk = (uint32_t)(dl & 63) >> 3;
     const uint8_t *r_col = smem + SMEM_R + (uint32_t)c_own * 2u;

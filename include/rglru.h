@@ -177,6 +177,15 @@ int32_t rglru_prefill_static_scratch(const rglru_shape_t *shape, const rglru_par
                                      void *conv_state_out, void *status_word, void *cuda_stream);
 
 /*
+ * Time limit of every device-side wait (a CTA waiting for another CTA's carry record, for a copy or for the tensor
+ * core).  A wait that runs out makes the kernel record RGLRU_ERR_TIMEOUT in the workspace header, let work in flight
+ * land, release its resources and return; nothing hangs and the context stays usable.  The default is 2 s, far above
+ * any legitimate wait; ns = 0 restores it.  Process-wide; takes effect for calls issued afterwards.  Returns the
+ * previous value.
+ */
+uint64_t rglru_set_wait_limit_ns(uint64_t ns);
+
+/*
  * Synchronises `cuda_stream` and returns the device-side status recorded in `workspace` by the
  * calls issued so far (RGLRU_OK, RGLRU_ERR_TIMEOUT, or RGLRU_ERR_CUDA if the stream itself
  * reports an error), then clears it.

@@ -22,7 +22,7 @@ FLAG_NONE, FLAG_FORCE_GENERIC = 0, 1
 
 EXPORTED = ["rglru_abi_version", "rglru_status_string", "rglru_workspace_bytes", "rglru_prefill",
             "rglru_decode_step", "rglru_backward", "rglru_host_staging_bytes", "rglru_prefill_host",
-            "rglru_query_status", "rglru_prefill_static_scratch"]
+            "rglru_query_status", "rglru_prefill_static_scratch", "rglru_set_wait_limit_ns"]
 
 
 class Shape(ctypes.Structure):
@@ -72,6 +72,8 @@ def load() -> ctypes.CDLL:
         lib.rglru_prefill_host.restype = i32
         lib.rglru_prefill_static_scratch.argtypes = [sp, pp] + [vp] * 8
         lib.rglru_prefill_static_scratch.restype = i32
+        lib.rglru_set_wait_limit_ns.argtypes = [ctypes.c_uint64]
+        lib.rglru_set_wait_limit_ns.restype = ctypes.c_uint64
         lib.rglru_query_status.argtypes = [vp, vp]
         lib.rglru_query_status.restype = i32
         _lib = lib
@@ -256,6 +258,11 @@ def prefill_host(x_host, params: Params, y_host, h_T_host, conv_state_out_host, 
                                 _ptr(workspace), workspace.numel(), _stream())
     if rc != OK:
         raise RglruError(rc, "rglru_prefill_host")
+
+
+def set_wait_limit_ns(ns: int) -> int:
+    """Time limit of device-side waits (0 restores the 2 s default); returns the previous value."""
+    return int(load().rglru_set_wait_limit_ns(int(ns)))
 
 
 def query_status(workspace) -> int:

@@ -275,6 +275,12 @@ int32_t rglru_prefill_host(const rglru_shape_t *s, const rglru_params_t *p, cons
     return RGLRU_OK;
 }
 
+uint64_t rglru_set_wait_limit_ns(uint64_t ns) {
+    const uint64_t prev = g_spin_limit_ns;
+    g_spin_limit_ns = ns == 0 ? 2000000000ull : ns;
+    return prev;
+}
+
 int32_t rglru_query_status(void *workspace, void *cuda_stream) {
     if (!workspace) return RGLRU_ERR_NULL;
     cudaStream_t st = (cudaStream_t)cuda_stream;

@@ -278,6 +278,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
         }
     }
     if (__any_sync(0xffffffffu, timed_out) && lane == 0) atomicExch(f.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
+    if (timed_out) {   // let the weight copies and MMAs in flight land before shared and tensor memory are given back
+        const uint64_t tw = gtimer();
+        while (gtimer() - tw < 50000ull) __nanosleep(1000);
+    }
 
     tc_fence_before();
     __syncthreads();

@@ -117,3 +117,18 @@ def test_status_word_reads_ok_on_fresh_workspace():
     from paper_2402_19427_b200 import binding
     ws = torch.randint(0, 255, (4096,), dtype=torch.uint8, device="cuda")
     assert binding.query_status(ws) == binding.OK
+
+
+def test_recorded_timeout_is_reported_once_and_wait_limit_knob_round_trips():
+    """Host side of the failure path: a status word as a kernel leaves it after a wait ran out (magic | code) is reported
+    by rglru_query_status and cleared; the wait limit can be changed and restored.  No wait is made to run out here."""
+    import torch
+    from paper_2402_19427_b200 import binding
+    ws = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    ws[:4] = torch.tensor([binding.ERR_TIMEOUT, 0x4C, 0x47, 0x52], dtype=torch.uint8)   # 0x52474C00 | 7, little endian
+    assert binding.query_status(ws) == binding.ERR_TIMEOUT
+    assert binding.query_status(ws) == binding.OK
+    prev = binding.set_wait_limit_ns(123456789)
+    assert prev == 2_000_000_000
+    assert binding.set_wait_limit_ns(0) == 123456789
+    assert binding.set_wait_limit_ns(0) == 2_000_000_000

@@ -165,6 +165,11 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    if rank == 0 or world == 1:
+        from paper_2402_19427_b200 import build
+        build.build()  # no-op when the library is up to date
+    if world > 1:
+        dist.barrier()
     binding.load()  # fails loudly if the CUDA library is missing
 
     cfg = dict(synth.CONFIGS[WORKLOAD])

@@ -12,6 +12,13 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
 
 
+@pytest.fixture(scope="session", autouse=True)
+def built_library():
+    """Compile the CUDA library once per session if it is missing or stale (nvcc cross-compiles without a GPU)."""
+    from paper_2402_19427_b200 import build
+    return build.build()
+
+
 @pytest.fixture(scope="session")
 def oracle():
     import oracle as _oracle

@@ -254,10 +254,8 @@ __global__ void __launch_bounds__(256) conv_forward_kernel(EwArgs a) {
         return a.cs_in ? bf2f(a.cs_in[((size_t)b * 3 + (3 + t)) * D + d]) : 0.0f;
     };
     float x3 = xat(t0 - 3), x2 = xat(t0 - 2), x1 = xat(t0 - 1);
-    for (int t = t0; t < t1; t += 8) {
-        float xs[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) xs[k] = bf2f(a.x[((size_t)b * T + t + k) * D + d]);
+    // eight tokens: u token-major (coalesced across the block) and eight fp16 values of this channel's row
+    auto batch8 = [&](int t, const float (&xs)[8]) -> uint4 {
         uint32_t packed[4];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
@@ -268,7 +266,22 @@ __global__ void __launch_bounds__(256) conv_forward_kernel(EwArgs a) {
             if (k & 1) packed[k >> 1] |= bits << 16; else packed[k >> 1] = bits;
             x3 = x2; x2 = x1; x1 = xs[k];
         }
-        *(uint4 *)(a.uT + (size_t)d * a.BTp + (size_t)b * T + t) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        return make_uint4(packed[0], packed[1], packed[2], packed[3]);
+    };
+    int t = t0;
+    for (; t + 16 <= t1; t += 16) {   // sixteen tokens: the channel-major store fills whole 32-byte sectors
+        float xa[8], xb[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { xa[k] = bf2f(a.x[((size_t)b * T + t + k) * D + d]); xb[k] = bf2f(a.x[((size_t)b * T + t + 8 + k) * D + d]); }
+        const uint4 lo = batch8(t, xa), hi = batch8(t + 8, xb);
+        uint4 *dst = (uint4 *)(a.uT + (size_t)d * a.BTp + (size_t)b * T + t);
+        dst[0] = lo; dst[1] = hi;
+    }
+    if (t < t1) {
+        float xa[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) xa[k] = bf2f(a.x[((size_t)b * T + t + k) * D + d]);
+        *(uint4 *)(a.uT + (size_t)d * a.BTp + (size_t)b * T + t) = batch8(t, xa);
     }
 }
 

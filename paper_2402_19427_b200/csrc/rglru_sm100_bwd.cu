@@ -346,7 +346,8 @@ __global__ void __launch_bounds__(256) scan_apply_kernel(EwArgs a) {
     float *p_du = a.du + tokb * sD + d;
     __half *p_ta = a.dzT + ((size_t)h * 2 * DH + n) * a.BTp + tokb, *p_tx = p_ta + (size_t)DH * a.BTp;
     const float h0v = a.h0 ? a.h0[(size_t)b * D + d] : 0.0f;
-    for (int tb = t1 - 8; tb >= t0; tb -= 8) {
+    // eight tokens at the running pointers, newest first; the channel-major copies of dz come back packed
+    auto batch8 = [&](int tb, uint32_t (&pa)[4], uint32_t (&px)[4]) {
         float dyv[8], hpv[8], zav[8], zxv[8], uv[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
@@ -356,7 +357,6 @@ __global__ void __launch_bounds__(256) scan_apply_kernel(EwArgs a) {
             zxv[k] = __half2float(p_z[k * sZ + DH]);
             uv[k] = __half2float(p_u[k * sD]);
         }
-        uint32_t pa[4], px[4];
 #pragma unroll
         for (int k = 7; k >= 0; --k) {
             const float r = sigmoid_fast(zav[k] + ba), gi = sigmoid_fast(zxv[k] + bx);
@@ -377,9 +377,25 @@ __global__ void __launch_bounds__(256) scan_apply_kernel(EwArgs a) {
             const uint32_t ba16 = (uint32_t)__half_as_ushort(ha), bx16 = (uint32_t)__half_as_ushort(hx);
             if (k & 1) { pa[k >> 1] = ba16 << 16; px[k >> 1] = bx16 << 16; } else { pa[k >> 1] |= ba16; px[k >> 1] |= bx16; }
         }
+        p_dy -= 8 * sD; p_y -= 8 * sD; p_z -= 8 * sZ; p_u -= 8 * sD; p_dz -= 8 * sZ; p_du -= 8 * sD;
+    };
+    int tb = t1 - 8;
+    // sixteen tokens per round, so that each channel-major row gets 32 adjacent bytes (a whole sector) at once
+    for (; tb - 8 >= t0; tb -= 16) {
+        uint32_t pa1[4], px1[4], pa0[4], px0[4];
+        batch8(tb, pa1, px1);
+        batch8(tb - 8, pa0, px0);
+        *(uint4 *)(p_ta - 8) = make_uint4(pa0[0], pa0[1], pa0[2], pa0[3]);
+        *(uint4 *)p_ta = make_uint4(pa1[0], pa1[1], pa1[2], pa1[3]);
+        *(uint4 *)(p_tx - 8) = make_uint4(px0[0], px0[1], px0[2], px0[3]);
+        *(uint4 *)p_tx = make_uint4(px1[0], px1[1], px1[2], px1[3]);
+        p_ta -= 16; p_tx -= 16;
+    }
+    if (tb >= t0) {
+        uint32_t pa[4], px[4];
+        batch8(tb, pa, px);
         *(uint4 *)p_ta = make_uint4(pa[0], pa[1], pa[2], pa[3]);
         *(uint4 *)p_tx = make_uint4(px[0], px[1], px[2], px[3]);
-        p_dy -= 8 * sD; p_y -= 8 * sD; p_z -= 8 * sZ; p_u -= 8 * sD; p_dz -= 8 * sZ; p_du -= 8 * sD; p_ta -= 8; p_tx -= 8;
     }
     float *pv = a.part_vec + ((size_t)b * a.nchunk + c) * 3 * D + d;
     pv[0] = s_lam; pv[(size_t)D] = s_ba; pv[(size_t)2 * D] = s_bx;

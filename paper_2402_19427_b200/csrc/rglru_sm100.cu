@@ -49,12 +49,11 @@ constexpr uint32_t X_ROW_BYTES = DH * 2;                   // 512
 constexpr uint32_t X_SLAB_BYTES = SLAB_ROWS * X_ROW_BYTES; // 17920
 constexpr uint32_t SMEM_U = 0;
 constexpr uint32_t SMEM_X = SMEM_U + US * U_STAGE_BYTES;
-constexpr uint32_t Y_ROW_BYTES = CH * 2;                   // 256: one token row of this CTA's channels
-constexpr uint32_t Y_HALF_BYTES = EPI_TOK * Y_ROW_BYTES;   // 16384: the 64 tokens of one epilogue half
-constexpr uint32_t SMEM_Y = SMEM_X + XS * X_SLAB_BYTES;    // bf16 y_s[2][64][128], staged for bulk stores
-constexpr uint32_t SMEM_AGG = SMEM_Y + 2 * Y_HALF_BYTES;   // float2 agg_s[2 tile parity][2 halves][4][32]
+constexpr uint32_t Y_WARP_BYTES = EPI_TOK * 32 * 2;        // 4096: one epilogue warp's 64 tokens x 32 channels
+constexpr uint32_t SMEM_Y = SMEM_X + XS * X_SLAB_BYTES;    // bf16 y_s[8 warps][64][32], staged for tiled stores
+constexpr uint32_t SMEM_AGG = SMEM_Y + 8 * Y_WARP_BYTES;   // float2 agg_s[2 tile parity][2 halves][4][32]
 constexpr uint32_t SMEM_BAR = SMEM_AGG + 2 * 2 * 4 * 32 * 8;
-constexpr int NUM_BARS = 2 * XS + 2 * US + 4 + 8 + 4;
+constexpr int NUM_BARS = 2 * XS + 2 * US + 4 + 8;
 constexpr uint32_t SMEM_MISC = SMEM_BAR + NUM_BARS * 8;    // tmem base, abort flag
 constexpr uint32_t SMEM_TOTAL = SMEM_MISC + 16;
 constexpr uint32_t SMEM_ALLOC = SMEM_TOTAL + 1024;         // slack for 1024-byte alignment
@@ -64,7 +63,7 @@ constexpr uint32_t TM_ACC_A = 0, TM_ACC_X = 128, TM_W_A = 256, TM_W_X = 384;
 
 
 struct Sm100Args {
-    // x as [B][T][D] with a box of SLAB_ROWS token rows x one head; y with a box of EPI_TOK rows x CH channels
+    // x as [B][T][D] with a box of SLAB_ROWS token rows x one head; y with a box of EPI_TOK rows x 32 channels
     alignas(64) CUtensorMap tm_x;
     alignas(64) CUtensorMap tm_y;
     FwdArgs f;
@@ -97,8 +96,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
     auto BAR_ACCFULL = [&](int k) { return bar0 + 8u * (2 * XS + 2 * US + k); };       // accumulators of token half k
     auto BAR_ACCEMPTY = [&](int k) { return bar0 + 8u * (2 * XS + 2 * US + 2 + k); };
     auto BAR_AGG = [&](int q, int k) { return bar0 + 8u * (2 * XS + 2 * US + 4 + q * 2 + k); };  // fold of half k, channel group q
-    auto BAR_YFREE = [&](int k) { return bar0 + 8u * (2 * XS + 2 * US + 12 + k); };
-    auto BAR_YFULL = [&](int k) { return bar0 + 8u * (2 * XS + 2 * US + 14 + k); };
     uint32_t *tmem_base_s = (uint32_t *)(smem + SMEM_MISC);
     volatile int *abort_flag = (volatile int *)(smem + SMEM_MISC + 4);
     float2 *agg_s = (float2 *)(smem + SMEM_AGG);
@@ -116,25 +113,28 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
     const int B_whole = (f.B / S) * S, shared_tiles = (f.B - B_whole) * p.tps;
     const int n_shared = kcta < shared_tiles ? (shared_tiles - kcta + S - 1) / S : 0;
     const int n_my_tiles = n_shared + (B_whole / S) * p.tps;
-    // tile number `it` of this CTA -> sequence b, tile ti within it; true when it is a shared tile
-    auto tile_of = [&](int it, int &b, int &ti) -> bool {
-        if (it < n_shared) {
-            const int g = kcta + it * S;
-            b = B_whole + g / p.tps; ti = g % p.tps;
-            return true;
+    // The CTA's tiles in order: tile_first gives (sequence b, tile ti within it) of tile 0, tile_next steps from tile
+    // `it` to tile `it + 1`; tile `it` is a shared one when it < n_shared.
+    auto tile_first = [&](int &b, int &ti) {
+        if (n_shared > 0) { b = B_whole + kcta / p.tps; ti = kcta % p.tps; } else { b = kcta; ti = 0; }
+    };
+    auto tile_next = [&](int it, int &b, int &ti) {
+        if (it + 1 < n_shared) {
+            ti += S;
+            while (ti >= p.tps) { ti -= p.tps; ++b; }
+        } else if (it + 1 == n_shared) {
+            b = kcta; ti = 0;
+        } else if (++ti == p.tps) {
+            ti = 0; b += S;
         }
-        const int j = it - n_shared;
-        b = kcta + (j / p.tps) * S; ti = j % p.tps;
-        return false;
     };
     const unsigned long long spin = p.spin_ns;
 
     if (tid == 0) {
         for (int s = 0; s < XS; ++s) { mbar_init(BAR_XFULL(s), 1); mbar_init(BAR_XEMPTY(s), 4); }
         for (int s = 0; s < US; ++s) { mbar_init(BAR_UFULL(s), 4); mbar_init(BAR_UEMPTY(s), 9); }
-        for (int k = 0; k < 2; ++k) { mbar_init(BAR_ACCFULL(k), 1); mbar_init(BAR_ACCEMPTY(k), 4); }
+        mbar_init(BAR_ACCFULL(0), 1); mbar_init(BAR_ACCEMPTY(0), 8);
         for (int q = 0; q < 4; ++q) { mbar_init(BAR_AGG(q, 0), 1); mbar_init(BAR_AGG(q, 1), 1); }
-        for (int k = 0; k < 2; ++k) { mbar_init(BAR_YFREE(k), 4); mbar_init(BAR_YFULL(k), 4); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -197,9 +197,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         // the two lanes of packed fp32x2 arithmetic.
         int slab_n = 0;
         bool ok = true;
-        for (int it = 0; it < n_my_tiles && ok; ++it) {
-            int b, ti;
-            tile_of(it, b, ti);
+        int b, ti;
+        tile_first(b, ti);
+        for (int it = 0; it < n_my_tiles && ok; tile_next(it, b, ti), ++it) {
             const int t0 = ti * TILE_N;
             const int st = it % US;
             ok = warp_wait(BAR_UEMPTY(st), ((it / US) & 1) ^ 1, spin, abort_flag);
@@ -285,9 +285,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         const __nv_bfloat16 *cs_in = (const __nv_bfloat16 *)f.cs_in;
         int slab_n = 0;
         bool ok = true;
-        for (int it = 0; it < n_my_tiles && ok; ++it) {
-            int b, ti;
-            tile_of(it, b, ti);
+        int b, ti;
+        tile_first(b, ti);
+        for (int it = 0; it < n_my_tiles && ok; tile_next(it, b, ti), ++it) {
             const int t0 = ti * TILE_N;
             const int nslab = min(TILE_N / SLAB, (T - t0 + SLAB - 1) / SLAB);
             for (int s = 0; s < nslab; ++s, ++slab_n) {
@@ -320,9 +320,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         if (!ok && lane == 0) record_timeout(f.status, abort_flag);
       } else if (warp == 5) {
         // ================================================================ MMA issuer
-        // The 128-token tile is issued as two 64-token halves with separate accumulators, so the MMAs of
-        // one half overlap the epilogue of the other and of the previous tile.
-        constexpr uint32_t idesc = make_idesc_f16(128, EPI_TOK);
+        // One N = 128 instruction per gate and K step: an N = 64 instruction takes about 45 cycles where 32 would be
+        // its share, an N = 128 one the full-rate 64, so halves would cost more tensor time than they overlap.
+        constexpr uint32_t idesc = make_idesc_f16(128, TILE_N);
         bool ok = true;
         if (lane == 0) {
             for (int it = 0; it < n_my_tiles && ok; ++it) {
@@ -330,22 +330,19 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
                 ok = mbar_wait(BAR_UFULL(st), (it / US) & 1, spin, abort_flag);
                 if (!ok) break;
                 const uint32_t u_base = base + SMEM_U + st * U_STAGE_BYTES;
-                for (int kh = 0; kh < 2; ++kh) {
-                    ok = mbar_wait(BAR_ACCEMPTY(kh), (it & 1) ^ 1, spin, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    // rows kh*64 .. kh*64+63 of every K block; the start-address field of the descriptor counts 16-byte units
-                    const uint64_t bd0 = make_desc_sw128(u_base + (uint32_t)kh * EPI_TOK * 128u);
-                    const uint32_t acc = tmem + kh * EPI_TOK;
+                ok = mbar_wait(BAR_ACCEMPTY(0), (it & 1) ^ 1, spin, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                // the start-address field of the descriptor counts 16-byte units
+                const uint64_t bd0 = make_desc_sw128(u_base);
 #pragma unroll
-                    for (int ks = 0; ks < DH / 16; ++ks) {
-                        const uint64_t bd = bd0 + (uint64_t)(((ks >> 2) * U_KBLOCK_BYTES + (ks & 3) * 32) >> 4);
-                        mma_ts(acc + TM_ACC_A, tmem + TM_W_A + ks * 8, bd, idesc, ks > 0);
-                        mma_ts(acc + TM_ACC_X, tmem + TM_W_X + ks * 8, bd, idesc, ks > 0);
-                    }
-                    if (kh == 1) tc_commit(BAR_UEMPTY(st));
-                    tc_commit(BAR_ACCFULL(kh));
+                for (int ks = 0; ks < DH / 16; ++ks) {
+                    const uint64_t bd = bd0 + (uint64_t)(((ks >> 2) * U_KBLOCK_BYTES + (ks & 3) * 32) >> 4);
+                    mma_ts(tmem + TM_ACC_A, tmem + TM_W_A + ks * 8, bd, idesc, ks > 0);
+                    mma_ts(tmem + TM_ACC_X, tmem + TM_W_X + ks * 8, bd, idesc, ks > 0);
                 }
+                tc_commit(BAR_UEMPTY(st));
+                tc_commit(BAR_ACCFULL(0));
             }
             if (!ok) record_timeout(f.status, abort_flag);
         }
@@ -372,19 +369,31 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             u_off[j] = (uint32_t)(hc >> 6) * U_KBLOCK_BYTES + ((((uint32_t)(hc & 63) >> 3) ^ (uint32_t)j) << 4) + (uint32_t)(hc & 7) * 2 +
                        (uint32_t)(k * EPI_TOK) * 128u;
         const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16);
-        uint16_t *y_s = (uint16_t *)(smem + SMEM_Y + (uint32_t)k * Y_HALF_BYTES + (uint32_t)c_own * 2u);  // this thread's column of the y staging tile
+        const uint32_t y_warp_off = SMEM_Y + (uint32_t)(k * 4 + q) * Y_WARP_BYTES;
+        uint16_t *y_s = (uint16_t *)(smem + y_warp_off) + lane;   // this thread's column of the warp's y block [64 tokens][32 channels]
+        const uint32_t y_s_addr = base + y_warp_off;
         const __nv_bfloat16 *x = (const __nv_bfloat16 *)f.x;
         const __nv_bfloat16 *cs_in = (const __nv_bfloat16 *)f.cs_in;
         float h_prev_own = 0.0f;  // state at the end of this CTA's previous tile
+        float h_scan_end = 0.0f;  // state at the end of this warp's 64 tokens of the previous tile
         bool ok = true;
-        for (int it = 0; it < n_my_tiles && ok; ++it) {
-            int b, ti;
-            const bool shared = tile_of(it, b, ti);
+        int b, ti;
+        tile_first(b, ti);
+        for (int it = 0; it < n_my_tiles && ok; tile_next(it, b, ti), ++it) {
+            const bool shared = it < n_shared;
             const int g = b * p.tps + ti;   // tile number within the half-head: index of its carry record
             const int t0 = ti * TILE_N;
             const int st = it % US;
             const int nv = max(0, min(EPI_TOK, T - t0 - k * EPI_TOK));  // valid tokens of this warp
-            ok = warp_wait(BAR_ACCFULL(k), it & 1, spin, abort_flag);
+            if (k == 0 && it > 0) {
+                // The first half left the previous tile without the second half's fold; it takes it now, before its own
+                // next arrival on BAR_AGG (so that neither side is ever more than one barrier phase ahead of the other).
+                ok = warp_wait(BAR_AGG(q, 1), (it - 1) & 1, spin, abort_flag);
+                if (!ok) break;
+                const float2 other = agg_s[((((it - 1) & 1) * 2 + 1) * 4 + q) * 32 + lane];
+                h_prev_own = fmaf(other.x, h_scan_end, other.y);
+            }
+            ok = warp_wait(BAR_ACCFULL(0), it & 1, spin, abort_flag);
             if (!ok) break;
             tc_fence_after();
             // A2[j] / V2[j]: tokens j (low half) and j + 32 (high half) of this warp's 64 tokens
@@ -396,7 +405,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(BAR_ACCEMPTY(k));  // the accumulators now live in registers
+            if (lane == 0) mbar_arrive(BAR_ACCEMPTY(0));  // the accumulators now live in registers
             // gates, decay, input scale: (z_a, z_x) -> (a_t, v_t) in place
             const uint8_t *u_tile = smem + SMEM_U + st * U_STAGE_BYTES;
             auto gates = [&](auto poly_tag) {
@@ -428,16 +437,20 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             for (int j = 0; j < EPI_TOK / 2; ++j) { P2 = mul2(P2, A2[j]); HL2 = fma2(A2[j], HL2, V2[j]); }
             const float P_lo = lo2(P2), hl_lo = lo2(HL2);
             const float P = P_lo * hi2(P2), hl = fmaf(hi2(P2), hl_lo, hi2(HL2));
-            // ---- the two halves of the tile exchange their folds; the second half publishes the tile's
+            // ---- the second half of the tile needs the fold of the first; the first half goes on without waiting
+            //      and picks up the second half's fold at the start of the next tile
+            //      (the second half arrives only after its own wait: then neither barrier can run two phases ahead)
             agg_s[(((it & 1) * 2 + k) * 4 + q) * 32 + lane] = make_float2(P, hl);
+            float P_0 = P, hl_0 = hl, P_t = 0.0f, hl_t = 0.0f;    // tokens [0, 64); whole tile (second half only)
+            if (k == 1) {
+                ok = warp_wait(BAR_AGG(q, 0), it & 1, spin, abort_flag);
+                if (!ok) break;
+                const float2 other = agg_s[(((it & 1) * 2 + 0) * 4 + q) * 32 + lane];
+                P_0 = other.x; hl_0 = other.y;
+                P_t = P_0 * P; hl_t = fmaf(P, hl_0, hl);
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(BAR_AGG(q, k));
-            ok = warp_wait(BAR_AGG(q, k ^ 1), it & 1, spin, abort_flag);
-            if (!ok) break;
-            const float2 other = agg_s[(((it & 1) * 2 + (k ^ 1)) * 4 + q) * 32 + lane];
-            const float P_0 = k ? other.x : P, hl_0 = k ? other.y : hl;     // tokens [0, 64)
-            const float P_1 = k ? P : other.x, hl_1 = k ? hl : other.y;     // tokens [64, 128)
-            const float P_t = P_0 * P_1, hl_t = fmaf(P_1, hl_0, hl_1);      // whole tile
             if (shared && S > 1 && k == 1) {
                 uint4 rec;
                 rec.x = __float_as_uint(P_t); rec.y = p.tag; rec.z = __float_as_uint(hl_t); rec.w = p.tag;
@@ -492,16 +505,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
                 for (int j = MAX_S - 1; j >= 1; --j)
                     if (j <= nback) h = fmaf(__uint_as_float(rec[j - 1].x), h, __uint_as_float(rec[j - 1].z));
             }
-            h_prev_own = fmaf(P_t, h, hl_t);          // state at the end of this tile
+            if (k == 1) h_prev_own = fmaf(P_t, h, hl_t);   // state at the end of this tile (the first half works it out later)
             if (k == 1) h = fmaf(P_0, h, hl_0);       // state at the start of the second half
-            // ---- the y staging rows of this half must have been read out by the previous tile's bulk stores
-            if (it > 0) {
-                if (q == 0 && lane == 0) bulk_wait_read0();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(BAR_YFREE(k));
-                ok = warp_wait(BAR_YFREE(k), (it - 1) & 1, spin, abort_flag);
-                if (!ok) break;
-            }
+            // ---- the warp's y block must have been read out by its previous tiled store
+            if (lane == 0) bulk_wait_read0();
+            __syncwarp();
             // ---- the recurrence h_t = a_t h_{t-1} + v_t (Eq. 4), both halves in lock step; y_t = h_t
             f32x2 H2 = pack2(h, fmaf(P_lo, h, hl_lo));
 #pragma unroll
@@ -509,13 +517,18 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
                 H2 = fma2(A2[j], H2, V2[j]);
                 const __nv_bfloat162 o = __floats2bfloat162_rn(lo2(H2), hi2(H2));
                 const uint32_t ow = *(const uint32_t *)&o;
-                y_s[j * (Y_ROW_BYTES / 2)] = (uint16_t)(ow & 0xFFFFu);
-                y_s[(j + 32) * (Y_ROW_BYTES / 2)] = (uint16_t)(ow >> 16);
+                y_s[j * 32] = (uint16_t)(ow & 0xFFFFu);             // row j of the warp's block: 32 channels x 2 bytes
+                y_s[(j + 32) * 32] = (uint16_t)(ow >> 16);
             }
             h = hi2(H2);
+            h_scan_end = h;
             fence_async_smem();   // y rows become visible to the bulk-copy engine
             __syncwarp();
-            if (lane == 0) mbar_arrive(BAR_YFULL(k));
+            if (lane == 0) {
+                // the warp's 64 tokens x 32 channels go out as one tiled store; rows at or beyond T are clipped
+                if (nv > 0) tma_store_3d(&p.tm_y, head * DH + half * CH + q * 32, t0 + k * EPI_TOK, b, y_s_addr);
+                bulk_commit();
+            }
             if (k == 1 && ti == p.tps - 1) {
                 // end of a sequence: h_T (unrounded state) and the last three raw inputs, bit-exact
                 f.h_T[(size_t)b * D + d] = h;
@@ -530,16 +543,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
 #pragma unroll
                 for (int kk = 0; kk < 3; ++kk) cs_out[((size_t)b * 3 + kk) * D + d] = keep[kk];
             }
-            // ---- y: once the four warps of this half have written their columns, one thread sends the
-            //      64 x 128 tile to HBM with a single tiled TMA store
-            ok = warp_wait(BAR_YFULL(k), it & 1, spin, abort_flag);
-            if (!ok) break;
-            if (q == 0 && lane == 0) {
-                if (nv > 0) tma_store_3d(&p.tm_y, head * DH + half * CH, t0 + k * EPI_TOK, b, base + SMEM_Y + (uint32_t)k * Y_HALF_BYTES);
-                bulk_commit();
-            }
         }
-        if (q == 0 && lane == 0) bulk_wait0();
+        if (lane == 0) bulk_wait0();
         ok = __all_sync(0xffffffffu, ok);
         if (!ok && lane == 0) record_timeout(f.status, abort_flag);
     }
@@ -653,7 +658,7 @@ cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes,
         attr_set = true;
     }
     Sm100Args p;
-    if (!make_activation_map(&p.tm_x, a.x, a.B, a.T, a.D, DH, SLAB_ROWS) || !make_activation_map(&p.tm_y, a.y, a.B, a.T, a.D, CH, EPI_TOK))
+    if (!make_activation_map(&p.tm_x, a.x, a.B, a.T, a.D, DH, SLAB_ROWS) || !make_activation_map(&p.tm_y, a.y, a.B, a.T, a.D, 32, EPI_TOK))
         return cudaErrorNotSupported;
     p.f = a;
     p.tps = (a.T + TILE_N - 1) / TILE_N;

@@ -53,7 +53,7 @@ constexpr uint32_t Y_WARP_BYTES = EPI_TOK * 32 * 2;        // 4096: one epilogue
 constexpr uint32_t SMEM_Y = SMEM_X + XS * X_SLAB_BYTES;    // bf16 y_s[8 warps][64][32], staged for tiled stores
 constexpr uint32_t SMEM_AGG = SMEM_Y + 8 * Y_WARP_BYTES;   // float2 agg_s[2 tile parity][2 halves][4][32]
 constexpr uint32_t SMEM_BAR = SMEM_AGG + 2 * 2 * 4 * 32 * 8;
-constexpr int NUM_BARS = 2 * XS + 2 * US + 4 + 8;
+constexpr int NUM_BARS = 2 * XS + 2 * US + 4 + 8 + 1;
 constexpr uint32_t SMEM_MISC = SMEM_BAR + NUM_BARS * 8;    // tmem base, abort flag
 constexpr uint32_t SMEM_TOTAL = SMEM_MISC + 16;
 constexpr uint32_t SMEM_ALLOC = SMEM_TOTAL + 1024;         // slack for 1024-byte alignment
@@ -96,6 +96,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
     auto BAR_ACCFULL = [&](int k) { return bar0 + 8u * (2 * XS + 2 * US + k); };       // accumulators of token half k
     auto BAR_ACCEMPTY = [&](int k) { return bar0 + 8u * (2 * XS + 2 * US + 2 + k); };
     auto BAR_AGG = [&](int q, int k) { return bar0 + 8u * (2 * XS + 2 * US + 4 + q * 2 + k); };  // fold of half k, channel group q
+    const uint32_t BAR_WREADY = bar0 + 8u * (2 * XS + 2 * US + 12);   // gate weights are in tensor memory
     uint32_t *tmem_base_s = (uint32_t *)(smem + SMEM_MISC);
     volatile int *abort_flag = (volatile int *)(smem + SMEM_MISC + 4);
     float2 *agg_s = (float2 *)(smem + SMEM_AGG);
@@ -132,9 +133,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
 
     if (tid == 0) {
         for (int s = 0; s < XS; ++s) { mbar_init(BAR_XFULL(s), 1); mbar_init(BAR_XEMPTY(s), 4); }
-        for (int s = 0; s < US; ++s) { mbar_init(BAR_UFULL(s), 4); mbar_init(BAR_UEMPTY(s), 9); }
-        mbar_init(BAR_ACCFULL(0), 1); mbar_init(BAR_ACCEMPTY(0), 8);
+        for (int s = 0; s < US; ++s) { mbar_init(BAR_UFULL(s), 4); mbar_init(BAR_UEMPTY(s), 10); }
+        mbar_init(BAR_ACCFULL(0), 2); mbar_init(BAR_ACCEMPTY(0), 8);
         for (int q = 0; q < 4; ++q) { mbar_init(BAR_AGG(q, 0), 1); mbar_init(BAR_AGG(q, 1), 1); }
+        mbar_init(BAR_WREADY, 8);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -164,10 +166,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             tmem_st8(taddr + c * 8, lo, hi);
         }
         tmem_st_wait();
+        // only the MMA issuers wait for the weights: loads and the conv of the first tiles run meanwhile
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR_WREADY);
     }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
 
     // Register budget per warpgroup (the four warps of a group execute the same setmaxnreg):
     // conv producers 72, loader / MMA issuer / idle 40, epilogue 200.
@@ -318,13 +321,17 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             }
         }
         if (!ok && lane == 0) record_timeout(f.status, abort_flag);
-      } else if (warp == 5) {
-        // ================================================================ MMA issuer
+      } else if (warp == 5 || warp == 6) {
+        // ================================================================ MMA issuers: warp 5 the W_a products, warp 6 the W_x products
+        // (one thread's issue stream runs at 70-85 cycles per instruction beside the busy warps of its scheduler;
+        // two streams on two schedulers keep the tensor pipe fed)
+        const uint32_t tm_w = warp == 5 ? TM_W_A : TM_W_X, tm_acc = warp == 5 ? TM_ACC_A : TM_ACC_X;
         // One N = 128 instruction per gate and K step: an N = 64 instruction takes about 45 cycles where 32 would be
         // its share, an N = 128 one the full-rate 64, so halves would cost more tensor time than they overlap.
         constexpr uint32_t idesc = make_idesc_f16(128, TILE_N);
         bool ok = true;
         if (lane == 0) {
+            ok = mbar_wait(BAR_WREADY, 0, spin, abort_flag);
             for (int it = 0; it < n_my_tiles && ok; ++it) {
                 const int st = it % US;
                 ok = mbar_wait(BAR_UFULL(st), (it / US) & 1, spin, abort_flag);
@@ -338,8 +345,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
 #pragma unroll
                 for (int ks = 0; ks < DH / 16; ++ks) {
                     const uint64_t bd = bd0 + (uint64_t)(((ks >> 2) * U_KBLOCK_BYTES + (ks & 3) * 32) >> 4);
-                    mma_ts(tmem + TM_ACC_A, tmem + TM_W_A + ks * 8, bd, idesc, ks > 0);
-                    mma_ts(tmem + TM_ACC_X, tmem + TM_W_X + ks * 8, bd, idesc, ks > 0);
+                    mma_ts(tmem + tm_acc, tmem + tm_w + ks * 8, bd, idesc, ks > 0);
                 }
                 tc_commit(BAR_UEMPTY(st));
                 tc_commit(BAR_ACCFULL(0));

@@ -32,7 +32,7 @@ N_ROTATE = 4                 # distinct input/output buffer sets cycled between 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes per prefill launch on the bench workload from the committed ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
-NCU_TRAFFIC_BYTES = 128464896   # 86.98 MB read + 41.48 MB written (profiles/sm100_prefill_kernel_cfg1.md)
+NCU_TRAFFIC_BYTES = 132525056   # 86.90 MB read + 45.63 MB written (profiles/sm100_prefill_kernel_cfg1.md)
 
 
 def load_peaks():

@@ -197,7 +197,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
 __device__ __forceinline__ float bf2f(__nv_bfloat16 v) { return __bfloat162float(v); }
 __device__ __forceinline__ float sigmoid_acc(float z) { return 1.0f / (1.0f + expf(-z)); }
 // Hardware-approximate versions for the per-element work (relative error ~1e-6, far inside the gradient tolerance)
-__device__ __forceinline__ float sigmoid_fast(float z) { return __frcp_rn(1.0f + __expf(-z)); }
+__device__ __forceinline__ float rcp_fast(float x) { float y; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float rsqrt_fast(float x) { float y; asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float sigmoid_fast(float z) { return rcp_fast(1.0f + __expf(-z)); }
 // 1 - exp(x) for x <= 0 without cancellation near 0
 __device__ __forceinline__ float one_minus_exp(float x) {
     if (x > -0.25f) {   // -x (1 + x/2 + x^2/6 + x^3/24 + x^4/120 + x^5/720): relative truncation error < 2e-7
@@ -328,7 +330,7 @@ __global__ void __launch_bounds__(256) scan_carry_kernel(EwArgs a) {
 // pass 3: the scan with its carry and every element-wise adjoint (derived from Eq. 1-4):
 //   g_t = dy_t + a_{t+1} g_{t+1};  dL = g a (h_{t-1} - a v / m);  dv = g m;  di = dv u;  du = dv i;
 //   dr = -s dL;  dz_a = dr r (1-r);  dz_x = di i (1-i);  dLambda += dL c r sigmoid(-Lambda).   grid (D/256, nchunk, B)
-__global__ void __launch_bounds__(256) scan_apply_kernel(EwArgs a) {
+__global__ void __launch_bounds__(256, 3) scan_apply_kernel(EwArgs a) {
     const int d = blockIdx.x * 256 + threadIdx.x, c = blockIdx.y, b = blockIdx.z;
     const int T = a.T, D = a.D, h = d / DH, n = d % DH;
     const int t0 = c * CHUNK, t1 = min(T, t0 + CHUNK);
@@ -339,11 +341,11 @@ __global__ void __launch_bounds__(256) scan_apply_kernel(EwArgs a) {
     float s_lam = 0.0f, s_ba = 0.0f, s_bx = 0.0f;
     // running pointers at token t1 - 8 (the loop walks backwards in steps of eight tokens)
     const size_t tokb = (size_t)b * T + (t1 - 8);
-    const size_t sD = (size_t)D, sZ = (size_t)a.H * 2 * DH;          // token strides of [tok][D] and [tok][H][2][256] arrays
-    const __nv_bfloat16 *p_dy = a.dy + tokb * sD + d, *p_y = a.y + (tokb - 1) * sD + d;
-    const __half *p_z = a.z + tokb * sZ + (size_t)h * 2 * DH + n, *p_u = a.u + tokb * sD + d;
-    __half *p_dz = a.dz + tokb * sZ + (size_t)h * 2 * DH + n;
-    float *p_du = a.du + tokb * sD + d;
+    const uint32_t sD = (uint32_t)D, sZ = (uint32_t)a.H * 2 * DH;      // token strides of [tok][D] and [tok][H][2][256] arrays; eight tokens' worth fits 32 bits
+    const __nv_bfloat16 *p_dy = a.dy + tokb * (size_t)sD + d, *p_y = a.y + (tokb - 1) * (size_t)sD + d;
+    const __half *p_z = a.z + tokb * (size_t)sZ + (size_t)h * 2 * DH + n, *p_u = a.u + tokb * (size_t)sD + d;
+    __half *p_dz = a.dz + tokb * (size_t)sZ + (size_t)h * 2 * DH + n;
+    float *p_du = a.du + tokb * (size_t)sD + d;
     __half *p_ta = a.dzT + ((size_t)h * 2 * DH + n) * a.BTp + tokb, *p_tx = p_ta + (size_t)DH * a.BTp;
     const float h0v = a.h0 ? a.h0[(size_t)b * D + d] : 0.0f;
     // eight tokens at the running pointers, newest first; the channel-major copies of dz come back packed
@@ -361,7 +363,7 @@ __global__ void __launch_bounds__(256) scan_apply_kernel(EwArgs a) {
         for (int k = 7; k >= 0; --k) {
             const float r = sigmoid_fast(zav[k] + ba), gi = sigmoid_fast(zxv[k] + bx);
             const float L = -s * r, at = __expf(L), m2 = one_minus_exp(2.0f * L);
-            const float mt = sqrtf(m2), rm = m2 > 0.0f ? rsqrtf(m2) : 0.0f;
+            const float rm = m2 > 0.0f ? rsqrt_fast(m2) : 0.0f, mt = m2 * rm;   // 1/sqrt(1 - a^2) and sqrt(1 - a^2) from one MUFU
             const float g = dyv[k] + carry;
             carry = at * g;
             const float v = gi * uv[k];
@@ -377,7 +379,7 @@ __global__ void __launch_bounds__(256) scan_apply_kernel(EwArgs a) {
             const uint32_t ba16 = (uint32_t)__half_as_ushort(ha), bx16 = (uint32_t)__half_as_ushort(hx);
             if (k & 1) { pa[k >> 1] = ba16 << 16; px[k >> 1] = bx16 << 16; } else { pa[k >> 1] |= ba16; px[k >> 1] |= bx16; }
         }
-        p_dy -= 8 * sD; p_y -= 8 * sD; p_z -= 8 * sZ; p_u -= 8 * sD; p_dz -= 8 * sZ; p_du -= 8 * sD;
+        p_dy -= 8 * (size_t)sD; p_y -= 8 * (size_t)sD; p_z -= 8 * (size_t)sZ; p_u -= 8 * (size_t)sD; p_dz -= 8 * (size_t)sZ; p_du -= 8 * (size_t)sD;
     };
     int tb = t1 - 8;
     // sixteen tokens per round, so that each channel-major row gets 32 adjacent bytes (a whole sector) at once

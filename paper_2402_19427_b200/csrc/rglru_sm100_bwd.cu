@@ -9,7 +9,7 @@
 //   3. scan_fold / scan_carry / scan_apply
 //                        reverse-time scan g_t = dy_t + a_{t+1} g_{t+1} over chunks of 128 tokens (fold, carry across
 //                        chunks, re-run with the carry), then the element-wise adjoints: dz_a, dz_x (fp16, token-major
-//                        and channel-major), the direct part of du (fp32), partial sums of dLambda, db_a, db_x
+//                        and channel-major), the direct part of du (fp16), partial sums of dLambda, db_a, db_x
 //   4. GEMM              du += dz_a W_a + dz_x W_x
 //   5. GEMM (split K)    dW_a | dW_x = dz^T u over all tokens, fp32 partial sums per split, reduced in fixed order
 //   6. Conv1D adjoint    dx, dconv_w, dconv_b with sliding windows, fixed-order reductions
@@ -47,7 +47,7 @@ struct GemmArgs {
     int nx, ny;        // tile grid: nx x ny x H
     int kblocks;       // 64-wide K blocks per CTA
     int rows_valid;    // MODE_Z / MODE_DU: number of tokens; MODE_DW: 512
-    void *out;         // MODE_Z: __half z[tok][H][2][256]; MODE_DU: float du[tok][D] (+=); MODE_DW: float part[split][2][H][256][256]
+    void *out;         // MODE_Z: __half z[tok][H][2][256]; MODE_DU: __half du[tok][D] (+=); MODE_DW: float part[split][2][H][256][256]
     uint32_t *status;
     unsigned long long spin_ns;
 };
@@ -164,13 +164,19 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
 #pragma unroll
                     for (int j = 0; j < 4; ++j) ((uint4 *)dst)[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
                 } else if (p.mode == MODE_DU) {
-                    float4 *dst = (float4 *)((float *)p.out + (size_t)row * p.D + h * DH + c0);
+                    // du is kept in fp16 like dz (bf16 failed the dx tolerance where the taps of the Conv1D adjoint cancel)
+                    uint4 *dst = (uint4 *)((__half *)p.out + (size_t)row * p.D + h * DH + c0);
+                    uint4 o[4];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        float4 o = dst[j];
-                        o.x += lo2(v[2 * j]); o.y += hi2(v[2 * j]); o.z += lo2(v[2 * j + 1]); o.w += hi2(v[2 * j + 1]);
-                        dst[j] = o;
+                    for (int j = 0; j < 4; ++j) o[j] = dst[j];
+                    uint32_t *ow = (uint32_t *)o;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const float2 old = __half22float2(*(const __half2 *)&ow[j]);
+                        ow[j] = pack_f16_sat(old.x + lo2(v[j]), old.y + hi2(v[j]));
                     }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) dst[j] = o[j];
                 } else {
                     const int g = row >> 8, o_row = row & 255;
                     float4 *dst = (float4 *)((float *)p.out + ((((size_t)ty * 2 + g) * p.H + h) * 256 + o_row) * 256 + c0);
@@ -223,7 +229,7 @@ struct EwArgs {
     const float *conv_b, *b_a, *b_x, *lambda, *h0;
     __half *u, *uT, *dz, *dzT;
     const __half *z;
-    float *du;                        // [tok][D]
+    __half *du;                       // [tok][D]
     float2 *fold;                     // [B][nchunk][D]: (prod a_t, carry out of the chunk for zero carry in)
     float *xin;                       // [B][nchunk][D]: a_{t+1} g_{t+1} entering the chunk from later tokens
     float *part_vec;                  // [B*nchunk][3][D]
@@ -345,7 +351,7 @@ __global__ void __launch_bounds__(256, 3) scan_apply_kernel(EwArgs a) {
     const __nv_bfloat16 *p_dy = a.dy + tokb * (size_t)sD + d, *p_y = a.y + (tokb - 1) * (size_t)sD + d;
     const __half *p_z = a.z + tokb * (size_t)sZ + (size_t)h * 2 * DH + n, *p_u = a.u + tokb * (size_t)sD + d;
     __half *p_dz = a.dz + tokb * (size_t)sZ + (size_t)h * 2 * DH + n;
-    float *p_du = a.du + tokb * (size_t)sD + d;
+    __half *p_du = a.du + tokb * (size_t)sD + d;
     __half *p_ta = a.dzT + ((size_t)h * 2 * DH + n) * a.BTp + tokb, *p_tx = p_ta + (size_t)DH * a.BTp;
     const float h0v = a.h0 ? a.h0[(size_t)b * D + d] : 0.0f;
     // eight tokens at the running pointers, newest first; the channel-major copies of dz come back packed
@@ -372,7 +378,7 @@ __global__ void __launch_bounds__(256, 3) scan_apply_kernel(EwArgs a) {
             const float dza = -s * dL * r * (1.0f - r), dzx = dv * uv[k] * gi * (1.0f - gi);
             s_lam = fmaf(dL * r, dsdlam_neg, s_lam);
             s_ba += dza; s_bx += dzx;
-            p_du[k * sD] = dv * gi;
+            p_du[k * sD] = to_half_sat(dv * gi);
             const __half ha = to_half_sat(dza), hx = to_half_sat(dzx);
             p_dz[k * sZ] = ha;
             p_dz[k * sZ + DH] = hx;
@@ -409,7 +415,7 @@ __global__ void __launch_bounds__(256, 3) scan_apply_kernel(EwArgs a) {
 struct ConvBwdArgs {
     int B, T, D, nchunk;
     const __nv_bfloat16 *x, *conv_w, *cs_in;
-    const float *du;
+    const __half *du;
     __nv_bfloat16 *dx;
     float *part_conv;   // [B*nchunk][5][D]
 };
@@ -425,7 +431,7 @@ __global__ void __launch_bounds__(256) conv_backward_kernel(ConvBwdArgs a) {
         if (t >= 0) return bf2f(a.x[((size_t)b * T + t) * D + d]);
         return a.cs_in ? bf2f(a.cs_in[((size_t)b * 3 + (3 + t)) * D + d]) : 0.0f;
     };
-    auto duat = [&](int t) -> float { return t < T ? a.du[((size_t)b * T + t) * D + d] : 0.0f; };
+    auto duat = [&](int t) -> float { return t < T ? __half2float(a.du[((size_t)b * T + t) * D + d]) : 0.0f; };
     float x1 = xat(t0 - 1), x2 = xat(t0 - 2), x3 = xat(t0 - 3);     // x_{t-1}, x_{t-2}, x_{t-3}
     float g0 = duat(t0), g1 = duat(t0 + 1), g2 = duat(t0 + 2);     // du_t, du_{t+1}, du_{t+2}
     for (int tb = t0; tb < t1; tb += 8) {
@@ -479,7 +485,7 @@ BwdLayout bwd_layout(int B, int T, int D, int H) {
     L.off_z = take(L.BT * D * 2 * 2);
     L.off_dz = take(L.BT * D * 2 * 2);
     L.off_dzT = take((size_t)D * 2 * L.BTp * 2);
-    L.off_du = take(L.BT * D * 4);
+    L.off_du = take(L.BT * D * 2);
     L.off_y = take(L.BT * D * 2);
     L.off_hT = take((size_t)B * D * 4);
     L.off_cs = take((size_t)B * 3 * D * 2);
@@ -518,7 +524,7 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
     char *ws = (char *)ws_body;
     __half *u = (__half *)(ws + L.off_u), *uT = (__half *)(ws + L.off_uT), *z = (__half *)(ws + L.off_z);
     __half *dz = (__half *)(ws + L.off_dz), *dzT = (__half *)(ws + L.off_dzT), *WT = (__half *)(ws + L.off_wt), *W16 = (__half *)(ws + L.off_w16);
-    float *du = (float *)(ws + L.off_du);
+    __half *du = (__half *)(ws + L.off_du);
 
     // 0. h_{t-1} comes from the forward output; run the forward when the caller kept none
     const void *y = y_saved;

@@ -59,6 +59,16 @@ struct GemmArgs {
 //   MODE_Z : (token tiles, 2 gates, H)   A = u[tok][h][k]        B = W_gate[h][out][k]
 //   MODE_DU: (token tiles, 1, H)         A = dz[tok][h][k=512]   B = W^T[h][in][k=512]
 //   MODE_DW: (4 row tiles, splits, H)    A = dz^T[h][row][tok]   B = u^T[h][in][tok], K = this split's tokens
+// 32-byte accesses: one whole DRAM sector per thread and instruction where a thread owns a row (pointers 32-byte aligned)
+__device__ __forceinline__ void st_global_v8(void *ptr, const uint32_t (&r)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(ptr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]),
+                 "r"(r[6]), "r"(r[7]) : "memory");
+}
+__device__ __forceinline__ void ld_global_v8(const void *ptr, uint32_t (&r)[8]) {
+    asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]),
+                 "=r"(r[6]), "=r"(r[7]) : "l"(ptr) : "memory");
+}
+
 __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_constant__ GemmArgs p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -74,6 +84,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const unsigned long long spin = p.spin_ns;
     const int ntiles = p.nx * p.ny * p.H;
+    // each CTA takes a contiguous run of tiles (tx fastest), so that consecutive tiles share their B operand
+    const int tile_begin = (int)((long long)blockIdx.x * ntiles / gridDim.x), tile_end = (int)((long long)(blockIdx.x + 1) * ntiles / gridDim.x);
 
     if (tid == 0) {
         for (int s = 0; s < GEMM_STAGES; ++s) { mbar_init(BAR_FULL(s), 1); mbar_init(BAR_EMPTY(s), 1); }
@@ -92,14 +104,20 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
         // ---- TMA producer
         if (lane == 0) {
             int kbg = 0;   // K blocks issued so far, over all tiles (ring position)
-            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+            // MODE_Z has as many K blocks as the ring has stages, so K block kb always lands in stage kb: while the
+            // (head, gate) of the tile stays the same its B operand (the weights, 128 KB) is simply left where it is
+            const bool b_stays = p.mode == MODE_Z && p.kblocks == GEMM_STAGES;
+            int prev_b = -1;
+            for (int tile = tile_begin; tile < tile_end && ok; ++tile) {
                 const int tx = tile % p.nx, ty = (tile / p.nx) % p.ny, h = tile / (p.nx * p.ny);
                 const CUtensorMap *tb = (p.mode == MODE_Z && ty == 1) ? &p.tm_b1 : &p.tm_b0;
+                const bool load_b = !(b_stays && prev_b == tile / p.nx);
+                prev_b = tile / p.nx;
                 for (int kb = 0; kb < p.kblocks; ++kb, ++kbg) {
                     const int s = kbg % GEMM_STAGES;
                     ok = mbar_wait(BAR_EMPTY(s), ((kbg / GEMM_STAGES) & 1) ^ 1, spin, abort_flag);
                     if (!ok) break;
-                    mbar_expect_tx(BAR_FULL(s), STAGE_BYTES);
+                    mbar_expect_tx(BAR_FULL(s), load_b ? STAGE_BYTES : A_STAGE_BYTES);
                     const uint32_t a_dst = base + s * STAGE_BYTES, b_dst = a_dst + A_STAGE_BYTES;
                     if (p.mode == MODE_DW) {
                         const int k0 = (ty * p.kblocks + kb) * 64;
@@ -107,7 +125,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                         tma_load_3d(b_dst, tb, k0, 0, h, BAR_FULL(s));
                     } else {
                         tma_load_3d(a_dst, &p.tm_a, kb * 64, h, tx * 128, BAR_FULL(s));
-                        tma_load_3d(b_dst, tb, kb * 64, 0, h, BAR_FULL(s));
+                        if (load_b) tma_load_3d(b_dst, tb, kb * 64, 0, h, BAR_FULL(s));
                     }
                 }
             }
@@ -118,7 +136,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_f16(128, 256);
             int kbg = 0, it = 0;
-            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
+            for (int tile = tile_begin; tile < tile_end && ok; ++tile, ++it) {
                 const int acc = it & 1;
                 ok = mbar_wait(BAR_ACCEMPTY(acc), ((it >> 1) & 1) ^ 1, spin, abort_flag);   // epilogue of tile it - 2 done
                 if (!ok) break;
@@ -141,7 +159,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
         // ---- epilogue: warp owns TMEM lanes 32 (warp & 3) .. +31 = rows of the tile
         const int q = warp & 3;
         int it = 0;
-        for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
+        for (int tile = tile_begin; tile < tile_end && ok; ++tile, ++it) {
             const int tx = tile % p.nx, ty = (tile / p.nx) % p.ny, h = tile / (p.nx * p.ny);
             const int acc = it & 1;
             const int row = tx * 128 + q * 32 + lane;
@@ -158,30 +176,37 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                 if (!valid) continue;
                 if (p.mode == MODE_Z) {
                     __half *dst = (__half *)p.out + (((size_t)row * p.H + h) * 2 + ty) * 256 + c0;
-                    uint32_t w[16];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) { const __half2 hh = __floats2half2_rn(lo2(v[j]), hi2(v[j])); w[j] = *(const uint32_t *)&hh; }
+                    for (int j8 = 0; j8 < 2; ++j8) {
+                        uint32_t w[8];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) ((uint4 *)dst)[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                        for (int j = 0; j < 8; ++j) { const __half2 hh = __floats2half2_rn(lo2(v[8 * j8 + j]), hi2(v[8 * j8 + j])); w[j] = *(const uint32_t *)&hh; }
+                        st_global_v8(dst + 16 * j8, w);
+                    }
                 } else if (p.mode == MODE_DU) {
                     // du is kept in fp16 like dz (bf16 failed the dx tolerance where the taps of the Conv1D adjoint cancel)
-                    uint4 *dst = (uint4 *)((__half *)p.out + (size_t)row * p.D + h * DH + c0);
-                    uint4 o[4];
+                    __half *dst = (__half *)p.out + (size_t)row * p.D + h * DH + c0;
+                    uint32_t o0[8], o1[8];
+                    ld_global_v8(dst, o0);
+                    ld_global_v8(dst + 16, o1);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) o[j] = dst[j];
-                    uint32_t *ow = (uint32_t *)o;
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const float2 old = __half22float2(*(const __half2 *)&ow[j]);
-                        ow[j] = pack_f16_sat(old.x + lo2(v[j]), old.y + hi2(v[j]));
+                    for (int j = 0; j < 8; ++j) {
+                        const float2 a0 = __half22float2(*(const __half2 *)&o0[j]), a1 = __half22float2(*(const __half2 *)&o1[j]);
+                        o0[j] = pack_f16_sat(a0.x + lo2(v[j]), a0.y + hi2(v[j]));
+                        o1[j] = pack_f16_sat(a1.x + lo2(v[8 + j]), a1.y + hi2(v[8 + j]));
                     }
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) dst[j] = o[j];
+                    st_global_v8(dst, o0);
+                    st_global_v8(dst + 16, o1);
                 } else {
                     const int g = row >> 8, o_row = row & 255;
-                    float4 *dst = (float4 *)((float *)p.out + ((((size_t)ty * 2 + g) * p.H + h) * 256 + o_row) * 256 + c0);
+                    float *dst = (float *)p.out + ((((size_t)ty * 2 + g) * p.H + h) * 256 + o_row) * 256 + c0;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) dst[j] = make_float4(lo2(v[2 * j]), hi2(v[2 * j]), lo2(v[2 * j + 1]), hi2(v[2 * j + 1]));
+                    for (int j = 0; j < 4; ++j) {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) { w[2 * e] = __float_as_uint(lo2(v[4 * j + e])); w[2 * e + 1] = __float_as_uint(hi2(v[4 * j + e])); }
+                        st_global_v8(dst + 8 * j, w);
+                    }
                 }
             }
             tc_fence_before();
@@ -393,10 +418,17 @@ __global__ void __launch_bounds__(256, 3) scan_apply_kernel(EwArgs a) {
         uint32_t pa1[4], px1[4], pa0[4], px0[4];
         batch8(tb, pa1, px1);
         batch8(tb - 8, pa0, px0);
-        *(uint4 *)(p_ta - 8) = make_uint4(pa0[0], pa0[1], pa0[2], pa0[3]);
-        *(uint4 *)p_ta = make_uint4(pa1[0], pa1[1], pa1[2], pa1[3]);
-        *(uint4 *)(p_tx - 8) = make_uint4(px0[0], px0[1], px0[2], px0[3]);
-        *(uint4 *)p_tx = make_uint4(px1[0], px1[1], px1[2], px1[3]);
+        if ((reinterpret_cast<uintptr_t>(p_ta - 8) & 31) == 0) {
+            const uint32_t wa[8] = {pa0[0], pa0[1], pa0[2], pa0[3], pa1[0], pa1[1], pa1[2], pa1[3]};
+            const uint32_t wx[8] = {px0[0], px0[1], px0[2], px0[3], px1[0], px1[1], px1[2], px1[3]};
+            st_global_v8(p_ta - 8, wa);
+            st_global_v8(p_tx - 8, wx);
+        } else {
+            *(uint4 *)(p_ta - 8) = make_uint4(pa0[0], pa0[1], pa0[2], pa0[3]);
+            *(uint4 *)p_ta = make_uint4(pa1[0], pa1[1], pa1[2], pa1[3]);
+            *(uint4 *)(p_tx - 8) = make_uint4(px0[0], px0[1], px0[2], px0[3]);
+            *(uint4 *)p_tx = make_uint4(px1[0], px1[1], px1[2], px1[3]);
+        }
         p_ta -= 16; p_tx -= 16;
     }
     if (tb >= t0) {

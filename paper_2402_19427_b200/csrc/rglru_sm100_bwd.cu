@@ -84,8 +84,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const unsigned long long spin = p.spin_ns;
     const int ntiles = p.nx * p.ny * p.H;
-    // each CTA takes a contiguous run of tiles (tx fastest), so that consecutive tiles share their B operand
-    const int tile_begin = (int)((long long)blockIdx.x * ntiles / gridDim.x), tile_end = (int)((long long)(blockIdx.x + 1) * ntiles / gridDim.x);
+    // Tiles are dealt round-robin.  (Contiguous runs per CTA, with the B operand left in shared memory while head and gate
+    // stay the same, measured 4 % slower on the whole backward: the operand re-reads hit L2 and were not the limit.)
 
     if (tid == 0) {
         for (int s = 0; s < GEMM_STAGES; ++s) { mbar_init(BAR_FULL(s), 1); mbar_init(BAR_EMPTY(s), 1); }
@@ -104,20 +104,14 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
         // ---- TMA producer
         if (lane == 0) {
             int kbg = 0;   // K blocks issued so far, over all tiles (ring position)
-            // MODE_Z has as many K blocks as the ring has stages, so K block kb always lands in stage kb: while the
-            // (head, gate) of the tile stays the same its B operand (the weights, 128 KB) is simply left where it is
-            const bool b_stays = p.mode == MODE_Z && p.kblocks == GEMM_STAGES;
-            int prev_b = -1;
-            for (int tile = tile_begin; tile < tile_end && ok; ++tile) {
+            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
                 const int tx = tile % p.nx, ty = (tile / p.nx) % p.ny, h = tile / (p.nx * p.ny);
                 const CUtensorMap *tb = (p.mode == MODE_Z && ty == 1) ? &p.tm_b1 : &p.tm_b0;
-                const bool load_b = !(b_stays && prev_b == tile / p.nx);
-                prev_b = tile / p.nx;
                 for (int kb = 0; kb < p.kblocks; ++kb, ++kbg) {
                     const int s = kbg % GEMM_STAGES;
                     ok = mbar_wait(BAR_EMPTY(s), ((kbg / GEMM_STAGES) & 1) ^ 1, spin, abort_flag);
                     if (!ok) break;
-                    mbar_expect_tx(BAR_FULL(s), load_b ? STAGE_BYTES : A_STAGE_BYTES);
+                    mbar_expect_tx(BAR_FULL(s), STAGE_BYTES);
                     const uint32_t a_dst = base + s * STAGE_BYTES, b_dst = a_dst + A_STAGE_BYTES;
                     if (p.mode == MODE_DW) {
                         const int k0 = (ty * p.kblocks + kb) * 64;
@@ -125,7 +119,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                         tma_load_3d(b_dst, tb, k0, 0, h, BAR_FULL(s));
                     } else {
                         tma_load_3d(a_dst, &p.tm_a, kb * 64, h, tx * 128, BAR_FULL(s));
-                        if (load_b) tma_load_3d(b_dst, tb, kb * 64, 0, h, BAR_FULL(s));
+                        tma_load_3d(b_dst, tb, kb * 64, 0, h, BAR_FULL(s));
                     }
                 }
             }
@@ -136,7 +130,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_f16(128, 256);
             int kbg = 0, it = 0;
-            for (int tile = tile_begin; tile < tile_end && ok; ++tile, ++it) {
+            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
                 const int acc = it & 1;
                 ok = mbar_wait(BAR_ACCEMPTY(acc), ((it >> 1) & 1) ^ 1, spin, abort_flag);   // epilogue of tile it - 2 done
                 if (!ok) break;
@@ -159,7 +153,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
         // ---- epilogue: warp owns TMEM lanes 32 (warp & 3) .. +31 = rows of the tile
         const int q = warp & 3;
         int it = 0;
-        for (int tile = tile_begin; tile < tile_end && ok; ++tile, ++it) {
+        for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
             const int tx = tile % p.nx, ty = (tile / p.nx) % p.ny, h = tile / (p.nx * p.ny);
             const int acc = it & 1;
             const int row = tx * 128 + q * 32 + lane;
@@ -288,13 +282,14 @@ __global__ void __launch_bounds__(256) conv_forward_kernel(EwArgs a) {
     };
     float x3 = xat(t0 - 3), x2 = xat(t0 - 2), x1 = xat(t0 - 1);
     // eight tokens: u token-major (coalesced across the block) and eight fp16 values of this channel's row
-    auto batch8 = [&](int t, const float (&xs)[8]) -> uint4 {
+    const uint32_t sD = (uint32_t)D;   // token stride; sixteen tokens' worth fits 32 bits
+    auto batch8 = [&](__half *pu, const float (&xs)[8]) -> uint4 {
         uint32_t packed[4];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             const float uv = fmaf(w[3], x3, fmaf(w[2], x2, fmaf(w[1], x1, fmaf(w[0], xs[k], cb))));
             const __half ub = to_half_sat(uv);
-            a.u[((size_t)b * T + t + k) * D + d] = ub;
+            pu[k * sD] = ub;
             const uint32_t bits = (uint32_t)__half_as_ushort(ub);
             if (k & 1) packed[k >> 1] |= bits << 16; else packed[k >> 1] = bits;
             x3 = x2; x2 = x1; x1 = xs[k];
@@ -305,16 +300,22 @@ __global__ void __launch_bounds__(256) conv_forward_kernel(EwArgs a) {
     for (; t + 16 <= t1; t += 16) {   // sixteen tokens: the channel-major store fills whole 32-byte sectors
         float xa[8], xb[8];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) { xa[k] = bf2f(a.x[((size_t)b * T + t + k) * D + d]); xb[k] = bf2f(a.x[((size_t)b * T + t + 8 + k) * D + d]); }
-        const uint4 lo = batch8(t, xa), hi = batch8(t + 8, xb);
-        uint4 *dst = (uint4 *)(a.uT + (size_t)d * a.BTp + (size_t)b * T + t);
-        dst[0] = lo; dst[1] = hi;
+        const __nv_bfloat16 *px = a.x + ((size_t)b * T + t) * D + d;
+        __half *pu = a.u + ((size_t)b * T + t) * D + d;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { xa[k] = bf2f(px[k * sD]); xb[k] = bf2f(px[(8 + k) * sD]); }
+        const uint4 lo = batch8(pu, xa), hi = batch8(pu + 8 * (size_t)sD, xb);
+        __half *dst = a.uT + (size_t)d * a.BTp + (size_t)b * T + t;
+        if ((reinterpret_cast<uintptr_t>(dst) & 31) == 0) {
+            const uint32_t wv[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+            st_global_v8(dst, wv);
+        } else { ((uint4 *)dst)[0] = lo; ((uint4 *)dst)[1] = hi; }
     }
     if (t < t1) {
         float xa[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) xa[k] = bf2f(a.x[((size_t)b * T + t + k) * D + d]);
-        *(uint4 *)(a.uT + (size_t)d * a.BTp + (size_t)b * T + t) = batch8(t, xa);
+        *(uint4 *)(a.uT + (size_t)d * a.BTp + (size_t)b * T + t) = batch8(a.u + ((size_t)b * T + t) * D + d, xa);
     }
 }
 
@@ -327,8 +328,8 @@ __global__ void __launch_bounds__(256) scan_fold_kernel(EwArgs a) {
     const float s = decay_rate(a.lambda[d], a.c), ba = a.b_a[d];
     float carry = 0.0f, Q = 1.0f;
     const size_t tokb = (size_t)b * T + (t1 - 8);
-    const size_t sD = (size_t)D, sZ = (size_t)a.H * 2 * DH;
-    const __nv_bfloat16 *p_dy = a.dy + tokb * sD + d;
+    const uint32_t sD = (uint32_t)D, sZ = (uint32_t)a.H * 2 * DH;
+    const __nv_bfloat16 *p_dy = a.dy + tokb * (size_t)sD + d;
     const __half *p_z = a.z + tokb * sZ + (size_t)h * 2 * DH + n;
     for (int tb = t1 - 8; tb >= t0; tb -= 8) {
         float dyv[8], zav[8];
@@ -341,7 +342,7 @@ __global__ void __launch_bounds__(256) scan_fold_kernel(EwArgs a) {
             carry = at * g;
             Q *= at;
         }
-        p_dy -= 8 * sD; p_z -= 8 * sZ;
+        p_dy -= 8 * (size_t)sD; p_z -= 8 * (size_t)sZ;
     }
     a.fold[((size_t)b * a.nchunk + c) * D + d] = make_float2(Q, carry);
 }
@@ -466,14 +467,24 @@ __global__ void __launch_bounds__(256) conv_backward_kernel(ConvBwdArgs a) {
     auto duat = [&](int t) -> float { return t < T ? __half2float(a.du[((size_t)b * T + t) * D + d]) : 0.0f; };
     float x1 = xat(t0 - 1), x2 = xat(t0 - 2), x3 = xat(t0 - 3);     // x_{t-1}, x_{t-2}, x_{t-3}
     float g0 = duat(t0), g1 = duat(t0 + 1), g2 = duat(t0 + 2);     // du_t, du_{t+1}, du_{t+2}
+    const uint32_t sD = (uint32_t)D;   // token stride; eleven tokens' worth fits 32 bits
     for (int tb = t0; tb < t1; tb += 8) {
         float xs[8], gs[8];
+        const size_t row = ((size_t)b * T + tb) * D + d;
+        const __nv_bfloat16 *px = a.x + row;
+        const __half *pg = a.du + row;
+        __nv_bfloat16 *pdx = a.dx + row;
+        if (tb + 11 <= T) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) { xs[k] = bf2f(a.x[((size_t)b * T + tb + k) * D + d]); gs[k] = duat(tb + k + 3); }
+            for (int k = 0; k < 8; ++k) { xs[k] = bf2f(px[k * sD]); gs[k] = __half2float(pg[(k + 3) * sD]); }
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) { xs[k] = bf2f(px[k * sD]); gs[k] = duat(tb + k + 3); }
+        }
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             const float g3 = gs[k], x0 = xs[k];
-            a.dx[((size_t)b * T + tb + k) * D + d] = __float2bfloat16_rn(fmaf(w[3], g3, fmaf(w[2], g2, fmaf(w[1], g1, w[0] * g0))));
+            pdx[k * sD] = __float2bfloat16_rn(fmaf(w[3], g3, fmaf(w[2], g2, fmaf(w[1], g1, w[0] * g0))));
             sw[0] = fmaf(g0, x0, sw[0]); sw[1] = fmaf(g0, x1, sw[1]); sw[2] = fmaf(g0, x2, sw[2]); sw[3] = fmaf(g0, x3, sw[3]);
             sb += g0;
             g0 = g1; g1 = g2; g2 = g3;

@@ -374,6 +374,24 @@ __global__ void reduce_partials_kernel(const float *in, int nparts, size_t strid
     out[i] = acc;
 }
 
+// out[i] = sum over p of in[p * stride + i] in a fixed order (four interleaved running sums, added at the end), the row being
+// split over three output arrays
+__global__ void reduce_partials3_kernel(const float *in, int nparts, size_t stride, float *out0, size_t n0, float *out1, size_t n1,
+                                        float *out2, size_t n2) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n0 + n1 + n2) return;
+    float *out = i < n0 ? (out0 ? out0 + i : nullptr) : i < n0 + n1 ? (out1 ? out1 + (i - n0) : nullptr) : (out2 ? out2 + (i - n0 - n1) : nullptr);
+    if (out == nullptr) return;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    int p = 0;
+    for (; p + 4 <= nparts; p += 4) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[j] += in[(size_t)(p + j) * stride + i];
+    }
+    for (; p < nparts; ++p) acc[0] += in[(size_t)p * stride + i];
+    *out = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+}
+
 size_t fwd_smem_bytes(int Dh) { return sizeof(float) * ((size_t)GT * Dh + Dh + 2 * NB * (NT + 1)); }
 
 template <typename K>
@@ -426,6 +444,14 @@ cudaError_t generic_decode(const FwdArgs &a, int io, cudaStream_t st) {
 cudaError_t reduce_partials(const float *in, int nparts, size_t stride, float *out, size_t n, cudaStream_t st) {
     if (out == nullptr || n == 0) return cudaSuccess;
     reduce_partials_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(in, nparts, stride, out, n);
+    return cudaGetLastError();
+}
+
+cudaError_t reduce_partials3(const float *in, int nparts, size_t stride, float *out0, size_t n0, float *out1, size_t n1, float *out2,
+                             size_t n2, cudaStream_t st) {
+    const size_t n = n0 + n1 + n2;
+    if (n == 0 || (out0 == nullptr && out1 == nullptr && out2 == nullptr)) return cudaSuccess;
+    reduce_partials3_kernel<<<(unsigned)((n + 127) / 128), 128, 0, st>>>(in, nparts, stride, out0, n0, out1, n1, out2, n2);
     return cudaGetLastError();
 }
 

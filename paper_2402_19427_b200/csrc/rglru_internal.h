@@ -80,5 +80,9 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &b, const void *y_saved, 
                            cudaStream_t st);
 // out[i] = sum over p of in[p * stride + i] in ascending p (fixed order: run-to-run identical results)
 cudaError_t reduce_partials(const float *in, int nparts, size_t stride, float *out, size_t n, cudaStream_t st);
+// A row of n0 + n1 + n2 values summed over the parts and split over up to three output arrays (any of them may be null or
+// empty); four interleaved running sums over ascending p, added at the end: also a fixed order.
+cudaError_t reduce_partials3(const float *in, int nparts, size_t stride, float *out0, size_t n0, float *out1, size_t n1, float *out2,
+                             size_t n2, cudaStream_t st);
 
 }  // namespace rglru

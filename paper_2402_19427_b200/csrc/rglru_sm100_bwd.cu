@@ -382,6 +382,7 @@ __global__ void __launch_bounds__(256, 3) scan_apply_kernel(EwArgs a) {
     const float h0v = a.h0 ? a.h0[(size_t)b * D + d] : 0.0f;
     // eight tokens at the running pointers, newest first; the channel-major copies of dz come back packed
     auto batch8 = [&](int tb, uint32_t (&pa)[4], uint32_t (&px)[4]) {
+        float dza_hi = 0.0f, dzx_hi = 0.0f;
         float dyv[8], hpv[8], zav[8], zxv[8], uv[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
@@ -405,11 +406,16 @@ __global__ void __launch_bounds__(256, 3) scan_apply_kernel(EwArgs a) {
             s_lam = fmaf(dL * r, dsdlam_neg, s_lam);
             s_ba += dza; s_bx += dzx;
             p_du[k * sD] = to_half_sat(dv * gi);
-            const __half ha = to_half_sat(dza), hx = to_half_sat(dzx);
-            p_dz[k * sZ] = ha;
-            p_dz[k * sZ + DH] = hx;
-            const uint32_t ba16 = (uint32_t)__half_as_ushort(ha), bx16 = (uint32_t)__half_as_ushort(hx);
-            if (k & 1) { pa[k >> 1] = ba16 << 16; px[k >> 1] = bx16 << 16; } else { pa[k >> 1] |= ba16; px[k >> 1] |= bx16; }
+            // tokens k (odd) and k - 1 share one packed conversion: the pair is what the channel-major copy stores
+            if (k & 1) { dza_hi = dza; dzx_hi = dzx; }
+            else {
+                const uint32_t wa = pack_f16_sat(dza, dza_hi), wx = pack_f16_sat(dzx, dzx_hi);
+                pa[k >> 1] = wa; px[k >> 1] = wx;
+                p_dz[k * sZ] = __ushort_as_half((unsigned short)(wa & 0xFFFFu));
+                p_dz[(k + 1) * sZ] = __ushort_as_half((unsigned short)(wa >> 16));
+                p_dz[k * sZ + DH] = __ushort_as_half((unsigned short)(wx & 0xFFFFu));
+                p_dz[(k + 1) * sZ + DH] = __ushort_as_half((unsigned short)(wx >> 16));
+            }
         }
         p_dy -= 8 * (size_t)sD; p_y -= 8 * (size_t)sD; p_z -= 8 * (size_t)sZ; p_u -= 8 * (size_t)sD; p_dz -= 8 * (size_t)sZ; p_du -= 8 * (size_t)sD;
     };
@@ -645,21 +651,17 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
         g.nx = 4; g.ny = L.S;
         tc_gemm_kernel<<<gemm_grid(g), GEMM_THREADS, GEMM_SMEM_ALLOC, st>>>(g);
         const size_t wsz = (size_t)H * DH * DH;
-        if ((e = reduce_partials(part, L.S, 2 * wsz, q.dW_a, wsz, st)) != cudaSuccess) return e;
-        if ((e = reduce_partials(part + wsz, L.S, 2 * wsz, q.dW_x, wsz, st)) != cudaSuccess) return e;
+        if ((e = reduce_partials3(part, L.S, 2 * wsz, q.dW_a, wsz, q.dW_x, wsz, nullptr, 0, st)) != cudaSuccess) return e;
     }
     // 6. per-channel sums, Conv1D adjoint
     const int nparts = B * L.nchunk;
-    if ((e = reduce_partials(a.part_vec, nparts, (size_t)3 * D, q.dlambda, D, st)) != cudaSuccess) return e;
-    if ((e = reduce_partials(a.part_vec + D, nparts, (size_t)3 * D, q.db_a, D, st)) != cudaSuccess) return e;
-    if ((e = reduce_partials(a.part_vec + 2 * (size_t)D, nparts, (size_t)3 * D, q.db_x, D, st)) != cudaSuccess) return e;
+    if ((e = reduce_partials3(a.part_vec, nparts, (size_t)3 * D, q.dlambda, D, q.db_a, D, q.db_x, D, st)) != cudaSuccess) return e;
     ConvBwdArgs cb{};
     cb.B = B; cb.T = T; cb.D = D; cb.nchunk = L.nchunk;
     cb.x = a.x; cb.conv_w = a.conv_w; cb.cs_in = a.cs_in; cb.du = du; cb.dx = (__nv_bfloat16 *)q.dx;
     cb.part_conv = (float *)(ws + L.off_pconv);
     conv_backward_kernel<<<grid_ew, 256, 0, st>>>(cb);
-    if ((e = reduce_partials(cb.part_conv, nparts, (size_t)5 * D, q.dconv_w, (size_t)4 * D, st)) != cudaSuccess) return e;
-    if ((e = reduce_partials(cb.part_conv + 4 * (size_t)D, nparts, (size_t)5 * D, q.dconv_b, D, st)) != cudaSuccess) return e;
+    if ((e = reduce_partials3(cb.part_conv, nparts, (size_t)5 * D, q.dconv_w, (size_t)4 * D, q.dconv_b, D, nullptr, 0, st)) != cudaSuccess) return e;
     return cudaGetLastError();
 }
 

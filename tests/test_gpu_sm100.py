@@ -28,6 +28,18 @@ def test_shapes_with_state_and_bias(oracle, B, T, H):
     assert np.array_equal(cso, cr)
 
 
+def test_more_half_heads_than_sms_runs_in_waves(oracle):
+    """80 heads = 160 half-head CTAs on 148 SMs: no time split, an ordinary launch whose CTAs run in two waves."""
+    B, T, H = 2, 130, 80
+    D = 256 * H
+    assert uses_sm100(B, T, D, H)
+    inp = synth.make_inputs(B, T, D, H, io="bf16", seed=77, with_state=True, bias_scale=0.5)
+    y, hT, cso = gpu_prefill(inp, h0=inp["h0"], cs=inp["conv_state"])
+    yr, hr, cr = oracle_prefill(oracle, inp, h0=inp["h0"].astype(np.float64), cs=inp["conv_state"].astype(np.float64))
+    assert_close("y", y, yr, "bf16"); assert_close("h_T", hT, hr, "bf16")
+    assert np.array_equal(cso, cr)
+
+
 def test_zero_state_defaults_and_generic_agreement(oracle):
     inp = synth.make_inputs(2, 200, 512, 2, io="bf16", seed=3)
     y, hT, cso = gpu_prefill(inp)

@@ -3,17 +3,18 @@
 // One persistent CTA per SM owns HALF a head (128 channels): its 2 x 128 rows of W_a and W_x stay
 // resident in tensor memory as the A operand of tcgen05.mma for the whole launch.  The CTA walks
 // tiles of 128 tokens:
-//   TMA warp       x rows of the whole head (the gates need all 256 input channels) -> shared memory
-//   conv warps     causal width-4 depthwise conv in fp32 -> bf16 tile U[128 tokens][256 ch] in the
+//   TMA warp       x rows of the whole head (the gates need all 256 input channels) -> shared memory, tiled copies
+//   conv warps     causal width-4 depthwise conv in fp32 -> fp16 tile U[128 tokens][256 ch] in the
 //                  K-major 128B-swizzled layout tcgen05.mma reads as its B operand
-//   MMA warp       Z_a^T = W_a U^T and Z_x^T = W_x U^T: channels on TMEM lanes, time along TMEM columns
+//   MMA warps      Z_a^T = W_a U^T (one warp) and Z_x^T = W_x U^T (another): channels on TMEM lanes, time along
+//                  TMEM columns, one N = 128 instruction per K step
 //   epilogue warps tcgen05.ld (time runs along registers, so the scan needs no shuffles), gates,
-//                  log-space decay, the linear recurrence in fp32, y written straight to HBM
+//                  log-space decay, the linear recurrence in fp32, y through a per-warp tiled store
 // x is read from HBM once per head (the two half-head CTAs share it through L2), y is written once;
 // u, r, i, a never leave the SM.
 //
-// Time is split across CTAs so that every SM has work even for a single long sequence: the S CTAs
-// of a half-head take its 128-token tiles round-robin.  A tile first folds itself to the aggregate
+// Time is split across CTAs so that every SM has work even for a single long sequence: sequences that
+// cannot be dealt out whole go to the S CTAs of a half-head tile by tile, round-robin.  Such a tile first folds itself to the aggregate
 // (prod a_t, h_end from zero state), publishes it, and obtains its incoming state from its own
 // previous tile plus the S-1 aggregates published by the other CTAs (decoupled look-back); only
 // then does it run the real scan and write y.  Waits on other CTAs are bounded and end in

@@ -166,12 +166,13 @@ def test_backward_tensor_core_path(oracle, B, T, H, with_y):
         assert_close("d" + k, to_np(g[k]), gr[k], "bf16")
 
 
-def test_prefill_host_pipelined_chunks_match_device_prefill(oracle):
-    """rglru_prefill_host cuts the batch into chunks of sequences that are copied in, run and copied out concurrently;
-    the result must be the forward of the whole batch."""
+@pytest.mark.parametrize("B,T,H", [(5, 300, 2), (2, 1300, 1), (40, 20, 1)])
+def test_prefill_host_pipelined_chunks_match_device_prefill(oracle, B, T, H):
+    """rglru_prefill_host cuts the batch into chunks of whole sequences (one each, or several when there are more
+    sequences than chunks) that are copied in, run and copied out concurrently; the result must be the forward of the
+    whole batch."""
     import torch
     from paper_2402_19427_b200 import binding
-    B, T, H = 5, 300, 2
     D = 256 * H
     inp = synth.make_inputs(B, T, D, H, io="bf16", seed=77, with_state=True, bias_scale=0.2)
     params = binding.Params.from_numpy(inp["params"], "bf16")

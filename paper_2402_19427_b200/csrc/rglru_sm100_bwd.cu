@@ -331,7 +331,23 @@ __global__ void __launch_bounds__(256) scan_fold_kernel(EwArgs a) {
     const uint32_t sD = (uint32_t)D, sZ = (uint32_t)a.H * 2 * DH;
     const __nv_bfloat16 *p_dy = a.dy + tokb * (size_t)sD + d;
     const __half *p_z = a.z + tokb * sZ + (size_t)h * 2 * DH + n;
-    for (int tb = t1 - 8; tb >= t0; tb -= 8) {
+    int tb = t1 - 8;
+    // the kernel waits on memory: 16-token rounds keep 32 loads per thread in flight at 60 registers (32-token rounds
+    // need 128 and measured the same); the pointers sit 8 tokens below the top of the round
+    for (; tb - 8 >= t0; tb -= 16) {
+        float dyv[16], zav[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) { dyv[k] = bf2f(p_dy[(k - 8) * (int)sD]); zav[k] = __half2float(p_z[(k - 8) * (int)sZ]); }
+#pragma unroll
+        for (int k = 15; k >= 0; --k) {
+            const float at = __expf(-s * sigmoid_fast(zav[k] + ba));
+            const float g = dyv[k] + carry;
+            carry = at * g;
+            Q *= at;
+        }
+        p_dy -= 16 * (size_t)sD; p_z -= 16 * (size_t)sZ;
+    }
+    for (; tb >= t0; tb -= 8) {
         float dyv[8], zav[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) { dyv[k] = bf2f(p_dy[k * sD]); zav[k] = __half2float(p_z[k * sZ]); }

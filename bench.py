@@ -267,7 +267,9 @@ def run_ours(args):
     roof.update({"peaks": peak_kind, "kernel": "rglru prefill (dominant kernel of the step)",
                  "launch_us": launch_s * 1e6, "hbm_gbs_achieved": nbytes / launch_s / 1e9,
                  "hbm_frac": nbytes / launch_s / 1e9 / peaks["hbm_gbs"], "tensor_tflops_achieved": flops / launch_s / 1e12,
-                 "tensor_frac": flops / launch_s / 1e12 / peaks["bf16_tflops"], "algorithmic_bytes": nbytes, "gate_flops": flops})
+                 "tensor_frac": flops / launch_s / 1e12 / peaks["bf16_tflops"], "algorithmic_bytes": nbytes, "gate_flops": flops,
+                 # for context only: the same work against the data-sheet figures (8 TB/s, 2.25 PFLOP/s dense bf16)
+                 "frac_of_nominal": max(nbytes / 8.0e12, flops / 2.25e15) / launch_s})
 
     extra = {}
     if rank == 0 and not args.no_extras:

@@ -299,7 +299,6 @@ __global__ void __launch_bounds__(256) conv_forward_kernel(EwArgs a) {
     int t = t0;
     for (; t + 16 <= t1; t += 16) {   // sixteen tokens: the channel-major store fills whole 32-byte sectors
         float xa[8], xb[8];
-#pragma unroll
         const __nv_bfloat16 *px = a.x + ((size_t)b * T + t) * D + d;
         __half *pu = a.u + ((size_t)b * T + t) * D + d;
 #pragma unroll

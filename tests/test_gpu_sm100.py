@@ -166,6 +166,28 @@ def test_backward_tensor_core_path(oracle, B, T, H, with_y):
         assert_close("d" + k, to_np(g[k]), gr[k], "bf16")
 
 
+def test_backward_is_run_to_run_identical():
+    """Every parameter gradient is a sum over B*T tokens taken in a fixed order (per-chunk partial sums, then one reduction
+    over the chunks; no atomics), so two runs on the same inputs agree bit for bit; so do dx and the prefill outputs."""
+    import torch
+    from paper_2402_19427_b200 import binding
+    B, T, H = 3, 520, 2
+    D = 256 * H
+    inp = synth.make_inputs(B, T, D, H, io="bf16", seed=31, with_dy=True)
+    params = binding.Params.from_numpy(inp["params"], "bf16")
+    x = to_dev(inp["x"], "bf16"); dy = to_dev(inp["dy"], "bf16")
+    shape = binding.make_shape(B, T, D, H, torch.bfloat16)
+    ws = binding.alloc_workspace(shape, binding.OP_BACKWARD, x.device)
+    runs = []
+    for _ in range(2):
+        y = binding.prefill(x, params)[0]
+        g = binding.backward(x, params, dy, y=y, workspace=ws)
+        torch.cuda.synchronize()
+        runs.append({k: to_np(v).copy() for k, v in g.items()} | {"y": to_np(y).copy()})
+    for k in runs[0]:
+        assert np.array_equal(runs[0][k], runs[1][k]), k
+
+
 @pytest.mark.parametrize("B,T,H", [(5, 300, 2), (2, 1300, 1), (40, 20, 1)])
 def test_prefill_host_pipelined_chunks_match_device_prefill(oracle, B, T, H):
     """rglru_prefill_host cuts the batch into chunks of whole sequences (one each, or several when there are more

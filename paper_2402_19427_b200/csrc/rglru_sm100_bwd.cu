@@ -366,11 +366,22 @@ __global__ void __launch_bounds__(256) scan_fold_kernel(EwArgs a) {
 __global__ void __launch_bounds__(256) scan_carry_kernel(EwArgs a) {
     const int d = blockIdx.x * 256 + threadIdx.x, b = blockIdx.y;
     float X = 0.0f;
-    for (int c = a.nchunk - 1; c >= 0; --c) {
-        const size_t i = ((size_t)b * a.nchunk + c) * a.D + d;
-        a.xin[i] = X;
-        const float2 f = a.fold[i];
-        X = fmaf(f.x, X, f.y);
+    // sixteen folds are requested at once (loads interleaved with the stores below would go out one at a time)
+    for (int c1 = a.nchunk; c1 > 0; c1 -= 16) {
+        float2 f[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const int c = c1 - 1 - j;
+            f[j] = c >= 0 ? a.fold[((size_t)b * a.nchunk + c) * a.D + d] : make_float2(1.0f, 0.0f);
+        }
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const int c = c1 - 1 - j;
+            if (c >= 0) {
+                a.xin[((size_t)b * a.nchunk + c) * a.D + d] = X;
+                X = fmaf(f[j].x, X, f[j].y);
+            }
+        }
     }
 }
 

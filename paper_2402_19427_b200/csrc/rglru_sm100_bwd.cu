@@ -255,14 +255,25 @@ struct EwArgs {
 };
 
 // fp16 copies of the gate weights: W16[g][h][o][n] = W_g[h][o][n] and WT[h][n][g*256 + o] = W_g[h][o][n]
+// One block per 32 x 32 tile of one (gate, head) matrix; the transposed copy goes through shared memory so that both
+// copies are written with consecutive threads on consecutive addresses.  grid (8, 8, 2 H), block (32, 8)
 __global__ void convert_w_kernel(const __nv_bfloat16 *Wa, const __nv_bfloat16 *Wx, __half *W16, __half *WT, int H) {
-    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;   // over [g][h][o][n]
-    if (i >= (size_t)H * 2 * DH * DH) return;
-    const int n = (int)(i % DH), o = (int)((i / DH) % DH), h = (int)((i / (DH * DH)) % H), g = (int)(i / ((size_t)H * DH * DH));
-    const float v = __bfloat162float((g ? Wx : Wa)[((size_t)h * DH + o) * DH + n]);
-    const __half hv = __float2half_rn(fminf(fmaxf(v, -65504.0f), 65504.0f));
-    W16[i] = hv;
-    WT[((size_t)h * DH + n) * (2 * DH) + g * DH + o] = hv;
+    __shared__ __half tile[32][33];
+    const int g = blockIdx.z / H, h = blockIdx.z % H;
+    const int o0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
+    const __nv_bfloat16 *W = (g ? Wx : Wa) + (size_t)h * DH * DH;
+    __half *W16m = W16 + ((size_t)g * H + h) * DH * DH;
+#pragma unroll
+    for (int r = threadIdx.y; r < 32; r += 8) {
+        const float v = __bfloat162float(W[(size_t)(o0 + r) * DH + n0 + threadIdx.x]);
+        const __half hv = __float2half_rn(fminf(fmaxf(v, -65504.0f), 65504.0f));
+        W16m[(size_t)(o0 + r) * DH + n0 + threadIdx.x] = hv;
+        tile[r][threadIdx.x] = hv;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = threadIdx.y; r < 32; r += 8)
+        WT[((size_t)h * DH + n0 + r) * (2 * DH) + g * DH + o0 + threadIdx.x] = tile[threadIdx.x][r];
 }
 
 __device__ __forceinline__ __half to_half_sat(float v) { return __float2half_rn(fminf(fmaxf(v, -65504.0f), 65504.0f)); }
@@ -626,8 +637,7 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
     a.fold = (float2 *)(ws + L.off_fold); a.xin = (float *)(ws + L.off_xin); a.part_vec = (float *)(ws + L.off_pvec);
 
     // 1. W^T for the du contraction, conv output
-    const size_t nW = (size_t)H * 2 * DH * DH;
-    convert_w_kernel<<<(unsigned)((nW + 255) / 256), 256, 0, st>>>((const __nv_bfloat16 *)q.W_a, (const __nv_bfloat16 *)q.W_x, W16, WT, H);
+    convert_w_kernel<<<dim3(DH / 32, DH / 32, 2 * H), dim3(32, 8), 0, st>>>((const __nv_bfloat16 *)q.W_a, (const __nv_bfloat16 *)q.W_x, W16, WT, H);
     const dim3 grid_ew(D / 256, L.nchunk, B);
     conv_forward_kernel<<<grid_ew, 256, 0, st>>>(a);
 

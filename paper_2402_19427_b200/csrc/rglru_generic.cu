@@ -384,6 +384,13 @@ __global__ void reduce_partials3_kernel(const float *in, int nparts, size_t stri
     if (out == nullptr) return;
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     int p = 0;
+    for (; p + 16 <= nparts; p += 16) {   // sixteen loads in flight, still four running sums in a fixed order
+        float v[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = in[(size_t)(p + j) * stride + i];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) acc[j & 3] += v[j];
+    }
     for (; p + 4 <= nparts; p += 4) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[j] += in[(size_t)(p + j) * stride + i];

@@ -1,30 +1,33 @@
 // sm_100a fused prefill for the RG-LRU temporal core (bf16 io, head width 256).
 //
-// One persistent CTA per SM owns HALF a head (128 channels): its 2 x 128 rows of W_a and W_x stay
-// resident in tensor memory as the A operand of tcgen05.mma for the whole launch.  The CTA walks
-// tiles of 128 tokens:
-//   TMA warp       x rows of the whole head (the gates need all 256 input channels) -> shared memory, tiled copies
-//   conv warps     causal width-4 depthwise conv in fp32 -> fp16 tile U[128 tokens][256 ch] in the
-//                  K-major 128B-swizzled layout tcgen05.mma reads as its B operand
-//   MMA warps      Z_a^T = W_a U^T (one warp) and Z_x^T = W_x U^T (another): channels on TMEM lanes, time along
-//                  TMEM columns, one N = 128 instruction per K step
-//   epilogue warps tcgen05.ld (time runs along registers, so the scan needs no shuffles), gates,
-//                  log-space decay, the linear recurrence in fp32, y through a per-warp tiled store
-// x is read from HBM once per head (the two half-head CTAs share it through L2), y is written once;
-// u, r, i, a never leave the SM.
+// A head is owned by a pair of CTAs (a cluster of two, one CTA per SM).  CTA r of the pair keeps rows
+// [128 r, 128 r + 128) of W_a and W_x resident in its tensor memory as the A operand of the two-CTA form of
+// tcgen05.mma (M = 256 over the pair) for the whole launch.  The pair walks tiles of 64 tokens; CTA r convolves tokens
+// [32 r, 32 r + 32) of a tile for all 256 channels of the head, so the Conv1D runs once per element:
+//   loader warp    35 token rows (32 + 3 of history) of the head's x -> shared memory, one tiled TMA copy per tile
+//   conv warps     causal width-4 depthwise conv in fp32 -> fp16 tile U[32 tokens][256 ch] in the K-major
+//                  128B-swizzled layout tcgen05.mma reads as this CTA's half of the B operand
+//   MMA warps      (leader CTA only) Z_a^T = W_a U^T and Z_x^T = W_x U^T, N = 64 tokens, K = 256: channels on TMEM
+//                  lanes, time along TMEM columns, two accumulator buffers used alternately
+//   gate warps     tcgen05.ld a batch of (z_a, z_x), u from the U tile of the CTA that convolved the token (its own
+//                  or the peer's through distributed shared memory), gates, log-space decay, input scale, and
+//                  (a_t, v_t) written back over (z_a, z_x) with tcgen05.st; they hold no state and never wait for it
+//   scan warps     pull a tile's (a_t, v_t) into registers, free the accumulator buffer, run the linear recurrence
+//                  h_t = a_t h_{t-1} + v_t in fp32 with the exact incoming state, y through a per-warp tiled store
+// x is read from HBM once, y written once; u, r, i, a never leave the pair.
 //
-// Time is split across CTAs so that every SM has work even for a single long sequence: sequences that
-// cannot be dealt out whole go to the S CTAs of a half-head tile by tile, round-robin.  Such a tile first folds itself to the aggregate
-// (prod a_t, h_end from zero state), publishes it, and obtains its incoming state from its own
-// previous tile plus the S-1 aggregates published by the other CTAs (decoupled look-back); only
-// then does it run the real scan and write y.  Waits on other CTAs are bounded and end in
-// RGLRU_ERR_TIMEOUT; the launch is cooperative so that all CTAs are co-resident.
+// Time is split across pairs so that every SM has work even for a single long sequence: sequences that cannot be
+// dealt out whole go to the S pairs of a head tile by tile, round-robin.  The scan warp folds such a tile to the
+// aggregate (prod a_t, h_end from zero state), publishes it, and obtains its incoming state from its own previous
+// tile plus the S-1 aggregates published by the other pairs (decoupled look-back); only then does it run the scan.
+// Waits are bounded and end in RGLRU_ERR_TIMEOUT; the launch is cooperative so that all CTAs are co-resident.
 #include <cooperative_groups.h>
 #include <cuda.h>
 #include <cuda_bf16.h>
 
 #include <atomic>
 #include <chrono>
+#include <mutex>
 #include <type_traits>
 
 #include "rglru_internal.h"
@@ -36,39 +39,37 @@ namespace {
 
 constexpr int DH = 256;            // head width handled by this kernel
 constexpr int CH = 128;            // channels per CTA (half a head)
-constexpr int TILE_N = 128;        // tokens per MMA tile
-constexpr int SLAB = 32;           // tokens per TMA slab
-constexpr int SLAB_ROWS = SLAB + 3;
-constexpr int XS = 3;              // x slab ring depth
-constexpr int US = 2;              // U tile stages
-constexpr int NUM_THREADS = 512;
-constexpr int EPI_TOK = 64;        // tokens per epilogue warp
-constexpr int MAX_S = 8;           // at most this many CTAs share one half-head's time axis
-constexpr uint32_t U_STAGE_BYTES = TILE_N * DH * 2;       // 65536
-constexpr uint32_t U_KBLOCK_BYTES = TILE_N * 128;          // 16384: one 64-channel K block
+constexpr int TILE = 64;           // tokens per MMA tile of a pair
+constexpr int HALF = 32;           // tokens of a tile one CTA convolves (one TMA slab)
+constexpr int SLAB_ROWS = HALF + 3;
+constexpr int XS = 4;              // x slab ring depth
+constexpr int US = 6;              // U tile stages
+constexpr int NUM_THREADS = 640;
+constexpr int MAX_S = 8;           // at most this many pairs share one head's time axis
+constexpr uint32_t U_STAGE_BYTES = HALF * DH * 2;          // 16384
+constexpr uint32_t U_KBLOCK_BYTES = HALF * 128;            // 4096: one 64-channel K block
 constexpr uint32_t X_ROW_BYTES = DH * 2;                   // 512
 constexpr uint32_t X_SLAB_BYTES = SLAB_ROWS * X_ROW_BYTES; // 17920
 constexpr uint32_t SMEM_U = 0;
 constexpr uint32_t SMEM_X = SMEM_U + US * U_STAGE_BYTES;
-constexpr uint32_t Y_WARP_BYTES = EPI_TOK * 32 * 2;        // 4096: one epilogue warp's 64 tokens x 32 channels
-constexpr uint32_t SMEM_Y = SMEM_X + XS * X_SLAB_BYTES;    // bf16 y_s[8 warps][64][32], staged for tiled stores
-constexpr uint32_t SMEM_AGG = SMEM_Y + 8 * Y_WARP_BYTES;   // float2 agg_s[2 tile parity][2 halves][4][32]
-constexpr uint32_t SMEM_BAR = SMEM_AGG + 2 * 2 * 4 * 32 * 8;
+constexpr uint32_t Y_BUF_BYTES = TILE * 32 * 2;            // 4096: one scan warp's 64 tokens x 32 channels
+constexpr uint32_t SMEM_Y = SMEM_X + XS * X_SLAB_BYTES;    // bf16 y_s[4 warps][2 buffers][64][32], staged for tiled stores
+constexpr uint32_t SMEM_BAR = SMEM_Y + 4 * 2 * Y_BUF_BYTES;
 constexpr int NUM_BARS = 2 * XS + 2 * US + 4 + 8 + 1;
 constexpr uint32_t SMEM_MISC = SMEM_BAR + NUM_BARS * 8;    // tmem base, abort flag
 constexpr uint32_t SMEM_TOTAL = SMEM_MISC + 16;
 constexpr uint32_t SMEM_ALLOC = SMEM_TOTAL + 1024;         // slack for 1024-byte alignment
 
-// TMEM columns
-constexpr uint32_t TM_ACC_A = 0, TM_ACC_X = 128, TM_W_A = 256, TM_W_X = 384;
-
+// TMEM columns: accumulator buffer bf holds z_a (later a_t) in [128 bf, 128 bf + 64) and z_x (later v_t) in the next 64
+constexpr uint32_t TM_W_A = 256, TM_W_X = 384;
+__host__ __device__ constexpr uint32_t tm_acc(int bf, int gate) { return (uint32_t)(bf * 128 + gate * 64); }
 
 struct Sm100Args {
-    // x as [B][T][D] with a box of SLAB_ROWS token rows x one head; y with a box of EPI_TOK rows x 32 channels
+    // x as [B][T][D] with a box of SLAB_ROWS token rows x one head; y with a box of TILE rows x 32 channels
     alignas(64) CUtensorMap tm_x;
     alignas(64) CUtensorMap tm_y;
     FwdArgs f;
-    int S;             // CTAs per half-head (time split factor)
+    int S;             // pairs per head (time split factor)
     int tps;           // tiles per sequence
     int tiles_total;   // B * tps
     uint32_t tag;      // validity tag of this call's aggregate records
@@ -78,12 +79,7 @@ struct Sm100Args {
 
 using namespace ptx;
 
-__device__ __forceinline__ void record_timeout(uint32_t *status, volatile int *abort_flag) {
-    *abort_flag = 1;
-    atomicExch(status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
-}
-
-__global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __grid_constant__ Sm100Args p) {
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __grid_constant__ Sm100Args p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
@@ -92,31 +88,41 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
     // barrier indices
     auto BAR_XFULL = [&](int s) { return bar0 + 8u * s; };
     auto BAR_XEMPTY = [&](int s) { return bar0 + 8u * (XS + s); };
-    auto BAR_UFULL = [&](int s) { return bar0 + 8u * (2 * XS + s); };
+    auto BAR_UFULL = [&](int s) { return bar0 + 8u * (2 * XS + s); };              // used in the leader CTA only
     auto BAR_UEMPTY = [&](int s) { return bar0 + 8u * (2 * XS + US + s); };
-    auto BAR_ACCFULL = [&](int k) { return bar0 + 8u * (2 * XS + 2 * US + k); };       // accumulators of token half k
-    auto BAR_ACCEMPTY = [&](int k) { return bar0 + 8u * (2 * XS + 2 * US + 2 + k); };
-    auto BAR_AGG = [&](int q, int k) { return bar0 + 8u * (2 * XS + 2 * US + 4 + q * 2 + k); };  // fold of half k, channel group q
-    const uint32_t BAR_WREADY = bar0 + 8u * (2 * XS + 2 * US + 12);   // gate weights are in tensor memory
+    auto BAR_ACCFULL = [&](int bf) { return bar0 + 8u * (2 * XS + 2 * US + bf); };
+    auto BAR_ACCEMPTY = [&](int bf) { return bar0 + 8u * (2 * XS + 2 * US + 2 + bf); };   // leader CTA only
+    auto BAR_GDONE = [&](int bf, int q) { return bar0 + 8u * (2 * XS + 2 * US + 4 + bf * 4 + q); };
+    const uint32_t BAR_WREADY = bar0 + 8u * (2 * XS + 2 * US + 12);               // leader CTA only: both CTAs' weights are in tensor memory
     uint32_t *tmem_base_s = (uint32_t *)(smem + SMEM_MISC);
     volatile int *abort_flag = (volatile int *)(smem + SMEM_MISC + 4);
-    float2 *agg_s = (float2 *)(smem + SMEM_AGG);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const FwdArgs &f = p.f;
     const int T = f.T, D = f.D, S = p.S;
-    const int group = blockIdx.x / S, kcta = blockIdx.x % S;  // group = head * 2 + half
-    const int head = group >> 1, half = group & 1;
-    // Work of this CTA.  Sequences are dealt out whole where that keeps the S CTAs of the half-head balanced: CTA kcta
+    // CTA `rank` of the pair owns output channels [128 rank, 128 rank + 128) of the head and convolves tokens
+    // [32 rank, 32 rank + 32) of every tile for both CTAs.  Rank 0 is the leader: it issues the MMAs of the pair.
+    const uint32_t rank = cluster_ctarank();
+    const int pair = blockIdx.x >> 1;
+    const int head = pair / S, kcta = pair % S;
+    const int group = head * 2 + (int)rank;   // index of this half-head's carry records
+    const uint32_t peer_abort = map_to_cta(base + SMEM_MISC + 4, rank ^ 1u);
+    auto record_timeout = [&]() {
+        *abort_flag = 1;
+        st_cluster_u32(peer_abort, 1u);   // the peer would otherwise run into its own limit waiting for this CTA
+        atomicExch(f.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
+    };
+    // Work of this pair.  Sequences are dealt out whole where that keeps the S pairs of the head balanced: pair kcta
     // gets sequences kcta, kcta + S, ... of the first (B / S) * S ones and walks each from start to end, so a tile's
-    // incoming state is simply the state the CTA itself reached ("local" tiles: no record, no look-back).  The B % S
-    // sequences left over are split in time, tile g of them going to CTA g % S ("shared" tiles, decoupled look-back).
-    // Shared tiles come first, so that the S CTAs pass through them in step.
+    // incoming state is simply the state the pair itself reached ("local" tiles: no record, no look-back).  The B % S
+    // sequences left over are split in time, tile g of them going to pair g % S ("shared" tiles, decoupled look-back).
+    // Shared tiles come first, so that the S pairs pass through them in step.
     const int B_whole = (f.B / S) * S, shared_tiles = (f.B - B_whole) * p.tps;
     const int n_shared = kcta < shared_tiles ? (shared_tiles - kcta + S - 1) / S : 0;
     const int n_my_tiles = n_shared + (B_whole / S) * p.tps;
-    // The CTA's tiles in order: tile_first gives (sequence b, tile ti within it) of tile 0, tile_next steps from tile
-    // `it` to tile `it + 1`; tile `it` is a shared one when it < n_shared.
+    // The pair's tiles in order: tile_first gives (sequence b, tile ti within it) of tile 0, tile_next steps from tile
+    // `it` to tile `it + 1`; tile `it` is a shared one when it < n_shared.  Tile `it` uses U stage it % US and
+    // accumulator buffer it & 1 in both CTAs.
     auto tile_first = [&](int &b, int &ti) {
         if (n_shared > 0) { b = B_whole + kcta / p.tps; ti = kcta % p.tps; } else { b = kcta; ti = 0; }
     };
@@ -134,16 +140,22 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
 
     if (tid == 0) {
         for (int s = 0; s < XS; ++s) { mbar_init(BAR_XFULL(s), 1); mbar_init(BAR_XEMPTY(s), 4); }
-        for (int s = 0; s < US; ++s) { mbar_init(BAR_UFULL(s), 4); mbar_init(BAR_UEMPTY(s), 10); }
-        mbar_init(BAR_ACCFULL(0), 2); mbar_init(BAR_ACCEMPTY(0), 8);
-        for (int q = 0; q < 4; ++q) { mbar_init(BAR_AGG(q, 0), 1); mbar_init(BAR_AGG(q, 1), 1); }
-        mbar_init(BAR_WREADY, 8);
+        // U stage full: the four conv warps of both CTAs (counted in the leader).  Free again: both MMA issuers' commits plus
+        // the four gate warps of each CTA that read u from this CTA's stage.
+        for (int s = 0; s < US; ++s) { mbar_init(BAR_UFULL(s), 8); mbar_init(BAR_UEMPTY(s), 10); }
+        for (int bf = 0; bf < 2; ++bf) {
+            mbar_init(BAR_ACCFULL(bf), 2);    // one commit per MMA issuer
+            mbar_init(BAR_ACCEMPTY(bf), 8);   // the four scan warps of both CTAs
+            for (int q = 0; q < 4; ++q) mbar_init(BAR_GDONE(bf, q), 2);
+        }
+        mbar_init(BAR_WREADY, 16);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 5) { tmem_alloc(smem_u32(tmem_base_s), 512); tmem_relinquish(); }
+    if (warp == 5) { tmem_alloc2(smem_u32(tmem_base_s), 512); tmem_relinquish2(); }
     tc_fence_before();
-    __syncthreads();
+    cluster_arrive();   // the peer's barriers must exist before anything arrives on them
+    cluster_wait();
     tc_fence_after();
     const uint32_t tmem = *tmem_base_s;
 
@@ -153,10 +165,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
     // Eq. 4 directly), and both operands of one MMA must have one type: the bf16 weights are converted to
     // fp16 here, which is exact for every weight of magnitude within [2^-14, 65504] and rounds tinier ones
     // to a multiple of 2^-24.
-    if (warp >= 8) {
+    if (warp >= 8 && warp < 16) {
         const int q = warp & 3, g = (warp - 8) >> 2;  // g = 0: W_a, 1: W_x
         const __nv_bfloat16 *W = (const __nv_bfloat16 *)(g ? f.W_x : f.W_a);
-        const uint4 *row = (const uint4 *)(W + ((size_t)head * DH + half * CH + q * 32 + lane) * DH);
+        const uint4 *row = (const uint4 *)(W + ((size_t)head * DH + rank * CH + q * 32 + lane) * DH);
         const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (g ? TM_W_X : TM_W_A);
         auto cvt2 = [](uint32_t w) { return pack_f16_sat(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u)); };
 #pragma unroll 4
@@ -170,11 +182,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         // only the MMA issuers wait for the weights: loads and the conv of the first tiles run meanwhile
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(BAR_WREADY);
+        if (lane == 0) mbar_arrive_at(BAR_WREADY, 0);
     }
 
-    // Register budget per warpgroup (the four warps of a group execute the same setmaxnreg):
-    // conv producers 72, loader / MMA issuer / idle 40, epilogue 200.
+    // Register budget per warpgroup (the four warps of a group execute the same setmaxnreg; the increases draw on
+    // what the decreases release: 128 (96-72) + 128 (96-40) = 256 (104-96) + 128 (160-96)):
+    // conv producers 72, loader / MMA issuers / idle 40, gate warps 104, scan warps 160.
     if (warp < 4) {
         // ================================================================ conv producers
         reg_dec<72>();
@@ -193,174 +206,133 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
             const float *bp = f.conv_b + head * DH + hc;
             b01 = pack2(bp[0], bp[1]); b23 = pack2(bp[2], bp[3]);
         } else { b01 = pack2(0.f, 0.f); b23 = b01; }
-        const uint32_t x_thread_off = (uint32_t)hc * 2;
-        const uint32_t u_chunk = (uint32_t)(l16 >> 1), u_half = (uint32_t)(l16 & 1) * 8;
-        // Token tt of a tile is stored in row perm(tt) of the U tile (= accumulator column perm(tt)):
-        // within each group of 64 tokens, tokens j and j + 32 sit in adjacent rows 2j and 2j + 1, so that
-        // the epilogue finds them in one register pair and can run the two halves of its 64 tokens as
-        // the two lanes of packed fp32x2 arithmetic.
-        int slab_n = 0;
+        // this thread's 16 tokens are rows 16 tg .. 16 tg + 15 of the slab (plus three rows of history) and of the U tile;
+        // U row r keeps its 16-byte chunk c at position c ^ (r & 7) (128-byte swizzle)
+        const uint32_t x_thread_off = (uint32_t)hc * 2 + (uint32_t)(tg * 16) * X_ROW_BYTES;
+        const uint32_t u_chunk = (uint32_t)(l16 >> 1);
+        const uint32_t u_thread_off = SMEM_U + pblk * U_KBLOCK_BYTES + (uint32_t)(l16 & 1) * 8 + (uint32_t)(tg * 16) * 128u;
+        uint32_t sw[8];
+#pragma unroll
+        for (int m = 0; m < 8; ++m) sw[m] = u_thread_off + ((u_chunk ^ (uint32_t)m) << 4);
         bool ok = true;
-        int b, ti;
-        tile_first(b, ti);
-        for (int it = 0; it < n_my_tiles && ok; tile_next(it, b, ti), ++it) {
-            const int t0 = ti * TILE_N;
-            const int st = it % US;
-            ok = warp_wait(BAR_UEMPTY(st), ((it / US) & 1) ^ 1, spin, abort_flag);
+        for (int it = 0; it < n_my_tiles; ++it) {
+            const int st = it % US, slot = it % XS;
+            ok = warp_wait_cl(BAR_UEMPTY(st), ((it / US) & 1) ^ 1, spin, abort_flag);
             if (!ok) break;
-            const uint32_t u_base = SMEM_U + st * U_STAGE_BYTES + pblk * U_KBLOCK_BYTES + u_half;  // offset from smem
-            const int nslab = min(TILE_N / SLAB, (T - t0 + SLAB - 1) / SLAB);
-            for (int s = 0; s < nslab; ++s, ++slab_n) {
-                const int slot = slab_n % XS;
-                ok = warp_wait(BAR_XFULL(slot), (slab_n / XS) & 1, spin, abort_flag);
-                if (!ok) break;
-                const int ts0 = t0 + s * SLAB;
-                const bool zero_halo = (ts0 == 0) && (f.cs_in == nullptr);
-                const int nvalid = min(SLAB, T - ts0) - tg * 16;  // tokens of this thread's group that exist
-                const uint8_t *xs = smem + SMEM_X + slot * X_SLAB_BYTES + x_thread_off + (uint32_t)(tg * 16) * X_ROW_BYTES;
-                auto load_row = [&](int r, f32x2 &v01, f32x2 &v23) {   // r: row relative to this thread's first halo row
-                    const uint2 w = *(const uint2 *)(xs + (uint32_t)r * X_ROW_BYTES);
-                    v01 = pack2(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xFFFF0000u));
-                    v23 = pack2(__uint_as_float(w.y << 16), __uint_as_float(w.y & 0xFFFF0000u));
-                };
-                // row of token i of this thread: rowbase + 2 i; its 16-byte chunk is swizzled by (row & 7) = (p + 2 i) & 7
-                const uint32_t pbit = (uint32_t)(s & 1);
-                const uint32_t row_addr = u_base + (uint32_t)((s >> 1) * 64 + (s & 1) + 32 * tg) * 128u;
-                uint32_t sw[4];
+            ok = warp_wait(BAR_XFULL(slot), (it / XS) & 1, spin, abort_flag);
+            if (!ok) break;
+            const uint8_t *xs = smem + SMEM_X + slot * X_SLAB_BYTES + x_thread_off;
+            uint8_t *us = smem + st * U_STAGE_BYTES;
+            auto load_row = [&](int r, f32x2 &v01, f32x2 &v23) {   // r: row relative to this thread's first history row
+                const uint2 w = *(const uint2 *)(xs + (uint32_t)r * X_ROW_BYTES);
+                v01 = pack2(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xFFFF0000u));
+                v23 = pack2(__uint_as_float(w.y << 16), __uint_as_float(w.y & 0xFFFF0000u));
+            };
+            // Rows before the sequence start and at or beyond its end were filled with zeros by the copy, so all 16 tokens
+            // are convolved unconditionally; tokens that do not exist produce rows nobody uses.
+            // Four tokens at a time, tap by tap, so that eight independent FMA chains are in flight.
+            f32x2 h01[3], h23[3];   // x_{t-3}, x_{t-2}, x_{t-1}
 #pragma unroll
-                for (int m = 0; m < 4; ++m) sw[m] = row_addr + ((u_chunk ^ ((pbit + 2u * m) & 7u)) << 4);
-                if (nvalid > 0) {
-                    f32x2 a01, a23, b01x, b23x, c01, c23;  // x_{t-3}, x_{t-2}, x_{t-1}
-                    load_row(0, a01, a23); load_row(1, b01x, b23x); load_row(2, c01, c23);
-                    if (zero_halo && tg == 0) { a01 = a23 = b01x = b23x = c01 = c23 = pack2(0.f, 0.f); }
-                    if (nvalid >= 16) {
-                        // four tokens at a time, tap by tap, so that eight independent FMA chains are in flight
-                        f32x2 h01[3] = {a01, b01x, c01}, h23[3] = {a23, b23x, c23};
+            for (int k = 0; k < 3; ++k) load_row(k, h01[k], h23[k]);
 #pragma unroll
-                        for (int i0 = 0; i0 < 16; i0 += 4) {
-                            f32x2 r01[7], r23[7];   // rows t-3 .. t+3 of the batch
+            for (int i0 = 0; i0 < 16; i0 += 4) {
+                f32x2 r01[7], r23[7];   // rows t-3 .. t+3 of the batch
 #pragma unroll
-                            for (int k = 0; k < 3; ++k) { r01[k] = h01[k]; r23[k] = h23[k]; }
+                for (int k = 0; k < 3; ++k) { r01[k] = h01[k]; r23[k] = h23[k]; }
 #pragma unroll
-                            for (int k = 0; k < 4; ++k) load_row(3 + i0 + k, r01[3 + k], r23[3 + k]);
-                            f32x2 u01[4], u23[4];
+                for (int k = 0; k < 4; ++k) load_row(3 + i0 + k, r01[3 + k], r23[3 + k]);
+                f32x2 u01[4], u23[4];
 #pragma unroll
-                            for (int k = 0; k < 4; ++k) { u01[k] = fma2(w01[0], r01[3 + k], b01); u23[k] = fma2(w23[0], r23[3 + k], b23); }
+                for (int k = 0; k < 4; ++k) { u01[k] = fma2(w01[0], r01[3 + k], b01); u23[k] = fma2(w23[0], r23[3 + k], b23); }
 #pragma unroll
-                            for (int j = 1; j < 4; ++j) {
+                for (int j = 1; j < 4; ++j) {
 #pragma unroll
-                                for (int k = 0; k < 4; ++k) { u01[k] = fma2(w01[j], r01[3 + k - j], u01[k]); u23[k] = fma2(w23[j], r23[3 + k - j], u23[k]); }
-                            }
-#pragma unroll
-                            for (int k = 0; k < 4; ++k)
-                                *(uint2 *)(smem + sw[(i0 + k) & 3] + (uint32_t)(i0 + k) * 256u) =
-                                    make_uint2(pack_f16_sat(lo2(u01[k]), hi2(u01[k])), pack_f16_sat(lo2(u23[k]), hi2(u23[k])));
-#pragma unroll
-                            for (int k = 0; k < 3; ++k) { h01[k] = r01[4 + k]; h23[k] = r23[4 + k]; }
-                        }
-                    } else {
-                        for (int i = 0; i < nvalid; ++i) {
-                            f32x2 d01, d23;
-                            load_row(3 + i, d01, d23);
-                            f32x2 u01 = fma2(w01[0], d01, b01), u23 = fma2(w23[0], d23, b23);
-                            u01 = fma2(w01[1], c01, u01); u23 = fma2(w23[1], c23, u23);
-                            u01 = fma2(w01[2], b01x, u01); u23 = fma2(w23[2], b23x, u23);
-                            u01 = fma2(w01[3], a01, u01); u23 = fma2(w23[3], a23, u23);
-                            const uint32_t addr = row_addr + ((u_chunk ^ ((pbit + 2u * (uint32_t)i) & 7u)) << 4) + (uint32_t)i * 256u;
-                            *(uint2 *)(smem + addr) = make_uint2(pack_f16_sat(lo2(u01), hi2(u01)), pack_f16_sat(lo2(u23), hi2(u23)));
-                            a01 = b01x; a23 = b23x; b01x = c01; b23x = c23; c01 = d01; c23 = d23;
-                        }
-                    }
+                    for (int k = 0; k < 4; ++k) { u01[k] = fma2(w01[j], r01[3 + k - j], u01[k]); u23[k] = fma2(w23[j], r23[3 + k - j], u23[k]); }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(BAR_XEMPTY(slot));
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    *(uint2 *)(us + sw[(i0 + k) & 7] + (uint32_t)(i0 + k) * 128u) =
+                        make_uint2(pack_f16_sat(lo2(u01[k]), hi2(u01[k])), pack_f16_sat(lo2(u23[k]), hi2(u23[k])));
+#pragma unroll
+                for (int k = 0; k < 3; ++k) { h01[k] = r01[4 + k]; h23[k] = r23[4 + k]; }
             }
-            if (!ok) break;
             fence_async_smem();  // make the generic-proxy writes of U visible to the tensor core
             __syncwarp();
-            if (lane == 0) mbar_arrive(BAR_UFULL(st));
+            if (lane == 0) { mbar_arrive(BAR_XEMPTY(slot)); mbar_arrive_at(BAR_UFULL(st), 0); }
         }
-        if (!ok && lane == 0) record_timeout(f.status, abort_flag);
+        if (!ok && lane == 0) record_timeout();
     } else if (warp < 8) {
       reg_dec<40>();
       if (warp == 4) {
         // ================================================================ TMA loader
         const __nv_bfloat16 *x = (const __nv_bfloat16 *)f.x;
         const __nv_bfloat16 *cs_in = (const __nv_bfloat16 *)f.cs_in;
-        int slab_n = 0;
         bool ok = true;
         int b, ti;
         tile_first(b, ti);
-        for (int it = 0; it < n_my_tiles && ok; tile_next(it, b, ti), ++it) {
-            const int t0 = ti * TILE_N;
-            const int nslab = min(TILE_N / SLAB, (T - t0 + SLAB - 1) / SLAB);
-            for (int s = 0; s < nslab; ++s, ++slab_n) {
-                const int slot = slab_n % XS;
-                ok = warp_wait(BAR_XEMPTY(slot), ((slab_n / XS) & 1) ^ 1, spin, abort_flag);
-                if (!ok) break;
-                const int ts0 = t0 + s * SLAB;
-                const uint32_t dst = base + SMEM_X + slot * X_SLAB_BYTES;
-                if (ts0 == 0 && cs_in != nullptr) {
-                    // first slab of a sequence with an incoming conv state: the three halo rows come from
-                    // conv_state_in, so the slab is assembled from row copies
-                    const int hi_row = min(SLAB_ROWS, T + 3);
-                    if (lane == 0) mbar_expect_tx(BAR_XFULL(slot), (uint32_t)hi_row * X_ROW_BYTES);
-                    __syncwarp();
-                    for (int r = lane; r < hi_row; r += 32) {
-                        const int t = r - 3;
-                        const __nv_bfloat16 *src = t >= 0 ? x + ((size_t)b * T + t) * D + head * DH
-                                                          : cs_in + ((size_t)b * 3 + (3 + t)) * D + head * DH;
-                        bulk_g2s(dst + r * X_ROW_BYTES, src, X_ROW_BYTES, BAR_XFULL(slot));
-                    }
-                } else if (lane == 0) {
-                    // one tiled copy per slab: SLAB_ROWS token rows of this head starting three tokens early
-                    // (tokens before the sequence start and past its end read as zero)
-                    mbar_expect_tx(BAR_XFULL(slot), X_SLAB_BYTES);
-                    tma_load_3d(dst, &p.tm_x, head * DH, ts0 - 3, b, BAR_XFULL(slot));
-                }
+        for (int it = 0; it < n_my_tiles; tile_next(it, b, ti), ++it) {
+            const int slot = it % XS;
+            ok = warp_wait(BAR_XEMPTY(slot), ((it / XS) & 1) ^ 1, spin, abort_flag);
+            if (!ok) break;
+            const int ts0 = ti * TILE + (int)rank * HALF;   // first token this CTA convolves
+            const uint32_t dst = base + SMEM_X + slot * X_SLAB_BYTES;
+            if (ts0 == 0 && cs_in != nullptr) {
+                // first slab of a sequence with an incoming conv state: the three history rows come from
+                // conv_state_in, so the slab is assembled from row copies
+                const int hi_row = min(SLAB_ROWS, T + 3);
+                if (lane == 0) mbar_expect_tx(BAR_XFULL(slot), (uint32_t)hi_row * X_ROW_BYTES);
                 __syncwarp();
+                for (int r = lane; r < hi_row; r += 32) {
+                    const int t = r - 3;
+                    const __nv_bfloat16 *src = t >= 0 ? x + ((size_t)b * T + t) * D + head * DH
+                                                      : cs_in + ((size_t)b * 3 + (3 + t)) * D + head * DH;
+                    bulk_g2s(dst + r * X_ROW_BYTES, src, X_ROW_BYTES, BAR_XFULL(slot));
+                }
+            } else if (lane == 0) {
+                // one tiled copy per slab: SLAB_ROWS token rows of this head starting three tokens early
+                // (tokens before the sequence start and past its end read as zero)
+                mbar_expect_tx(BAR_XFULL(slot), X_SLAB_BYTES);
+                tma_load_3d(dst, &p.tm_x, head * DH, ts0 - 3, b, BAR_XFULL(slot));
             }
+            __syncwarp();
         }
-        if (!ok && lane == 0) record_timeout(f.status, abort_flag);
-      } else if (warp == 5 || warp == 6) {
-        // ================================================================ MMA issuers: warp 5 the W_a products, warp 6 the W_x products
-        // (one thread's issue stream runs at 70-85 cycles per instruction beside the busy warps of its scheduler;
-        // two streams on two schedulers keep the tensor pipe fed)
-        const uint32_t tm_w = warp == 5 ? TM_W_A : TM_W_X, tm_acc = warp == 5 ? TM_ACC_A : TM_ACC_X;
-        // One N = 128 instruction per gate and K step: an N = 64 instruction takes about 45 cycles where 32 would be
-        // its share, an N = 128 one the full-rate 64, so halves would cost more tensor time than they overlap.
-        constexpr uint32_t idesc = make_idesc_f16(128, TILE_N);
+        if (!ok && lane == 0) record_timeout();
+      } else if ((warp == 5 || warp == 6) && rank == 0) {
+        // ================================================================ MMA issuers of the pair: warp 5 the W_a products, warp 6 the W_x products
+        // (one thread's issue stream is slow beside the busy warps of its scheduler; two streams on two schedulers keep the tensor pipe fed)
+        const int gate = warp - 5;
+        const uint32_t tm_w = gate ? TM_W_X : TM_W_A;
+        constexpr uint32_t idesc = make_idesc_f16(256, TILE);
         bool ok = true;
         if (lane == 0) {
-            ok = mbar_wait(BAR_WREADY, 0, spin, abort_flag);
+            ok = mbar_wait_cl(BAR_WREADY, 0, spin, abort_flag);
             for (int it = 0; it < n_my_tiles && ok; ++it) {
-                const int st = it % US;
-                ok = mbar_wait(BAR_UFULL(st), (it / US) & 1, spin, abort_flag);
+                const int st = it % US, bf = it & 1;
+                ok = mbar_wait_cl(BAR_UFULL(st), (it / US) & 1, spin, abort_flag);
                 if (!ok) break;
-                const uint32_t u_base = base + SMEM_U + st * U_STAGE_BYTES;
-                ok = mbar_wait(BAR_ACCEMPTY(0), (it & 1) ^ 1, spin, abort_flag);
+                ok = mbar_wait_cl(BAR_ACCEMPTY(bf), ((it >> 1) & 1) ^ 1, spin, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                // the start-address field of the descriptor counts 16-byte units
-                const uint64_t bd0 = make_desc_sw128(u_base);
+                // the start-address field of the descriptor counts 16-byte units; the same offset addresses each CTA's own stage
+                const uint64_t bd0 = make_desc_sw128(base + SMEM_U + st * U_STAGE_BYTES);
+                const uint32_t acc = tmem + tm_acc(bf, gate);
 #pragma unroll
                 for (int ks = 0; ks < DH / 16; ++ks) {
                     const uint64_t bd = bd0 + (uint64_t)(((ks >> 2) * U_KBLOCK_BYTES + (ks & 3) * 32) >> 4);
-                    mma_ts(tmem + tm_acc, tmem + tm_w + ks * 8, bd, idesc, ks > 0);
+                    mma_ts2(acc, tmem + tm_w + ks * 8, bd, idesc, ks > 0);
                 }
-                tc_commit(BAR_UEMPTY(st));
-                tc_commit(BAR_ACCFULL(0));
+                tc_commit2(BAR_UEMPTY(st), (uint16_t)3);
+                tc_commit2(BAR_ACCFULL(bf), (uint16_t)3);
             }
-            if (!ok) record_timeout(f.status, abort_flag);
+            if (!ok) record_timeout();
         }
         __syncwarp();
       }
-    } else {
-        // ================================================================ epilogue
-        reg_inc<200>();
-        const int q = warp & 3, k = (warp - 8) >> 2;
-        const int c_own = q * 32 + lane;                 // channel within the CTA
-        const int hc = half * CH + c_own;                // channel within the head
+    } else if (warp < 16) {
+        // ================================================================ gate warps
+        reg_inc<104>();
+        const int q = warp & 3, g = (warp - 8) >> 2;     // lane quarter; tokens [32 g, 32 g + 32) of every tile, convolved by CTA g
+        const int hc = (int)rank * CH + q * 32 + lane;   // channel within the head
         const int d = head * DH + hc;                    // global channel
         // per-channel constants; s = c softplus(-Lambda) with libm-grade log1p/exp (Appendix A)
         const float lam = f.lambda[d];
@@ -369,174 +341,169 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         const f32x2 s2 = pack2(s, s);
         const f32x2 hba2 = pack2(0.5f * f.b_a[d], 0.5f * f.b_a[d]), hbx2 = pack2(0.5f * f.b_x[d], 0.5f * f.b_x[d]);
         const bool poly = __all_sync(0xffffffffu, s <= S_POLY);
-        // u[row][channel] in the swizzled U tile, one offset per row phase (row & 7)
+        // u[row][channel] in the swizzled U tile of CTA g, one offset per row phase (row & 7)
+        const bool remote = (uint32_t)g != rank;
+        const uint32_t u_cta = remote ? map_to_cta(base, (uint32_t)g) : base;
         uint32_t u_off[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j)
-            u_off[j] = (uint32_t)(hc >> 6) * U_KBLOCK_BYTES + ((((uint32_t)(hc & 63) >> 3) ^ (uint32_t)j) << 4) + (uint32_t)(hc & 7) * 2 +
-                       (uint32_t)(k * EPI_TOK) * 128u;
+            u_off[j] = u_cta + SMEM_U + (uint32_t)(hc >> 6) * U_KBLOCK_BYTES + ((((uint32_t)(hc & 63) >> 3) ^ (uint32_t)j) << 4) + (uint32_t)(hc & 7) * 2;
+        const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * HALF);
+        bool ok = true;
+        for (int it = 0; it < n_my_tiles; ++it) {
+            const int st = it % US, bf = it & 1;
+            ok = warp_wait_cl(BAR_ACCFULL(bf), (it >> 1) & 1, spin, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t ta = tm_lane + tm_acc(bf, 0), tx = tm_lane + tm_acc(bf, 1);
+            const uint32_t ust = (uint32_t)st * U_STAGE_BYTES;
+            auto batch = [&](auto poly_tag, auto remote_tag, int b2) {
+                constexpr bool POLY = decltype(poly_tag)::value;
+                constexpr bool REMOTE = decltype(remote_tag)::value;
+                f32x2 A2[8], V2[8];   // pairs of adjacent tokens 16 b2 + 2 j, + 1
+                tmem_ld16(ta + 16 * b2, A2);
+                tmem_ld16(tx + 16 * b2, V2);
+                float u[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    const uint32_t addr = u_off[e & 7] + ust + (uint32_t)(16 * b2 + e) * 128u;
+                    u[e] = f16_bits_to_f32((uint16_t)(REMOTE ? ld_cluster_u16(addr) : ld_shared_u16(addr)));
+                }
+                tmem_ld_wait();
+                gate_group<POLY, 4>(A2, V2, u, hba2, hbx2, s2);
+                gate_group<POLY, 4>(A2 + 4, V2 + 4, u + 8, hba2, hbx2, s2);
+                tmem_st16(ta + 16 * b2, A2);
+                tmem_st16(tx + 16 * b2, V2);
+            };
+            auto tile = [&](auto poly_tag, auto remote_tag) { batch(poly_tag, remote_tag, 0); batch(poly_tag, remote_tag, 1); };
+            if (poly) { if (remote) tile(std::true_type{}, std::true_type{}); else tile(std::true_type{}, std::false_type{}); }
+            else      { if (remote) tile(std::false_type{}, std::true_type{}); else tile(std::false_type{}, std::false_type{}); }
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(BAR_GDONE(bf, q));                  // (a_t, v_t) of this warp's half of the tile are in tensor memory
+                mbar_arrive_at(BAR_UEMPTY(st), (uint32_t)g);    // done reading u from CTA g's stage
+            }
+        }
+        if (!ok && lane == 0) record_timeout();
+    } else {
+        // ================================================================ scan warps
+        reg_inc<160>();
+        const int q = warp & 3;
+        const int c_own = q * 32 + lane;                 // channel within the CTA
+        const int d = head * DH + (int)rank * CH + c_own;  // global channel
         const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16);
-        const uint32_t y_warp_off = SMEM_Y + (uint32_t)(k * 4 + q) * Y_WARP_BYTES;
-        uint16_t *y_s = (uint16_t *)(smem + y_warp_off) + lane;   // this thread's column of the warp's y block [64 tokens][32 channels]
-        const uint32_t y_s_addr = base + y_warp_off;
+        const uint32_t y_warp_off = SMEM_Y + (uint32_t)q * 2 * Y_BUF_BYTES;
         const __nv_bfloat16 *x = (const __nv_bfloat16 *)f.x;
         const __nv_bfloat16 *cs_in = (const __nv_bfloat16 *)f.cs_in;
-        float h_prev_own = 0.0f;  // state at the end of this CTA's previous tile
-        float h_scan_end = 0.0f;  // state at the end of this warp's 64 tokens of the previous tile
+        float h_prev_own = 0.0f;  // state at the end of this pair's previous tile
         bool ok = true;
         int b, ti;
         tile_first(b, ti);
-        for (int it = 0; it < n_my_tiles && ok; tile_next(it, b, ti), ++it) {
+        for (int it = 0; it < n_my_tiles; tile_next(it, b, ti), ++it) {
             const bool shared = it < n_shared;
-            const int g = b * p.tps + ti;   // tile number within the half-head: index of its carry record
-            const int t0 = ti * TILE_N;
-            const int st = it % US;
-            const int nv = max(0, min(EPI_TOK, T - t0 - k * EPI_TOK));  // valid tokens of this warp
-            if (k == 0 && it > 0) {
-                // The first half left the previous tile without the second half's fold; it takes it now, before its own
-                // next arrival on BAR_AGG (so that neither side is ever more than one barrier phase ahead of the other).
-                ok = warp_wait(BAR_AGG(q, 1), (it - 1) & 1, spin, abort_flag);
-                if (!ok) break;
-                const float2 other = agg_s[((((it - 1) & 1) * 2 + 1) * 4 + q) * 32 + lane];
-                h_prev_own = fmaf(other.x, h_scan_end, other.y);
-            }
-            ok = warp_wait(BAR_ACCFULL(0), it & 1, spin, abort_flag);
+            const int gidx = (b - B_whole) * p.tps + ti;   // index of the tile's carry record (shared tiles only)
+            const int t0 = ti * TILE;
+            const int bf = it & 1;
+            const int nv = min(TILE, T - t0);  // valid tokens of the tile
+            ok = warp_wait(BAR_GDONE(bf, q), (it >> 1) & 1, spin, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            // A2[j] / V2[j]: tokens j (low half) and j + 32 (high half) of this warp's 64 tokens
-            f32x2 A2[EPI_TOK / 2], V2[EPI_TOK / 2];
-            tmem_ld32(tm_lane + TM_ACC_A + k * EPI_TOK, A2);
-            tmem_ld32(tm_lane + TM_ACC_A + k * EPI_TOK + 32, A2 + 16);
-            tmem_ld32(tm_lane + TM_ACC_X + k * EPI_TOK, V2);
-            tmem_ld32(tm_lane + TM_ACC_X + k * EPI_TOK + 32, V2 + 16);
+            float A[TILE], V[TILE];
+#pragma unroll
+            for (int c = 0; c < TILE; c += 16) {
+                tmem_ld16f(tm_lane + tm_acc(bf, 0) + c, A + c);
+                tmem_ld16f(tm_lane + tm_acc(bf, 1) + c, V + c);
+            }
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(BAR_ACCEMPTY(0));  // the accumulators now live in registers
-            // gates, decay, input scale: (z_a, z_x) -> (a_t, v_t) in place
-            const uint8_t *u_tile = smem + SMEM_U + st * U_STAGE_BYTES;
-            auto gates = [&](auto poly_tag) {
-                constexpr bool POLY = decltype(poly_tag)::value;
-#pragma unroll
-                for (int j = 0; j < EPI_TOK / 2; j += 4) {
-                    float u[8];   // rows 2j' (token j') and 2j' + 1 (token j' + 32) for j' = j .. j + 3
-#pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        u[e] = f16_bits_to_f32(*(const uint16_t *)(u_tile + u_off[(2 * j + e) & 7] + (uint32_t)(2 * j + e) * 128u));
-                    gate_group<POLY, 4>(A2 + j, V2 + j, u, hba2, hbx2, s2);
-                }
-            };
-            if (poly) gates(std::true_type{}); else gates(std::false_type{});
-            __syncwarp();
-            if (lane == 0) mbar_arrive(BAR_UEMPTY(st));  // done reading u
-            if (nv < EPI_TOK) {
+            if (lane == 0) mbar_arrive_at(BAR_ACCEMPTY(bf), 0);  // the tile's (a_t, v_t) now live in registers
+            if (nv < TILE) {
                 // ragged tail: tokens that do not exist hold the state (a = 1, v = 0)
 #pragma unroll
-                for (int j = 0; j < EPI_TOK / 2; ++j) {
-                    const bool v0 = j < nv, v1 = j + 32 < nv;
-                    A2[j] = pack2(v0 ? lo2(A2[j]) : 1.0f, v1 ? hi2(A2[j]) : 1.0f);
-                    V2[j] = pack2(v0 ? lo2(V2[j]) : 0.0f, v1 ? hi2(V2[j]) : 0.0f);
-                }
+                for (int j = 0; j < TILE; ++j) { const bool v = j < nv; A[j] = v ? A[j] : 1.0f; V[j] = v ? V[j] : 0.0f; }
             }
-            // ---- fold both halves at once: h_out = P h_in + hl for tokens [0,32) (low) and [32,64) (high)
-            f32x2 P2 = pack2(1.0f, 1.0f), HL2 = pack2(0.0f, 0.0f);
-#pragma unroll
-            for (int j = 0; j < EPI_TOK / 2; ++j) { P2 = mul2(P2, A2[j]); HL2 = fma2(A2[j], HL2, V2[j]); }
-            const float P_lo = lo2(P2), hl_lo = lo2(HL2);
-            const float P = P_lo * hi2(P2), hl = fmaf(hi2(P2), hl_lo, hi2(HL2));
-            // ---- the second half of the tile needs the fold of the first; the first half goes on without waiting
-            //      and picks up the second half's fold at the start of the next tile
-            //      (the second half arrives only after its own wait: then neither barrier can run two phases ahead)
-            agg_s[(((it & 1) * 2 + k) * 4 + q) * 32 + lane] = make_float2(P, hl);
-            float P_0 = P, hl_0 = hl, P_t = 0.0f, hl_t = 0.0f;    // tokens [0, 64); whole tile (second half only)
-            if (k == 1) {
-                ok = warp_wait(BAR_AGG(q, 0), it & 1, spin, abort_flag);
-                if (!ok) break;
-                const float2 other = agg_s[(((it & 1) * 2 + 0) * 4 + q) * 32 + lane];
-                P_0 = other.x; hl_0 = other.y;
-                P_t = P_0 * P; hl_t = fmaf(P, hl_0, hl);
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(BAR_AGG(q, k));
-            if (shared && S > 1 && k == 1) {
-                uint4 rec;
-                rec.x = __float_as_uint(P_t); rec.y = p.tag; rec.z = __float_as_uint(hl_t); rec.w = p.tag;
-                uint4 *dst = p.agg + ((size_t)group * p.tiles_total + g) * CH + c_own;
-                asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "r"(rec.x), "r"(rec.y), "r"(rec.z), "r"(rec.w) : "memory");
-            }
-            // ---- incoming state of the tile (both halves work it out for themselves): the state this CTA
-            //      reached at the end of its previous tile, or h0 near the start of a sequence, advanced by
-            //      the aggregates that the other CTAs published for the tiles in between (decoupled look-back)
+            // ---- incoming state of the tile: the state this pair reached at the end of its previous tile, or h0 near the
+            //      start of a sequence, advanced by the aggregates that the other pairs published for the tiles in between
             float h;
-            int nback;
             if (!shared) {
                 h = ti == 0 ? (f.h0 ? f.h0[(size_t)b * D + d] : 0.0f) : h_prev_own;
-                nback = 0;
-            } else if (ti == 0 || (S > 1 && ti < S)) {
-                h = f.h0 ? f.h0[(size_t)b * D + d] : 0.0f;
-                nback = ti;
             } else {
-                h = h_prev_own;
-                nback = S - 1;
-            }
-            if (nback > 0) {
-                // All records are requested at once, then polled until every lane sees this call's tag in
-                // both halves of each record (8-byte words are written atomically).
-                const uint4 *src = p.agg + ((size_t)group * p.tiles_total + g) * CH + c_own;
-                uint4 rec[MAX_S - 1];
-                uint64_t tstart = 0;
-                for (uint32_t npoll = 0;; ++npoll) {
-                    bool ready = true;
+                // fold the tile to h_out = P h_in + hl (two half chains side by side) and publish it before waiting for anyone
+                float P0 = 1.0f, H0 = 0.0f, P1 = 1.0f, H1 = 0.0f;
 #pragma unroll
-                    for (int j = 1; j < MAX_S; ++j) {
-                        if (j <= nback) {
-                            const uint4 *sj = src - (size_t)j * CH;
-                            asm volatile("ld.volatile.global.v4.b32 {%0, %1, %2, %3}, [%4];"
-                                         : "=r"(rec[j - 1].x), "=r"(rec[j - 1].y), "=r"(rec[j - 1].z), "=r"(rec[j - 1].w) : "l"(sj) : "memory");
-                        }
-                    }
-#pragma unroll
-                    for (int j = 1; j < MAX_S; ++j)
-                        if (j <= nback) ready = ready && rec[j - 1].y == p.tag && rec[j - 1].w == p.tag;
-                    if (__all_sync(0xffffffffu, ready)) break;
-                    if ((npoll & 15u) == 15u) {
-                        const uint64_t tnow = gtimer();
-                        if (tstart == 0) tstart = tnow;
-                        if (*abort_flag || tnow - tstart > spin) { ok = false; break; }
-                    }
-                    __nanosleep(32);
+                for (int j = 0; j < TILE / 2; ++j) {
+                    P0 *= A[j]; H0 = fmaf(A[j], H0, V[j]);
+                    P1 *= A[j + TILE / 2]; H1 = fmaf(A[j + TILE / 2], H1, V[j + TILE / 2]);
                 }
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
+                uint4 rec;
+                rec.x = __float_as_uint(P0 * P1); rec.y = p.tag; rec.z = __float_as_uint(fmaf(P1, H0, H1)); rec.w = p.tag;
+                uint4 *dst = p.agg + ((size_t)group * p.tiles_total + gidx) * CH + c_own;
+                asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "r"(rec.x), "r"(rec.y), "r"(rec.z), "r"(rec.w) : "memory");
+                int nback;
+                if (ti < S) { h = f.h0 ? f.h0[(size_t)b * D + d] : 0.0f; nback = ti; }
+                else { h = h_prev_own; nback = S - 1; }
+                if (nback > 0) {
+                    // All records are requested at once, then polled until every lane sees this call's tag in
+                    // both halves of each record (8-byte words are written atomically).
+                    const uint4 *src = p.agg + ((size_t)group * p.tiles_total + gidx) * CH + c_own;
+                    uint4 r[MAX_S - 1];
+                    uint64_t tstart = 0;
+                    for (uint32_t npoll = 0;; ++npoll) {
+                        bool ready = true;
 #pragma unroll
-                for (int j = MAX_S - 1; j >= 1; --j)
-                    if (j <= nback) h = fmaf(__uint_as_float(rec[j - 1].x), h, __uint_as_float(rec[j - 1].z));
+                        for (int j = 1; j < MAX_S; ++j) {
+                            if (j <= nback) {
+                                const uint4 *sj = src - (size_t)j * CH;
+                                asm volatile("ld.volatile.global.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                             : "=r"(r[j - 1].x), "=r"(r[j - 1].y), "=r"(r[j - 1].z), "=r"(r[j - 1].w) : "l"(sj) : "memory");
+                            }
+                        }
+#pragma unroll
+                        for (int j = 1; j < MAX_S; ++j)
+                            if (j <= nback) ready = ready && r[j - 1].y == p.tag && r[j - 1].w == p.tag;
+                        if (__all_sync(0xffffffffu, ready)) break;
+                        if ((npoll & 15u) == 15u) {
+                            const uint64_t tnow = gtimer();
+                            if (tstart == 0) tstart = tnow;
+                            if (*abort_flag || tnow - tstart > spin) { ok = false; break; }
+                        }
+                        __nanosleep(32);
+                    }
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+#pragma unroll
+                    for (int j = MAX_S - 1; j >= 1; --j)
+                        if (j <= nback) h = fmaf(__uint_as_float(r[j - 1].x), h, __uint_as_float(r[j - 1].z));
+                }
             }
-            if (k == 1) h_prev_own = fmaf(P_t, h, hl_t);   // state at the end of this tile (the first half works it out later)
-            if (k == 1) h = fmaf(P_0, h, hl_0);       // state at the start of the second half
-            // ---- the warp's y block must have been read out by its previous tiled store
-            if (lane == 0) bulk_wait_read0();
+            // ---- the y block written two tiles ago must have been read out by its tiled store
+            if (lane == 0) bulk_wait_read1();
             __syncwarp();
-            // ---- the recurrence h_t = a_t h_{t-1} + v_t (Eq. 4), both halves in lock step; y_t = h_t
-            f32x2 H2 = pack2(h, fmaf(P_lo, h, hl_lo));
+            // ---- the recurrence h_t = a_t h_{t-1} + v_t (Eq. 4); y_t = h_t
+            const uint32_t y_off = y_warp_off + (uint32_t)bf * Y_BUF_BYTES;
+            uint16_t *y_s = (uint16_t *)(smem + y_off) + lane;   // this thread's column of the warp's y block [64 tokens][32 channels]
 #pragma unroll
-            for (int j = 0; j < EPI_TOK / 2; ++j) {
-                H2 = fma2(A2[j], H2, V2[j]);
-                const __nv_bfloat162 o = __floats2bfloat162_rn(lo2(H2), hi2(H2));
+            for (int j = 0; j < TILE; j += 2) {
+                h = fmaf(A[j], h, V[j]);
+                const float h_even = h;
+                h = fmaf(A[j + 1], h, V[j + 1]);
+                const __nv_bfloat162 o = __floats2bfloat162_rn(h_even, h);
                 const uint32_t ow = *(const uint32_t *)&o;
                 y_s[j * 32] = (uint16_t)(ow & 0xFFFFu);             // row j of the warp's block: 32 channels x 2 bytes
-                y_s[(j + 32) * 32] = (uint16_t)(ow >> 16);
+                y_s[(j + 1) * 32] = (uint16_t)(ow >> 16);
             }
-            h = hi2(H2);
-            h_scan_end = h;
+            h_prev_own = h;
             fence_async_smem();   // y rows become visible to the bulk-copy engine
             __syncwarp();
             if (lane == 0) {
                 // the warp's 64 tokens x 32 channels go out as one tiled store; rows at or beyond T are clipped
-                if (nv > 0) tma_store_3d(&p.tm_y, head * DH + half * CH + q * 32, t0 + k * EPI_TOK, b, y_s_addr);
+                tma_store_3d(&p.tm_y, head * DH + (int)rank * CH + q * 32, t0, b, base + y_off);
                 bulk_commit();
             }
-            if (k == 1 && ti == p.tps - 1) {
+            if (ti == p.tps - 1) {
                 // end of a sequence: h_T (unrounded state) and the last three raw inputs, bit-exact
                 f.h_T[(size_t)b * D + d] = h;
                 __nv_bfloat16 keep[3];
@@ -553,7 +520,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         }
         if (lane == 0) bulk_wait0();
         ok = __all_sync(0xffffffffu, ok);
-        if (!ok && lane == 0) record_timeout(f.status, abort_flag);
+        if (!ok && lane == 0) record_timeout();
     }
 
     // ---- teardown: every role falls through to here, also after a timeout
@@ -563,20 +530,42 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __g
         while (gtimer() - tw < 50000ull) __nanosleep(1000);
     }
     tc_fence_before();
-    __syncthreads();
-    if (warp == 5) tmem_dealloc(tmem, 512);
+    cluster_arrive();   // neither CTA leaves while its peer may still read its shared memory or arrive on its barriers
+    cluster_wait();
+    if (warp == 5) tmem_dealloc2(tmem, 512);
 }
 
-int num_sms() {
-    static int cached = 0;
-    if (cached == 0) {
-        int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-            cached = n;
-        else
-            return 148;
+// Per-device launch facts, looked up once per device with that device current.
+struct DeviceInfo {
+    bool ready = false;
+    int sms = 148;
+    int max_pairs = 70;   // CTA pairs that can be resident at once
+};
+std::mutex g_dev_mutex;
+DeviceInfo g_dev[64];
+
+cudaError_t device_info(DeviceInfo *out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    DeviceInfo &di = g_dev[dev];
+    if (!di.ready) {
+        // opt in to the large dynamic shared memory once per device (function attributes are per context)
+        e = cudaFuncSetAttribute(sm100_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC);
+        if (e != cudaSuccess) return e;
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) di.sms = n;
+        cudaLaunchConfig_t q{};
+        q.gridDim = dim3(2 * di.sms); q.blockDim = dim3(NUM_THREADS); q.dynamicSmemBytes = SMEM_ALLOC;
+        int np = 0;
+        // a pair needs two free SMs of one cluster-capable group, so fewer than sms / 2 pairs may fit
+        di.max_pairs = (cudaOccupancyMaxActiveClusters(&np, sm100_prefill_kernel, &q) == cudaSuccess && np > 0) ? np : di.sms / 2 - 4;
+        di.ready = true;
     }
-    return cached;
+    *out = di;
+    return cudaSuccess;
 }
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point lookup (the library does not link libcuda)
@@ -637,9 +626,12 @@ bool sm100_prefill_supported(int B, int T, int D, int H, int io) {
 
 namespace {
 inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
+// Carry records exist for the sequences that are split in time: at most MAX_S - 1 of them (B mod S with S <= MAX_S).
+// Record (sequence slot, tile, half-head, channel) is indexed as [half-head][slot * tps + tile][channel].
+inline int record_slots(int B) { return B < MAX_S - 1 ? B : MAX_S - 1; }
 size_t agg_bytes(int B, int T, int H) {
-    const size_t tps = (T + TILE_N - 1) / TILE_N;
-    return up256((size_t)H * 2 * B * tps * CH * sizeof(uint4));
+    const size_t tps = (T + TILE - 1) / TILE;
+    return up256((size_t)H * 2 * record_slots(B) * tps * CH * sizeof(uint4));
 }
 inline bool ranges_overlap(const void *a, const void *b, size_t n) {
     if (!a || !b) return false;
@@ -657,26 +649,21 @@ size_t sm100_prefill_workspace_bytes(int B, int T, int D, int H) {
 }
 
 cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes, cudaStream_t st) {
-    static bool attr_set = false;
     cudaError_t e;
-    if (!attr_set) {
-        e = cudaFuncSetAttribute(sm100_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    DeviceInfo di;
+    if ((e = device_info(&di)) != cudaSuccess) return e;
     Sm100Args p;
-    if (!make_activation_map(&p.tm_x, a.x, a.B, a.T, a.D, DH, SLAB_ROWS) || !make_activation_map(&p.tm_y, a.y, a.B, a.T, a.D, 32, EPI_TOK))
+    if (!make_activation_map(&p.tm_x, a.x, a.B, a.T, a.D, DH, SLAB_ROWS) || !make_activation_map(&p.tm_y, a.y, a.B, a.T, a.D, 32, TILE))
         return cudaErrorNotSupported;
     p.f = a;
-    p.tps = (a.T + TILE_N - 1) / TILE_N;
-    p.tiles_total = a.B * p.tps;
-    const int groups = a.H * 2;
-    const int nsm = num_sms();
-    int S = nsm / groups;
+    p.tps = (a.T + TILE - 1) / TILE;
+    const int pairs = di.max_pairs < di.sms / 2 ? di.max_pairs : di.sms / 2;
+    int S = pairs / a.H;
     if (S < 1) S = 1;
     if (S > MAX_S) S = MAX_S;
-    if (S > p.tiles_total) S = p.tiles_total;
+    if (S > a.B * p.tps) S = a.B * p.tps;
     p.S = S;
+    p.tiles_total = record_slots(a.B) * p.tps;
     p.tag = next_tag();
     p.agg = (uint4 *)ws_body;
     p.spin_ns = g_spin_limit_ns;
@@ -691,14 +678,13 @@ cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes,
         if ((e = cudaMemcpyAsync(cs_copy, a.cs_in, cs_bytes, cudaMemcpyDeviceToDevice, st)) != cudaSuccess) return e;
         p.f.cs_in = cs_copy;
     }
-    dim3 grid(groups * S), block(NUM_THREADS);
-    if (S > 1) {
-        // CTAs wait on one another's aggregates: they must all be resident
-        void *args[] = {(void *)&p};
-        return cudaLaunchCooperativeKernel((const void *)sm100_prefill_kernel, grid, block, args, SMEM_ALLOC, st);
-    }
-    sm100_prefill_kernel<<<grid, block, SMEM_ALLOC, st>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(2 * a.H * S); cfg.blockDim = dim3(NUM_THREADS); cfg.dynamicSmemBytes = SMEM_ALLOC; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;   // pairs wait on one another's aggregates: they must all be resident
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr; cfg.numAttrs = (S > 1 && a.B % S != 0) ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, sm100_prefill_kernel, p);
 }
 
 }  // namespace rglru

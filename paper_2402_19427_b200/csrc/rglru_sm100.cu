@@ -9,11 +9,12 @@
 //                  128B-swizzled layout tcgen05.mma reads as this CTA's half of the B operand
 //   MMA warps      (leader CTA only) Z_a^T = W_a U^T and Z_x^T = W_x U^T, N = 64 tokens, K = 256: channels on TMEM
 //                  lanes, time along TMEM columns, two accumulator buffers used alternately
-//   gate warps     tcgen05.ld a batch of (z_a, z_x), u from the U tile of the CTA that convolved the token (its own
-//                  or the peer's through distributed shared memory), gates, log-space decay, input scale, and
-//                  (a_t, v_t) written back over (z_a, z_x) with tcgen05.st; they hold no state and never wait for it
-//   scan warps     pull a tile's (a_t, v_t) into registers, free the accumulator buffer, run the linear recurrence
-//                  h_t = a_t h_{t-1} + v_t in fp32 with the exact incoming state, y through a per-warp tiled store
+//   gate warps     tcgen05.ld half a tile of (z_a, z_x), u from the U tile of the CTA that convolved the token (its own
+//                  or the peer's through distributed shared memory), gates, log-space decay, input scale, then the
+//                  recurrence over the 32 tokens from zero state; (prod a, h from zero) written back over (z_a, z_x)
+//                  with tcgen05.st.  They carry no state between tiles and never wait for one.
+//   scan warps     hold the exact state: y_t = (h_t from zero) + (prod a up to t) h_in in fp32 for each half tile,
+//                  y through a per-warp tiled store, h_in of the next tile from the half tiles' end values
 // x is read from HBM once, y written once; u, r, i, a never leave the pair.
 //
 // Time is split across pairs so that every SM has work even for a single long sequence: sequences that cannot be
@@ -54,7 +55,8 @@ constexpr uint32_t SMEM_U = 0;
 constexpr uint32_t SMEM_X = SMEM_U + US * U_STAGE_BYTES;
 constexpr uint32_t Y_BUF_BYTES = TILE * 32 * 2;            // 4096: one scan warp's 64 tokens x 32 channels
 constexpr uint32_t SMEM_Y = SMEM_X + XS * X_SLAB_BYTES;    // bf16 y_s[4 warps][2 buffers][64][32], staged for tiled stores
-constexpr uint32_t SMEM_BAR = SMEM_Y + 4 * 2 * Y_BUF_BYTES;
+constexpr uint32_t SMEM_AGG = SMEM_Y + 4 * 2 * Y_BUF_BYTES;   // float2 agg_s[2 buffers][2 half tiles][128 channels]
+constexpr uint32_t SMEM_BAR = SMEM_AGG + 2 * 2 * CH * 8;
 constexpr int NUM_BARS = 2 * XS + 2 * US + 4 + 8 + 1;
 constexpr uint32_t SMEM_MISC = SMEM_BAR + NUM_BARS * 8;    // tmem base, abort flag
 constexpr uint32_t SMEM_TOTAL = SMEM_MISC + 16;
@@ -185,9 +187,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
         if (lane == 0) mbar_arrive_at(BAR_WREADY, 0);
     }
 
-    // Register budget per warpgroup (the four warps of a group execute the same setmaxnreg; the increases draw on
-    // what the decreases release: 128 (96-72) + 128 (96-40) = 256 (104-96) + 128 (160-96)):
-    // conv producers 72, loader / MMA issuers / idle 40, gate warps 104, scan warps 160.
+    // Register budget per warpgroup (the four warps of a group execute the same setmaxnreg; the increase draws on
+    // what the decreases release: 128 (96-72) + 128 (96-40) = 256 (136-96)):
+    // conv producers 72, loader / MMA issuers / idle 40, gate warps 136, scan warps the 96 of the launch.
     if (warp < 4) {
         // ================================================================ conv producers
         reg_dec<72>();
@@ -217,44 +219,50 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
         bool ok = true;
         for (int it = 0; it < n_my_tiles; ++it) {
             const int st = it % US, slot = it % XS;
-            ok = warp_wait_cl(BAR_UEMPTY(st), ((it / US) & 1) ^ 1, spin, abort_flag);
+            ok = warp_wait_far(BAR_UEMPTY(st), ((it / US) & 1) ^ 1, spin, abort_flag);
             if (!ok) break;
             ok = warp_wait(BAR_XFULL(slot), (it / XS) & 1, spin, abort_flag);
             if (!ok) break;
             const uint8_t *xs = smem + SMEM_X + slot * X_SLAB_BYTES + x_thread_off;
             uint8_t *us = smem + st * U_STAGE_BYTES;
-            auto load_row = [&](int r, f32x2 &v01, f32x2 &v23) {   // r: row relative to this thread's first history row
-                const uint2 w = *(const uint2 *)(xs + (uint32_t)r * X_ROW_BYTES);
+            auto load_row = [&](const uint8_t *row, f32x2 &v01, f32x2 &v23) {
+                const uint2 w = *(const uint2 *)row;
                 v01 = pack2(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xFFFF0000u));
                 v23 = pack2(__uint_as_float(w.y << 16), __uint_as_float(w.y & 0xFFFF0000u));
             };
             // Rows before the sequence start and at or beyond its end were filled with zeros by the copy, so all 16 tokens
             // are convolved unconditionally; tokens that do not exist produce rows nobody uses.
-            // Four tokens at a time, tap by tap, so that eight independent FMA chains are in flight.
+            // Four tokens at a time, tap by tap, so that eight independent FMA chains are in flight.  The loop over the
+            // halves of the 16 tokens stays rolled: the kernel's roles together must fit the instruction cache.
             f32x2 h01[3], h23[3];   // x_{t-3}, x_{t-2}, x_{t-1}
 #pragma unroll
-            for (int k = 0; k < 3; ++k) load_row(k, h01[k], h23[k]);
+            for (int k = 0; k < 3; ++k) load_row(xs + k * X_ROW_BYTES, h01[k], h23[k]);
+#pragma unroll 1
+            for (int trip = 0; trip < 2; ++trip) {
+                const uint8_t *xr = xs + (uint32_t)(3 + 8 * trip) * X_ROW_BYTES;
+                uint8_t *ur = us + (uint32_t)(8 * trip) * 128u;
 #pragma unroll
-            for (int i0 = 0; i0 < 16; i0 += 4) {
-                f32x2 r01[7], r23[7];   // rows t-3 .. t+3 of the batch
+                for (int i0 = 0; i0 < 8; i0 += 4) {
+                    f32x2 r01[7], r23[7];   // rows t-3 .. t+3 of the batch
 #pragma unroll
-                for (int k = 0; k < 3; ++k) { r01[k] = h01[k]; r23[k] = h23[k]; }
+                    for (int k = 0; k < 3; ++k) { r01[k] = h01[k]; r23[k] = h23[k]; }
 #pragma unroll
-                for (int k = 0; k < 4; ++k) load_row(3 + i0 + k, r01[3 + k], r23[3 + k]);
-                f32x2 u01[4], u23[4];
+                    for (int k = 0; k < 4; ++k) load_row(xr + (uint32_t)(i0 + k) * X_ROW_BYTES, r01[3 + k], r23[3 + k]);
+                    f32x2 u01[4], u23[4];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) { u01[k] = fma2(w01[0], r01[3 + k], b01); u23[k] = fma2(w23[0], r23[3 + k], b23); }
+                    for (int k = 0; k < 4; ++k) { u01[k] = fma2(w01[0], r01[3 + k], b01); u23[k] = fma2(w23[0], r23[3 + k], b23); }
 #pragma unroll
-                for (int j = 1; j < 4; ++j) {
+                    for (int j = 1; j < 4; ++j) {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) { u01[k] = fma2(w01[j], r01[3 + k - j], u01[k]); u23[k] = fma2(w23[j], r23[3 + k - j], u23[k]); }
+                        for (int k = 0; k < 4; ++k) { u01[k] = fma2(w01[j], r01[3 + k - j], u01[k]); u23[k] = fma2(w23[j], r23[3 + k - j], u23[k]); }
+                    }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        *(uint2 *)(ur + sw[i0 + k] + (uint32_t)(i0 + k) * 128u) =
+                            make_uint2(pack_f16_sat(lo2(u01[k]), hi2(u01[k])), pack_f16_sat(lo2(u23[k]), hi2(u23[k])));
+#pragma unroll
+                    for (int k = 0; k < 3; ++k) { h01[k] = r01[4 + k]; h23[k] = r23[4 + k]; }
                 }
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    *(uint2 *)(us + sw[(i0 + k) & 7] + (uint32_t)(i0 + k) * 128u) =
-                        make_uint2(pack_f16_sat(lo2(u01[k]), hi2(u01[k])), pack_f16_sat(lo2(u23[k]), hi2(u23[k])));
-#pragma unroll
-                for (int k = 0; k < 3; ++k) { h01[k] = r01[4 + k]; h23[k] = r23[4 + k]; }
             }
             fence_async_smem();  // make the generic-proxy writes of U visible to the tensor core
             __syncwarp();
@@ -272,7 +280,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
         tile_first(b, ti);
         for (int it = 0; it < n_my_tiles; tile_next(it, b, ti), ++it) {
             const int slot = it % XS;
-            ok = warp_wait(BAR_XEMPTY(slot), ((it / XS) & 1) ^ 1, spin, abort_flag);
+            ok = warp_wait_far(BAR_XEMPTY(slot), ((it / XS) & 1) ^ 1, spin, abort_flag);
             if (!ok) break;
             const int ts0 = ti * TILE + (int)rank * HALF;   // first token this CTA convolves
             const uint32_t dst = base + SMEM_X + slot * X_SLAB_BYTES;
@@ -280,6 +288,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
                 // first slab of a sequence with an incoming conv state: the three history rows come from
                 // conv_state_in, so the slab is assembled from row copies
                 const int hi_row = min(SLAB_ROWS, T + 3);
+                // rows past the end of a short sequence are zeroed, as the tiled copy would have done (stale shared memory
+                // could hold NaN patterns, and the gate arithmetic relies on a finite u for tokens that do not exist)
+                for (int i = lane; i < (SLAB_ROWS - hi_row) * (int)(X_ROW_BYTES / 16); i += 32)
+                    *(uint4 *)(smem + SMEM_X + slot * X_SLAB_BYTES + (uint32_t)hi_row * X_ROW_BYTES + (uint32_t)i * 16) = make_uint4(0, 0, 0, 0);
+                __syncwarp();
                 if (lane == 0) mbar_expect_tx(BAR_XFULL(slot), (uint32_t)hi_row * X_ROW_BYTES);
                 __syncwarp();
                 for (int r = lane; r < hi_row; r += 32) {
@@ -330,7 +343,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
       }
     } else if (warp < 16) {
         // ================================================================ gate warps
-        reg_inc<104>();
+        reg_inc<136>();
         const int q = warp & 3, g = (warp - 8) >> 2;     // lane quarter; tokens [32 g, 32 g + 32) of every tile, convolved by CTA g
         const int hc = (int)rank * CH + q * 32 + lane;   // channel within the head
         const int d = head * DH + hc;                    // global channel
@@ -349,52 +362,75 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
         for (int j = 0; j < 8; ++j)
             u_off[j] = u_cta + SMEM_U + (uint32_t)(hc >> 6) * U_KBLOCK_BYTES + ((((uint32_t)(hc & 63) >> 3) ^ (uint32_t)j) << 4) + (uint32_t)(hc & 7) * 2;
         const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * HALF);
+        float2 *agg_mine = (float2 *)(smem + SMEM_AGG) + g * CH + q * 32 + lane;
         bool ok = true;
-        for (int it = 0; it < n_my_tiles; ++it) {
+        int b, ti;
+        tile_first(b, ti);
+        for (int it = 0; it < n_my_tiles; tile_next(it, b, ti), ++it) {
             const int st = it % US, bf = it & 1;
+            const int nvh = T - ti * TILE - g * HALF;    // tokens of this warp's half tile that exist (may be <= 0 or >= HALF)
             ok = warp_wait_cl(BAR_ACCFULL(bf), (it >> 1) & 1, spin, abort_flag);
             if (!ok) break;
             tc_fence_after();
             const uint32_t ta = tm_lane + tm_acc(bf, 0), tx = tm_lane + tm_acc(bf, 1);
             const uint32_t ust = (uint32_t)st * U_STAGE_BYTES;
-            auto batch = [&](auto poly_tag, auto remote_tag, int b2) {
-                constexpr bool POLY = decltype(poly_tag)::value;
-                constexpr bool REMOTE = decltype(remote_tag)::value;
-                f32x2 A2[8], V2[8];   // pairs of adjacent tokens 16 b2 + 2 j, + 1
-                tmem_ld16(ta + 16 * b2, A2);
-                tmem_ld16(tx + 16 * b2, V2);
+            float c = 1.0f, h = 0.0f;   // running product of a_t and state from zero over this half tile
+            // Sixteen tokens (eight pairs of adjacent tokens) at a time: (z_a, z_x) from tensor memory and u from the U tile ->
+            // gates -> (a_t, v_t) -> scan from zero state -> column t becomes (prod_{s<=t} a_s, h_t from zero), written back
+            // in place.  Eight independent chains per instruction keep the pipes busy in spite of in-order issue; the loop
+            // over the two batches stays rolled to keep the code small.
+#pragma unroll 1
+            for (int bt = 0; bt < 2; ++bt) {
+                f32x2 ZA[8], ZX[8];
                 float u[16];
+                tmem_ld16(ta + 16 * bt, ZA);
+                tmem_ld16(tx + 16 * bt, ZX);
+                const uint32_t row0 = ust + (uint32_t)(16 * bt) * 128u;
+                if (remote) {
 #pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const uint32_t addr = u_off[e & 7] + ust + (uint32_t)(16 * b2 + e) * 128u;
-                    u[e] = f16_bits_to_f32((uint16_t)(REMOTE ? ld_cluster_u16(addr) : ld_shared_u16(addr)));
+                    for (int e = 0; e < 16; ++e) u[e] = f16_bits_to_f32((uint16_t)ld_cluster_u16(u_off[e & 7] + row0 + (uint32_t)e * 128u));
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) u[e] = f16_bits_to_f32((uint16_t)ld_shared_u16(u_off[e & 7] + row0 + (uint32_t)e * 128u));
                 }
                 tmem_ld_wait();
-                gate_group<POLY, 4>(A2, V2, u, hba2, hbx2, s2);
-                gate_group<POLY, 4>(A2 + 4, V2 + 4, u + 8, hba2, hbx2, s2);
-                tmem_st16(ta + 16 * b2, A2);
-                tmem_st16(tx + 16 * b2, V2);
-            };
-            auto tile = [&](auto poly_tag, auto remote_tag) { batch(poly_tag, remote_tag, 0); batch(poly_tag, remote_tag, 1); };
-            if (poly) { if (remote) tile(std::true_type{}, std::true_type{}); else tile(std::true_type{}, std::false_type{}); }
-            else      { if (remote) tile(std::false_type{}, std::true_type{}); else tile(std::false_type{}, std::false_type{}); }
+                if (nvh < HALF) {
+                    // ragged tail: a token that does not exist gets z_a = -inf-like, which the gate arithmetic turns into
+                    // a_t = 1, v_t = 0 exactly (r = 0, so log a = 0 and sqrt(1 - a^2) = 0; its u is finite), i.e. it holds the state
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        ZA[j] = pack2(16 * bt + 2 * j < nvh ? lo2(ZA[j]) : -1e30f, 16 * bt + 2 * j + 1 < nvh ? hi2(ZA[j]) : -1e30f);
+                }
+                if (poly) gate_group<true, 8>(ZA, ZX, u, hba2, hbx2, s2);
+                else gate_group<false, 8>(ZA, ZX, u, hba2, hbx2, s2);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float a0 = lo2(ZA[i]), a1 = hi2(ZA[i]);
+                    const float c0 = c * a0, h0 = fmaf(a0, h, lo2(ZX[i]));
+                    c = c0 * a1; h = fmaf(a1, h0, hi2(ZX[i]));
+                    ZA[i] = pack2(c0, c); ZX[i] = pack2(h0, h);
+                }
+                tmem_st16(ta + 16 * bt, ZA);
+                tmem_st16(tx + 16 * bt, ZX);
+            }
+            agg_mine[bf * 2 * CH] = make_float2(c, h);   // the half tile as one step: h_out = c h_in + h
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(BAR_GDONE(bf, q));                  // (a_t, v_t) of this warp's half of the tile are in tensor memory
+                mbar_arrive(BAR_GDONE(bf, q));                  // this warp's half of the tile is in tensor memory
                 mbar_arrive_at(BAR_UEMPTY(st), (uint32_t)g);    // done reading u from CTA g's stage
             }
         }
         if (!ok && lane == 0) record_timeout();
     } else {
         // ================================================================ scan warps
-        reg_inc<160>();
         const int q = warp & 3;
         const int c_own = q * 32 + lane;                 // channel within the CTA
         const int d = head * DH + (int)rank * CH + c_own;  // global channel
         const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16);
         const uint32_t y_warp_off = SMEM_Y + (uint32_t)q * 2 * Y_BUF_BYTES;
+        const float2 *agg_s = (const float2 *)(smem + SMEM_AGG) + c_own;
         const __nv_bfloat16 *x = (const __nv_bfloat16 *)f.x;
         const __nv_bfloat16 *cs_in = (const __nv_bfloat16 *)f.cs_in;
         float h_prev_own = 0.0f;  // state at the end of this pair's previous tile
@@ -406,40 +442,20 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
             const int gidx = (b - B_whole) * p.tps + ti;   // index of the tile's carry record (shared tiles only)
             const int t0 = ti * TILE;
             const int bf = it & 1;
-            const int nv = min(TILE, T - t0);  // valid tokens of the tile
             ok = warp_wait(BAR_GDONE(bf, q), (it >> 1) & 1, spin, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            float A[TILE], V[TILE];
-#pragma unroll
-            for (int c = 0; c < TILE; c += 16) {
-                tmem_ld16f(tm_lane + tm_acc(bf, 0) + c, A + c);
-                tmem_ld16f(tm_lane + tm_acc(bf, 1) + c, V + c);
-            }
-            tmem_ld_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_at(BAR_ACCEMPTY(bf), 0);  // the tile's (a_t, v_t) now live in registers
-            if (nv < TILE) {
-                // ragged tail: tokens that do not exist hold the state (a = 1, v = 0)
-#pragma unroll
-                for (int j = 0; j < TILE; ++j) { const bool v = j < nv; A[j] = v ? A[j] : 1.0f; V[j] = v ? V[j] : 0.0f; }
-            }
+            // the two half tiles as steps h_out = e.x h_in + e.y
+            const float2 e0 = agg_s[(bf * 2 + 0) * CH], e1 = agg_s[(bf * 2 + 1) * CH];
             // ---- incoming state of the tile: the state this pair reached at the end of its previous tile, or h0 near the
             //      start of a sequence, advanced by the aggregates that the other pairs published for the tiles in between
             float h;
             if (!shared) {
                 h = ti == 0 ? (f.h0 ? f.h0[(size_t)b * D + d] : 0.0f) : h_prev_own;
             } else {
-                // fold the tile to h_out = P h_in + hl (two half chains side by side) and publish it before waiting for anyone
-                float P0 = 1.0f, H0 = 0.0f, P1 = 1.0f, H1 = 0.0f;
-#pragma unroll
-                for (int j = 0; j < TILE / 2; ++j) {
-                    P0 *= A[j]; H0 = fmaf(A[j], H0, V[j]);
-                    P1 *= A[j + TILE / 2]; H1 = fmaf(A[j + TILE / 2], H1, V[j + TILE / 2]);
-                }
+                // publish the tile's aggregate before waiting for anyone
                 uint4 rec;
-                rec.x = __float_as_uint(P0 * P1); rec.y = p.tag; rec.z = __float_as_uint(fmaf(P1, H0, H1)); rec.w = p.tag;
+                rec.x = __float_as_uint(e0.x * e1.x); rec.y = p.tag; rec.z = __float_as_uint(fmaf(e1.x, e0.y, e1.y)); rec.w = p.tag;
                 uint4 *dst = p.agg + ((size_t)group * p.tiles_total + gidx) * CH + c_own;
                 asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "r"(rec.x), "r"(rec.y), "r"(rec.z), "r"(rec.w) : "memory");
                 int nback;
@@ -479,23 +495,46 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
                         if (j <= nback) h = fmaf(__uint_as_float(r[j - 1].x), h, __uint_as_float(r[j - 1].z));
                 }
             }
+            const float h_mid = fmaf(e0.x, h, e0.y);      // state after the first half tile
+            h_prev_own = fmaf(e1.x, h_mid, e1.y);         // state after the tile
             // ---- the y block written two tiles ago must have been read out by its tiled store
             if (lane == 0) bulk_wait_read1();
             __syncwarp();
-            // ---- the recurrence h_t = a_t h_{t-1} + v_t (Eq. 4); y_t = h_t
+            // ---- y_t = h_t = (h_t from zero) + (prod a up to t) h_in  (Eq. 4 unrolled over the half tile), 16 tokens at a time
             const uint32_t y_off = y_warp_off + (uint32_t)bf * Y_BUF_BYTES;
             uint16_t *y_s = (uint16_t *)(smem + y_off) + lane;   // this thread's column of the warp's y block [64 tokens][32 channels]
+            float C[2][16], H[2][16];
+            const uint32_t tc = tm_lane + tm_acc(bf, 0), th = tm_lane + tm_acc(bf, 1);
+            auto emit = [&](int set, float hb, uint16_t *dst) {
 #pragma unroll
-            for (int j = 0; j < TILE; j += 2) {
-                h = fmaf(A[j], h, V[j]);
-                const float h_even = h;
-                h = fmaf(A[j + 1], h, V[j + 1]);
-                const __nv_bfloat162 o = __floats2bfloat162_rn(h_even, h);
-                const uint32_t ow = *(const uint32_t *)&o;
-                y_s[j * 32] = (uint16_t)(ow & 0xFFFFu);             // row j of the warp's block: 32 channels x 2 bytes
-                y_s[(j + 1) * 32] = (uint16_t)(ow >> 16);
+                for (int j = 0; j < 16; j += 2) {
+                    const float y0 = fmaf(C[set][j], hb, H[set][j]), y1 = fmaf(C[set][j + 1], hb, H[set][j + 1]);
+                    const __nv_bfloat162 o = __floats2bfloat162_rn(y0, y1);
+                    const uint32_t ow = *(const uint32_t *)&o;
+                    dst[j * 32] = (uint16_t)(ow & 0xFFFFu);             // row of the warp's block: 32 channels x 2 bytes
+                    dst[(j + 1) * 32] = (uint16_t)(ow >> 16);
+                }
+            };
+            tmem_ld16f(tc, C[0]);
+            tmem_ld16f(th, H[0]);
+#pragma unroll 1
+            for (int trip = 0; trip < 2; ++trip) {   // trip 0: the first half tile (incoming state h), trip 1: the second (h_mid)
+                const float hb = trip == 0 ? h : h_mid;
+                tmem_ld_wait();
+                tmem_ld16f(tc + 32 * trip + 16, C[1]);
+                tmem_ld16f(th + 32 * trip + 16, H[1]);
+                emit(0, hb, y_s + (32 * trip) * 32);
+                tmem_ld_wait();
+                if (trip == 0) {
+                    tmem_ld16f(tc + 32, C[0]);
+                    tmem_ld16f(th + 32, H[0]);
+                } else {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_at(BAR_ACCEMPTY(bf), 0);  // the whole tile has been read out of tensor memory
+                }
+                emit(1, hb, y_s + (32 * trip + 16) * 32);
             }
-            h_prev_own = h;
             fence_async_smem();   // y rows become visible to the bulk-copy engine
             __syncwarp();
             if (lane == 0) {
@@ -505,7 +544,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
             }
             if (ti == p.tps - 1) {
                 // end of a sequence: h_T (unrounded state) and the last three raw inputs, bit-exact
-                f.h_T[(size_t)b * D + d] = h;
+                f.h_T[(size_t)b * D + d] = h_prev_own;
                 __nv_bfloat16 keep[3];
 #pragma unroll
                 for (int kk = 0; kk < 3; ++kk) {

@@ -31,27 +31,56 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// One test of the barrier phase.  The thread may be suspended until the phase completes or the hinted time has passed,
+// whichever comes first.
+constexpr uint32_t MBAR_SUSPEND_NS = 20000;
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     uint32_t ok;
-    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.b32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "n"(MBAR_SUSPEND_NS) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false when the limit ran out or the CTA is aborting.  mbarrier.try_wait
-// suspends the thread for a hardware-chosen window, so the loop polls rarely; the abort flag and the
-// global timer are consulted once every 32 polls to keep the loop itself cheap.
+// Up to 256 tests in a loop of three instructions (a suspended thread is woken by unrelated barrier traffic as well, so
+// tests are frequent and the loop around them must be cheap).
+__device__ __forceinline__ bool mbar_try256(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\n.reg .b32 n;\nmov.b32 n, 256;\nMBT_LOOP:\n"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n@p bra MBT_DONE;\n"
+                 "sub.u32 n, n, 1;\nsetp.ne.u32 p, n, 0;\n@p bra MBT_LOOP;\nsetp.ne.u32 p, n, 0;\n"
+                 "MBT_DONE:\nselp.b32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "n"(MBAR_SUSPEND_NS) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the limit ran out or the CTA is aborting; the abort flag and the global timer are
+// consulted once every 256 tests.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
-    if (mbar_try(bar, parity)) return true;
+    if (mbar_try256(bar, parity)) return true;
+    const uint64_t t0 = gtimer();
+    for (;;) {
+        if (mbar_try256(bar, parity)) return true;
+        if (*abort_flag || gtimer() - t0 > limit_ns) return false;
+    }
+}
+// Bounded wait for something that is normally many microseconds away (a ring slot several stages ahead): the thread sleeps
+// between tests instead of being woken by every barrier event of the CTA.
+__device__ __forceinline__ bool mbar_wait_far(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
+    uint32_t ok;
     uint64_t t0 = 0;
-    for (uint32_t n = 1;; ++n) {
-        if (mbar_try(bar, parity)) return true;
-        if ((n & 31u) == 0u) {
+    for (uint32_t n = 0;; ++n) {
+        asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        __nanosleep(400);
+        if ((n & 63u) == 63u) {
             if (*abort_flag) return false;
             const uint64_t t = gtimer();
             if (t0 == 0) t0 = t;
             else if (t - t0 > limit_ns) return false;
         }
     }
+}
+__device__ __forceinline__ bool warp_wait_far(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
+    return __all_sync(0xffffffffu, mbar_wait_far(bar, parity, limit_ns, abort_flag));
 }
 // All lanes wait; the verdict is made warp-uniform so that a warp never splits on a timeout.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
@@ -76,7 +105,8 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
     asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
                  ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
 }
-typedef unsigned long long f32x2;
+// Two fp32 values in an aligned register pair; arithmetic through the packed-fp32 builtins (fma.rn.f32x2 and friends).
+typedef float2 f32x2;
 // D[tmem] (+)= A[smem] * B[smem]^T, kind::f16 (A and B of one 16-bit type, fp32 accumulate), one CTA
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
     asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
@@ -118,7 +148,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, f32x2 *v) {
                    "=r"(r[30]), "=r"(r[31])
                  : "r"(taddr) : "memory");
 #pragma unroll
-    for (int j = 0; j < 16; ++j) asm("mov.b64 %0, {%1, %2};" : "=l"(v[j]) : "r"(r[2 * j]), "r"(r[2 * j + 1]));
+    for (int j = 0; j < 16; ++j) v[j] = make_float2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st8(uint32_t taddr, uint4 lo, uint4 hi) {
@@ -170,11 +200,11 @@ __host__ __device__ constexpr uint32_t make_idesc(int M, int N) {
 }
 
 // ---- packed fp32x2 arithmetic (one issue slot for two lanes' worth of FP32 work)
-__device__ __forceinline__ f32x2 pack2(float lo, float hi) { f32x2 v; asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi)); return v; }
-__device__ __forceinline__ float lo2(f32x2 v) { float lo, hi; asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); (void)hi; return lo; }
-__device__ __forceinline__ float hi2(f32x2 v) { float lo, hi; asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); (void)lo; return hi; }
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
-__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) { return make_float2(lo, hi); }
+__device__ __forceinline__ float lo2(f32x2 v) { return v.x; }
+__device__ __forceinline__ float hi2(f32x2 v) { return v.y; }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { return __fmul2_rn(a, b); }
 __device__ __forceinline__ float tanh_approx(float x) { float y; asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
 __device__ __forceinline__ float sqrt_approx(float x) { float y; asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
 __device__ __forceinline__ float ex2_approx(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
@@ -200,30 +230,18 @@ __device__ __forceinline__ void tc_commit2(uint32_t bar, uint16_t cta_mask) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                  ::"r"(bar), "h"(cta_mask) : "memory");
 }
-// Arrive on the barrier at this shared-memory offset in CTA `cta` of the cluster (this CTA included); release at cluster scope.
+// Arrive on the barrier at this shared-memory offset in CTA `cta` of the cluster (this CTA included).  The default
+// semantics (release at CTA scope) are used on purpose: a release at cluster scope was measured at 1.5-2 k cycles per
+// arrive.  What the arrivals publish is ordered by other means: tensor-memory accesses by tcgen05.fence, shared-memory
+// tiles for the tensor core by fence.proxy.async, and "done reading" signals publish nothing.
 __device__ __forceinline__ void mbar_arrive_at(uint32_t bar, uint32_t cta) {
-    asm volatile("{\n.reg .b32 ra;\nmapa.shared::cluster.u32 ra, %0, %1;\nmbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n}"
+    asm volatile("{\n.reg .b32 ra;\nmapa.shared::cluster.u32 ra, %0, %1;\nmbarrier.arrive.shared::cluster.b64 _, [ra];\n}"
                  ::"r"(bar), "r"(cta) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_cl(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait like mbar_wait, acquiring at cluster scope: for barriers that threads of the peer CTA arrive on.
+__device__ __forceinline__ bool mbar_try_cl(uint32_t bar, uint32_t parity) { return mbar_try(bar, parity); }
+// Bounded wait on a barrier that threads of the peer CTA arrive on (same code as mbar_wait: see mbar_arrive_at).
 __device__ __forceinline__ bool mbar_wait_cl(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
-    if (mbar_try_cl(bar, parity)) return true;
-    uint64_t t0 = 0;
-    for (uint32_t n = 1;; ++n) {
-        if (mbar_try_cl(bar, parity)) return true;
-        if ((n & 31u) == 0u) {
-            if (*abort_flag) return false;
-            const uint64_t t = gtimer();
-            if (t0 == 0) t0 = t;
-            else if (t - t0 > limit_ns) return false;
-        }
-    }
+    return mbar_wait(bar, parity, limit_ns, abort_flag);
 }
 __device__ __forceinline__ bool warp_wait_cl(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
     return __all_sync(0xffffffffu, mbar_wait_cl(bar, parity, limit_ns, abort_flag));
@@ -245,12 +263,12 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, f32x2 *v) {
                    "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
                  : "r"(taddr) : "memory");
 #pragma unroll
-    for (int j = 0; j < 8; ++j) asm("mov.b64 %0, {%1, %2};" : "=l"(v[j]) : "r"(r[2 * j]), "r"(r[2 * j + 1]));
+    for (int j = 0; j < 8; ++j) v[j] = make_float2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
 }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const f32x2 *v) {
     uint32_t r[16];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) asm("mov.b64 {%0, %1}, %2;" : "=r"(r[2 * j]), "=r"(r[2 * j + 1]) : "l"(v[j]));
+    for (int j = 0; j < 8; ++j) { r[2 * j] = __float_as_uint(v[j].x); r[2 * j + 1] = __float_as_uint(v[j].y); }
     asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
                  ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
                    "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
@@ -264,6 +282,32 @@ __device__ __forceinline__ void tmem_ld16f(uint32_t taddr, float *v) {
                  : "r"(taddr) : "memory");
 #pragma unroll
     for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+}
+// 32 consecutive columns from 16 register pairs
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const f32x2 *v) {
+    uint32_t r[32];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) { r[2 * j] = __float_as_uint(v[j].x); r[2 * j + 1] = __float_as_uint(v[j].y); }
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+                   "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]),
+                   "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),
+                   "r"(r[30]), "r"(r[31]) : "memory");
+}
+// 8 consecutive columns of this thread's lane as 4 register pairs (column 2j in the low half), and the matching store
+__device__ __forceinline__ void tmem_ld8p(uint32_t taddr, f32x2 *v) {
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]) : "r"(taddr) : "memory");
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[j] = make_float2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+}
+__device__ __forceinline__ void tmem_st8p(uint32_t taddr, const f32x2 *v) {
+    uint32_t r[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { r[2 * j] = __float_as_uint(v[j].x); r[2 * j + 1] = __float_as_uint(v[j].y); }
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
 }
 __device__ __forceinline__ void bulk_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 

@@ -187,12 +187,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
         if (lane == 0) mbar_arrive_at(BAR_WREADY, 0);
     }
 
-    // Register budget per warpgroup (the four warps of a group execute the same setmaxnreg; the increase draws on
-    // what the decreases release: 128 (96-72) + 128 (96-40) = 256 (136-96)):
-    // conv producers 72, loader / MMA issuers / idle 40, gate warps 136, scan warps the 96 of the launch.
+    // Register budget per warpgroup (the four warps of a group execute the same setmaxnreg; the increases draw on
+    // what the decreases release: 128 (96-64) + 128 (96-40) = 256 (112-96) + 128 (152-96)):
+    // conv producers 64, loader / MMA issuers / idle 40, gate warps 112, scan warps 152.
     if (warp < 4) {
         // ================================================================ conv producers
-        reg_dec<72>();
+        reg_dec<64>();
         const int pblk = warp;                       // K block = 64 channels of the head
         const int l16 = lane & 15, tg = lane >> 4;   // 4-channel chunk, token group of 16
         const int hc = pblk * 64 + l16 * 4;          // channel within the head
@@ -343,7 +343,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
       }
     } else if (warp < 16) {
         // ================================================================ gate warps
-        reg_inc<136>();
+        reg_inc<112>();
         const int q = warp & 3, g = (warp - 8) >> 2;     // lane quarter; tokens [32 g, 32 g + 32) of every tile, convolved by CTA g
         const int hc = (int)rank * CH + q * 32 + lane;   // channel within the head
         const int d = head * DH + hc;                    // global channel
@@ -425,6 +425,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
         if (!ok && lane == 0) record_timeout();
     } else {
         // ================================================================ scan warps
+        reg_inc<152>();
         const int q = warp & 3;
         const int c_own = q * 32 + lane;                 // channel within the CTA
         const int d = head * DH + (int)rank * CH + c_own;  // global channel
@@ -503,37 +504,24 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
             // ---- y_t = h_t = (h_t from zero) + (prod a up to t) h_in  (Eq. 4 unrolled over the half tile), 16 tokens at a time
             const uint32_t y_off = y_warp_off + (uint32_t)bf * Y_BUF_BYTES;
             uint16_t *y_s = (uint16_t *)(smem + y_off) + lane;   // this thread's column of the warp's y block [64 tokens][32 channels]
-            float C[2][16], H[2][16];
+            // The whole tile is pulled into registers and the accumulator buffer handed back before any arithmetic: the buffer's
+            // round trip (MMA -> gate warps -> here -> MMA) is what paces the kernel.
+            float C[TILE], H[TILE];
             const uint32_t tc = tm_lane + tm_acc(bf, 0), th = tm_lane + tm_acc(bf, 1);
-            auto emit = [&](int set, float hb, uint16_t *dst) {
 #pragma unroll
-                for (int j = 0; j < 16; j += 2) {
-                    const float y0 = fmaf(C[set][j], hb, H[set][j]), y1 = fmaf(C[set][j + 1], hb, H[set][j + 1]);
-                    const __nv_bfloat162 o = __floats2bfloat162_rn(y0, y1);
-                    const uint32_t ow = *(const uint32_t *)&o;
-                    dst[j * 32] = (uint16_t)(ow & 0xFFFFu);             // row of the warp's block: 32 channels x 2 bytes
-                    dst[(j + 1) * 32] = (uint16_t)(ow >> 16);
-                }
-            };
-            tmem_ld16f(tc, C[0]);
-            tmem_ld16f(th, H[0]);
-#pragma unroll 1
-            for (int trip = 0; trip < 2; ++trip) {   // trip 0: the first half tile (incoming state h), trip 1: the second (h_mid)
-                const float hb = trip == 0 ? h : h_mid;
-                tmem_ld_wait();
-                tmem_ld16f(tc + 32 * trip + 16, C[1]);
-                tmem_ld16f(th + 32 * trip + 16, H[1]);
-                emit(0, hb, y_s + (32 * trip) * 32);
-                tmem_ld_wait();
-                if (trip == 0) {
-                    tmem_ld16f(tc + 32, C[0]);
-                    tmem_ld16f(th + 32, H[0]);
-                } else {
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_at(BAR_ACCEMPTY(bf), 0);  // the whole tile has been read out of tensor memory
-                }
-                emit(1, hb, y_s + (32 * trip + 16) * 32);
+            for (int c0 = 0; c0 < TILE; c0 += 16) { tmem_ld16f(tc + c0, C + c0); tmem_ld16f(th + c0, H + c0); }
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_at(BAR_ACCEMPTY(bf), 0);
+#pragma unroll
+            for (int j = 0; j < TILE; j += 2) {
+                const float hb = j < HALF ? h : h_mid;
+                const float y0 = fmaf(C[j], hb, H[j]), y1 = fmaf(C[j + 1], hb, H[j + 1]);
+                const __nv_bfloat162 o = __floats2bfloat162_rn(y0, y1);
+                const uint32_t ow = *(const uint32_t *)&o;
+                y_s[j * 32] = (uint16_t)(ow & 0xFFFFu);             // row of the warp's block: 32 channels x 2 bytes
+                y_s[(j + 1) * 32] = (uint16_t)(ow >> 16);
             }
             fence_async_smem();   // y rows become visible to the bulk-copy engine
             __syncwarp();

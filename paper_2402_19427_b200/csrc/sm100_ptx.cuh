@@ -61,6 +61,26 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigne
         if (*abort_flag || gtimer() - t0 > limit_ns) return false;
     }
 }
+// Bounded wait that never suspends the thread: for hand-offs that are normally tens of cycles away, where the wake-up time of a
+// suspended thread would dominate.
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
+    uint32_t ok;
+    uint64_t t0 = 0;
+    for (uint32_t n = 0;; ++n) {
+        asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        if ((n & 1023u) == 1023u) {
+            if (*abort_flag) return false;
+            const uint64_t t = gtimer();
+            if (t0 == 0) t0 = t;
+            else if (t - t0 > limit_ns) return false;
+        }
+    }
+}
+__device__ __forceinline__ bool warp_wait_spin(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
+    return __all_sync(0xffffffffu, mbar_wait_spin(bar, parity, limit_ns, abort_flag));
+}
 // Bounded wait for something that is normally many microseconds away (a ring slot several stages ahead): the thread sleeps
 // between tests instead of being woken by every barrier event of the CTA.
 __device__ __forceinline__ bool mbar_wait_far(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
@@ -70,8 +90,8 @@ __device__ __forceinline__ bool mbar_wait_far(uint32_t bar, uint32_t parity, uns
         asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}"
                      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
         if (ok) return true;
-        __nanosleep(400);
-        if ((n & 63u) == 63u) {
+        __nanosleep(2000);
+        if ((n & 15u) == 15u) {
             if (*abort_flag) return false;
             const uint64_t t = gtimer();
             if (t0 == 0) t0 = t;
@@ -82,7 +102,8 @@ __device__ __forceinline__ bool mbar_wait_far(uint32_t bar, uint32_t parity, uns
 __device__ __forceinline__ bool warp_wait_far(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
     return __all_sync(0xffffffffu, mbar_wait_far(bar, parity, limit_ns, abort_flag));
 }
-// All lanes wait; the verdict is made warp-uniform so that a warp never splits on a timeout.
+// All lanes wait (a wait or sleep executed by part of a warp returns at once, as measured); the verdict is made
+// warp-uniform so that a warp never splits on a timeout.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity, limit_ns, abort_flag));
 }
@@ -194,6 +215,9 @@ __device__ __forceinline__ uint32_t pack_f16_sat(float lo, float hi) {
     uint32_t r; asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo)); return r;
 }
 __device__ __forceinline__ float f16_bits_to_f32(uint16_t h) { float r; asm("cvt.f32.f16 %0, %1;" : "=f"(r) : "h"(h)); return r; }
+// The same, kept in program order with respect to the other volatile statements around it: a conversion placed before a
+// barrier arrive proves that the load which produced its operand has completed by then.
+__device__ __forceinline__ float f16_bits_to_f32_ordered(uint16_t h) { float r; asm volatile("cvt.f32.f16 %0, %1;" : "=f"(r) : "h"(h)); return r; }
 // the same descriptor with bf16 A and B
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
@@ -244,7 +268,13 @@ __device__ __forceinline__ bool mbar_wait_cl(uint32_t bar, uint32_t parity, unsi
     return mbar_wait(bar, parity, limit_ns, abort_flag);
 }
 __device__ __forceinline__ bool warp_wait_cl(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag) {
-    return __all_sync(0xffffffffu, mbar_wait_cl(bar, parity, limit_ns, abort_flag));
+    return warp_wait(bar, parity, limit_ns, abort_flag);
+}
+// bulk copy from this CTA's shared memory into a peer's (addresses of the peer in the cluster window); the bytes are counted
+// on a barrier of the peer
+__device__ __forceinline__ void bulk_s2peer(uint32_t dst_cluster, uint32_t src_smem, uint32_t bytes, uint32_t bar_cluster) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_cluster), "r"(src_smem), "r"(bytes), "r"(bar_cluster) : "memory");
 }
 __device__ __forceinline__ uint32_t ld_cluster_u16(uint32_t cluster_addr) {
     uint16_t v; asm volatile("ld.shared::cluster.u16 %0, [%1];" : "=h"(v) : "r"(cluster_addr) : "memory"); return v;

@@ -6,15 +6,19 @@ state hand-off) over one batch of the training-shape workload (B=8, T=2048, D_RN
 state).  The same JSON line also carries the batched decode step (B=512) and the backward as extra measurements.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py --only prefill|decode|backward [--B .. --T .. --D .. --H ..] [--iters n]    (one op, for profilers)
 
-N > 1 is launched with torch.distributed.run, one rank per GPU; sequences are independent, so each rank runs the
-full workload on its own seeded batch (weak scaling, no data-path collective); the time is the max over ranks.
+N > 1: one rank per GPU, each on its own seeded batch (sequences are independent: weak scaling, no data-path
+collective); the time is the max over ranks.  Started without a rank environment, the script launches its own ranks
+through torch.distributed.run.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import subprocess
 import sys
 import threading
 import time
@@ -30,9 +34,20 @@ from paper_2402_19427_b200 import inputs as synth, sharding  # noqa: E402
 WORKLOAD = 1                 # index into synth.CONFIGS: the training-shape prefill
 N_ROTATE = 4                 # distinct input/output buffer sets cycled between steps (defeats L2 reuse)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes per prefill launch on the bench workload from the committed ncu capture
-# (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
-NCU_TRAFFIC_BYTES = 132525056   # 86.90 MB read + 45.63 MB written (profiles/sm100_prefill_kernel_cfg1.md)
+# DRAM bytes per prefill launch on the bench workload (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture,
+# profiles/sm100_prefill_kernel_cfg1.md) together with the SHA-256 of the kernel source the capture was taken from:
+# the figure is reported only while the benched kernel source still has that hash, else null.
+NCU_TRAFFIC = {"bytes": None, "kernel_sha256": None}
+KERNEL_SOURCE = os.path.join(ROOT, "paper_2402_19427_b200", "csrc", "rglru_sm100.cu")
+
+
+def captured_traffic():
+    try:
+        with open(KERNEL_SOURCE, "rb") as f:
+            sha = hashlib.sha256(f.read()).hexdigest()
+    except OSError:
+        return None
+    return NCU_TRAFFIC["bytes"] if sha == NCU_TRAFFIC["kernel_sha256"] else None
 
 
 def load_peaks():
@@ -54,6 +69,65 @@ def algorithmic_work(cfg):
     nbytes = 2 * elems * io + (4 * D + 2 * H * Dh * Dh) * io + 4 * D * 4 + B * D * 4 + B * 3 * D * io
     flops = elems * 4 * Dh
     return nbytes, flops
+
+
+def roofline(nbytes, flops, launch_s, peaks, peak_kind, traffic=None):
+    """The slower of (bytes at the copy rate, FLOPs at the tensor rate) is the bound; achieved = that quantity / time."""
+    t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
+    t_tc = flops / (peaks["bf16_tflops"] * 1e12)
+    if t_tc >= t_hbm:
+        roof = {"bound": "tensor", "achieved": flops / launch_s / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
+    else:
+        roof = {"bound": "hbm", "achieved": nbytes / launch_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = traffic
+    roof.update({"peaks": peak_kind, "launch_us": launch_s * 1e6, "hbm_gbs_achieved": nbytes / launch_s / 1e9,
+                 "hbm_frac": nbytes / launch_s / 1e9 / peaks["hbm_gbs"], "tensor_tflops_achieved": flops / launch_s / 1e12,
+                 "tensor_frac": flops / launch_s / 1e12 / peaks["bf16_tflops"], "algorithmic_bytes": nbytes, "gate_flops": flops,
+                 # for context only: the same work against the data-sheet figures (8 TB/s, 2.25 PFLOP/s dense bf16)
+                 "frac_of_nominal": max(nbytes / 8.0e12, flops / 2.25e15) / launch_s})
+    return roof
+
+
+def event_times_us(fn, reps, torch):
+    """Runs fn() reps times, each between its own pair of CUDA events on the current stream; returns the times in us."""
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for a, b in evs:
+        a.record(); fn(); b.record()
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) * 1e3 for a, b in evs]
+
+
+def time_prefill_config(binding, dev, index, peaks, peak_kind, reps=20):
+    """One of the other prefill shapes as a side record: `reps` launches over rotating buffer sets, median and min."""
+    import torch
+    cfg = dict(synth.CONFIGS[index])
+    B, T, D, H = cfg["B"], cfg["T"], cfg["D"], cfg["H"]
+    dt = torch.bfloat16
+    pr = synth.make_inputs(1, 4, D, H, io="bf16", seed=synth.BASE_SEED + index)["params"]
+    params = binding.Params.from_numpy(pr, "bf16", device=dev)
+    nset = max(2, int(np.ceil(300e6 / (2 * B * T * D * 2))))     # input + output of all sets exceed the 126 MB L2 twice over
+    g = torch.Generator(device=dev); g.manual_seed(index)
+    xs = [torch.randn(B, T, D, device=dev, generator=g).to(dt) for _ in range(nset)]
+    ys = [torch.empty_like(xs[0]) for _ in range(nset)]
+    shape = binding.make_shape(B, T, D, H, dt)
+    ws = binding.alloc_workspace(shape, binding.OP_PREFILL, dev)
+    k = [0]
+
+    def one():
+        binding.prefill(xs[k[0] % nset], params, y=ys[k[0] % nset], workspace=ws); k[0] += 1
+
+    for _ in range(3):
+        one()
+    torch.cuda.synchronize()
+    us = event_times_us(one, reps, torch)
+    status = binding.query_status(ws)
+    if status != binding.OK:
+        raise binding.RglruError(status, "device status after the side measurement")
+    nbytes, flops = algorithmic_work(cfg)
+    med = float(np.median(us))
+    return {"workload": workload_name(cfg), "us_median": med, "us_min": float(np.min(us)), "reps": reps,
+            "tokens_per_s": B * T / (med * 1e-6), "buffer_sets": nset, "roofline": roofline(nbytes, flops, med * 1e-6, peaks, peak_kind)}
 
 
 class ClockSampler:
@@ -256,24 +330,15 @@ def run_ours(args):
     peaks, peak_kind = load_peaks()
     nbytes, flops = algorithmic_work(cfg)
     launch_s = float(np.mean(per_launch_ms)) * 1e-3
-    t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
-    t_tc = flops / (peaks["bf16_tflops"] * 1e12)
-    if t_tc >= t_hbm:
-        roof = {"bound": "tensor", "achieved": flops / launch_s / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
-    else:
-        roof = {"bound": "hbm", "achieved": nbytes / launch_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = NCU_TRAFFIC_BYTES
-    roof.update({"peaks": peak_kind, "kernel": "rglru prefill (dominant kernel of the step)",
-                 "launch_us": launch_s * 1e6, "hbm_gbs_achieved": nbytes / launch_s / 1e9,
-                 "hbm_frac": nbytes / launch_s / 1e9 / peaks["hbm_gbs"], "tensor_tflops_achieved": flops / launch_s / 1e12,
-                 "tensor_frac": flops / launch_s / 1e12 / peaks["bf16_tflops"], "algorithmic_bytes": nbytes, "gate_flops": flops,
-                 # for context only: the same work against the data-sheet figures (8 TB/s, 2.25 PFLOP/s dense bf16)
-                 "frac_of_nominal": max(nbytes / 8.0e12, flops / 2.25e15) / launch_s})
+    roof = roofline(nbytes, flops, launch_s, peaks, peak_kind, traffic=captured_traffic())
+    roof["kernel"] = "rglru prefill (dominant kernel of the step)"
 
     extra = {}
     if rank == 0 and not args.no_extras:
-        extra = measure_extras(binding, dev, peaks)
+        # the other prefill shapes: the long sequence (every tile through the decoupled look-back) and the training shape of config 4
+        extra["prefill_long"] = time_prefill_config(binding, dev, 2, peaks, peak_kind)
+        extra["prefill_cfg4_forward"] = time_prefill_config(binding, dev, 4, peaks, peak_kind)
+        extra.update(measure_extras(binding, dev, peaks))
 
     if rank == 0:
         line = {"metric": "rglru_prefill_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
@@ -319,35 +384,56 @@ def measure_extras(binding, dev, peaks):
             binding.decode_step(xs[t], params, h, cs, y=y, workspace=ws)
 
     chain(); torch.cuda.synchronize()
-    reps = 3
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(reps):
-        chain()
-    e1.record(); torch.cuda.synchronize()
-    us_plain = e0.elapsed_time(e1) * 1e3 / (reps * steps)
-    # the same chain captured once in a CUDA graph (launch overhead off the critical path)
-    graph = torch.cuda.CUDAGraph()
-    side = torch.cuda.Stream()
-    side.wait_stream(torch.cuda.current_stream())
-    with torch.cuda.stream(side):
-        chain()
-        with torch.cuda.graph(graph, stream=side):
-            chain()
-    torch.cuda.current_stream().wait_stream(side)
-    graph.replay(); torch.cuda.synchronize()
-    e0.record()
-    for _ in range(reps):
-        graph.replay()
-    e1.record(); torch.cuda.synchronize()
-    us_graph = e0.elapsed_time(e1) * 1e3 / (reps * steps)
-    us = min(us_plain, us_graph)
+    reps = 20
+    us_plain_all = [t / steps for t in event_times_us(chain, reps, torch)]
+
+    def graph_of(fn):
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+            with torch.cuda.graph(graph, stream=side):
+                fn()
+        torch.cuda.current_stream().wait_stream(side)
+        graph.replay(); torch.cuda.synchronize()
+        return graph
+
+    # the same chain captured once in a CUDA graph (launch overhead off the critical path); one state set: h and the conv
+    # state (13 MB) stay in the 126 MB L2 between steps
+    graph = graph_of(chain)
+    us_graph_all = [t / steps for t in event_times_us(graph.replay, reps, torch)]
+    # the same number of steps over rotating state sets that together exceed L2 several times, so that every step's h and
+    # conv state come from and go to HBM (a server with many resident sequence groups)
+    nsets = 32
+    hs = [torch.randn(B, D, device=dev, generator=g) for _ in range(nsets)]
+    css = [torch.randn(B, 3, D, device=dev, generator=g).to(dt) for _ in range(nsets)]
+    ysr = [torch.empty(B, D, dtype=dt, device=dev) for _ in range(nsets)]
+
+    def chain_rot():
+        for t in range(steps):
+            binding.decode_step(xs[t], params, hs[t % nsets], css[t % nsets], y=ysr[t % nsets], workspace=ws)
+
+    graph_rot = graph_of(chain_rot)
+    us_rot_all = [t / steps for t in event_times_us(graph_rot.replay, reps, torch)]
     Dh = D // H
     dec_bytes = B * D * 2 * 2 + B * D * 4 * 2 + B * 3 * D * 2 + B * D * 2 + (4 * D + 2 * H * Dh * Dh) * 2 + 4 * D * 4
-    out["decode"] = {"workload": f"B={B} D_RNN={D} H={H} bf16 io, fp32 h, {steps} chained steps", "steps_per_s": 1e6 / us,
-                     "tokens_per_s": B * 1e6 / us, "us_per_step_plain_launches": us_plain, "us_per_step_cuda_graph": us_graph,
-                     "algorithmic_bytes_per_step": dec_bytes, "hbm_gbs_achieved": dec_bytes / (us * 1e-6) / 1e9,
-                     "roofline_frac": dec_bytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
+    us_plain, us_graph, us_rot = float(np.median(us_plain_all)), float(np.median(us_graph_all)), float(np.median(us_rot_all))
+    set_mb = (B * D * 4 + B * 3 * D * 2 + B * D * 2) / 1e6
+    out["decode"] = {"workload": f"B={B} D_RNN={D} H={H} bf16 io, fp32 h, {steps} chained steps", "reps": reps,
+                     "algorithmic_bytes_per_step": dec_bytes,
+                     "state_in_hbm": {"what": f"{nsets} rotating state sets ({nsets * set_mb:.0f} MB) > L2, CUDA graph",
+                                      "us_per_step_median": us_rot, "us_per_step_min": float(np.min(us_rot_all)),
+                                      "steps_per_s": 1e6 / us_rot, "tokens_per_s": B * 1e6 / us_rot,
+                                      "hbm_gbs_achieved": dec_bytes / (us_rot * 1e-6) / 1e9,
+                                      "roofline_frac": dec_bytes / (us_rot * 1e-6) / 1e9 / peaks["hbm_gbs"]},
+                     "state_in_l2": {"what": f"one state set ({set_mb:.0f} MB) that stays in L2 between steps, CUDA graph",
+                                     "us_per_step_median": us_graph, "us_per_step_min": float(np.min(us_graph_all)),
+                                     "steps_per_s": 1e6 / us_graph, "tokens_per_s": B * 1e6 / us_graph,
+                                     "hbm_gbs_equivalent": dec_bytes / (us_graph * 1e-6) / 1e9,
+                                     "roofline_frac": dec_bytes / (us_graph * 1e-6) / 1e9 / peaks["hbm_gbs"]},
+                     "us_per_step_plain_launches": us_plain, "us_per_step_plain_launches_min": float(np.min(us_plain_all))}
+    del hs, css, ysr
     del xs, h, cs, y
     # ---- backward
     c4 = synth.CONFIGS[4]
@@ -360,16 +446,63 @@ def measure_extras(binding, dev, peaks):
     shape = binding.make_shape(B, T, D, H, dt)
     ws = binding.alloc_workspace(shape, binding.OP_BACKWARD, dev)
     y_saved, _, _ = binding.prefill(x, params)          # a training step keeps the forward output for the backward
-    binding.backward(x, params, dy, y=y_saved, workspace=ws); torch.cuda.synchronize()
-    e0.record()
-    binding.backward(x, params, dy, y=y_saved, workspace=ws)
-    e1.record(); torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1)
+    for _ in range(2):
+        binding.backward(x, params, dy, y=y_saved, workspace=ws)
+    torch.cuda.synchronize()
+    ms_all = [t * 1e-3 for t in event_times_us(lambda: binding.backward(x, params, dy, y=y_saved, workspace=ws), 20, torch)]
+    ms = float(np.median(ms_all))
     bwd_flops = B * T * D * 12 * Dh
-    out["backward"] = {"workload": f"B={B} T={T} D_RNN={D} H={H} bf16 io, forward output saved", "tokens_per_s": B * T / (ms * 1e-3), "ms": ms,
+    bwd_bytes = B * T * D * 2 * 4
+    out["backward"] = {"workload": f"B={B} T={T} D_RNN={D} H={H} bf16 io, forward output saved", "reps": 20,
+                       "tokens_per_s": B * T / (ms * 1e-3), "ms": ms, "ms_min": float(np.min(ms_all)),
+                       "gate_flops": bwd_flops, "minimum_bytes": bwd_bytes,
                        "gate_tflops_achieved": bwd_flops / (ms * 1e-3) / 1e12,
                        "roofline_frac": bwd_flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
     return out
+
+
+def run_only(args):
+    """One op a few times on a seeded synthetic workload of the given shape; meant to be wrapped in a profiler."""
+    import torch
+    from paper_2402_19427_b200 import binding, build
+    build.build()
+    binding.load()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    dt = torch.bfloat16
+    cfg = dict(synth.CONFIGS[{"prefill": 1, "decode": 3, "backward": 4}[args.only]])
+    B, T, D, H = args.B or cfg["B"], args.T or cfg.get("T", 1), args.D or cfg["D"], args.H or cfg["H"]
+    pr = synth.make_inputs(1, 4, D, H, io="bf16", seed=1)["params"]
+    params = binding.Params.from_numpy(pr, "bf16", device=dev)
+    g = torch.Generator(device=dev); g.manual_seed(0)
+    if args.only == "decode":
+        x = torch.randn(B, D, device=dev, generator=g).to(dt)
+        h = torch.randn(B, D, device=dev, generator=g)
+        cs = torch.randn(B, 3, D, device=dev, generator=g).to(dt)
+        for _ in range(args.iters):
+            binding.decode_step(x, params, h, cs)
+    else:
+        xs = [torch.randn(B, T, D, device=dev, generator=g).to(dt) for _ in range(2)]
+        ys = [torch.empty_like(xs[0]) for _ in range(2)]
+        if args.only == "prefill":
+            shape = binding.make_shape(B, T, D, H, dt)
+            ws = binding.alloc_workspace(shape, binding.OP_PREFILL, dev)
+            for i in range(args.iters):
+                binding.prefill(xs[i % 2], params, y=ys[i % 2], workspace=ws)
+            if binding.query_status(ws) != binding.OK:
+                raise RuntimeError("device status")
+        else:
+            for i in range(args.iters):
+                binding.backward(xs[i % 2], params, ys[0].normal_())
+    torch.cuda.synchronize()
+    print(json.dumps({"only": args.only, "B": B, "T": T, "D": D, "H": H, "iters": args.iters}))
+
+
+def launch_command(args, argv):
+    """The torch.distributed.run command that starts one rank of this script per GPU on this node."""
+    port = int(os.environ.get("MASTER_PORT", "29531"))
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
 
 
 def main():
@@ -378,11 +511,28 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--no-extras", action="store_true", help="skip the decode and backward side measurements")
+    ap.add_argument("--no-extras", action="store_true", help="skip the side measurements (other prefill shapes, decode, backward)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--launch-dry-run", action="store_true", help="print the command that would start the ranks, and this process's rank environment")
+    ap.add_argument("--only", choices=["prefill", "decode", "backward"], help="run one op a few times and exit (for profilers)")
+    ap.add_argument("--B", type=int); ap.add_argument("--T", type=int); ap.add_argument("--D", type=int); ap.add_argument("--H", type=int)
+    ap.add_argument("--iters", type=int, default=3)
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.only:
+        run_only(args)
+        return
+    have_ranks = "RANK" in os.environ and "WORLD_SIZE" in os.environ
+    if args.launch_dry_run:
+        argv = [a for a in sys.argv[1:] if a != "--launch-dry-run"]
+        print(json.dumps({"gpus": args.gpus, "self_launch": args.gpus > 1 and not have_ranks,
+                          "command": launch_command(args, argv) if args.gpus > 1 and not have_ranks else None,
+                          "env": {k: os.environ.get(k) for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}}))
+        return
+    if args.gpus > 1 and not have_ranks:
+        # started as a plain script: become the launcher of one rank per GPU; rank 0 prints the JSON line
+        sys.exit(subprocess.call(launch_command(args, sys.argv[1:])))
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -57,6 +57,10 @@ typedef enum { RGLRU_OP_PREFILL = 0, RGLRU_OP_DECODE = 1, RGLRU_OP_BACKWARD = 2 
 /* flags */
 #define RGLRU_FLAG_NONE 0u
 #define RGLRU_FLAG_FORCE_GENERIC 1u /* use the shape-generic CUDA-core kernels even where a tensor-core kernel exists */
+/* Test hook of the failure path, honoured by the tensor-core rglru_prefill only: tiles that wait for another tile's carry
+ * record look for a tag that is never published, so the bounded wait (rglru_set_wait_limit_ns) runs out, the kernel drains
+ * and returns, and rglru_query_status reports RGLRU_ERR_TIMEOUT.  Outputs are undefined after such a call. */
+#define RGLRU_FLAG_TEST_CARRY_NEVER_ARRIVES 0x40000000u
 
 typedef struct {
     int32_t B;     /* sequences */

@@ -19,6 +19,7 @@ OK, ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALIGN, ERR_WORKSPACE, ERR_CUDA, ER
 F32, BF16 = 0, 1
 OP_PREFILL, OP_DECODE, OP_BACKWARD = 0, 1, 2
 FLAG_NONE, FLAG_FORCE_GENERIC = 0, 1
+FLAG_TEST_CARRY_NEVER_ARRIVES = 0x40000000   # failure-path test hook of the tensor-core prefill (see include/rglru.h)
 
 EXPORTED = ["rglru_abi_version", "rglru_status_string", "rglru_workspace_bytes", "rglru_prefill",
             "rglru_decode_step", "rglru_backward", "rglru_host_staging_bytes", "rglru_prefill_host",
@@ -217,7 +218,7 @@ def decode_step(x, params: Params, h, conv_state, c=8.0, flags=0, y=None, worksp
     return y
 
 
-def backward(x, params: Params, dy, h0=None, conv_state_in=None, y=None, c=8.0, flags=0, workspace=None):
+def backward(x, params: Params, dy, h0=None, conv_state_in=None, y=None, c=8.0, flags=0, workspace=None, out=None):
     """Gradients of sum(dy*y) (rglru_backward): dict with x (io dtype) and fp32 conv_w, conv_b, W_a, b_a, W_x, b_x, lam."""
     lib = load()
     B, T, D = x.shape
@@ -231,6 +232,10 @@ def backward(x, params: Params, dy, h0=None, conv_state_in=None, y=None, c=8.0, 
     g = dict(x=torch.empty_like(x), conv_w=torch.empty(4, D, **f32), conv_b=torch.empty(D, **f32),
              W_a=torch.empty(H, Dh, Dh, **f32), b_a=torch.empty(D, **f32), W_x=torch.empty(H, Dh, Dh, **f32),
              b_x=torch.empty(D, **f32), lam=torch.empty(D, **f32))
+    if out is not None:   # caller-provided gradient buffers (same keys, shapes and dtypes)
+        for k in g:
+            _chk(out[k], tuple(g[k].shape), g[k].dtype, "out[" + k + "]", dev)
+        g = out
     ws = alloc_workspace(shape, OP_BACKWARD, dev) if workspace is None else workspace
     rc = lib.rglru_backward(ctypes.byref(shape), ctypes.byref(params.ptrs), _ptr(x), _ptr(h0), _ptr(conv_state_in),
                             _ptr(y), _ptr(dy), _ptr(g["x"]), _ptr(g["conv_w"]), _ptr(g["conv_b"]), _ptr(g["W_a"]),

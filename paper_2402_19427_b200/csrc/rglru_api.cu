@@ -82,6 +82,7 @@ FwdArgs make_fwd(const rglru_shape_t *s, const rglru_params_t *p) {
     a.B = s->B; a.T = s->T; a.D = s->D; a.H = s->H; a.c = s->c;
     a.conv_w = p->conv_w; a.conv_b = p->conv_b; a.W_a = p->W_a; a.W_x = p->W_x;
     a.b_a = p->b_a; a.b_x = p->b_x; a.lambda = p->lambda;
+    a.flags = s->flags;
     return a;
 }
 

@@ -33,6 +33,7 @@ struct FwdArgs {
     // optional fp32 saves for the backward, each [B,T,D] (null when not saving)
     float *save_u, *save_r, *save_i, *save_hprev;
     uint32_t *status;         // workspace header
+    uint32_t flags;           // RGLRU_FLAG_* of the call
 };
 
 struct BwdArgs {

@@ -75,6 +75,7 @@ struct Sm100Args {
     int tps;           // tiles per sequence
     int tiles_total;   // B * tps
     uint32_t tag;      // validity tag of this call's aggregate records
+    uint32_t tag_wait; // the tag the look-back waits for: `tag`, or a value nobody publishes under the failure-path test flag
     uint4 *agg;        // [H*2][tiles_total][128] records {P, tag, h_loc, tag}
     unsigned long long spin_ns;
 };
@@ -480,7 +481,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
                         }
 #pragma unroll
                         for (int j = 1; j < MAX_S; ++j)
-                            if (j <= nback) ready = ready && r[j - 1].y == p.tag && r[j - 1].w == p.tag;
+                            if (j <= nback) ready = ready && r[j - 1].y == p.tag_wait && r[j - 1].w == p.tag_wait;
                         if (__all_sync(0xffffffffu, ready)) break;
                         if ((npoll & 15u) == 15u) {
                             const uint64_t tnow = gtimer();
@@ -692,6 +693,7 @@ cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes,
     p.S = S;
     p.tiles_total = record_slots(a.B) * p.tps;
     p.tag = next_tag();
+    p.tag_wait = (a.flags & RGLRU_FLAG_TEST_CARRY_NEVER_ARRIVES) ? ~p.tag : p.tag;
     p.agg = (uint4 *)ws_body;
     p.spin_ns = g_spin_limit_ns;
     if (ws_body_bytes < sm100_prefill_workspace_bytes(a.B, a.T, a.D, a.H)) return cudaErrorInvalidValue;

@@ -68,3 +68,32 @@ def gpu_prefill(inp, flags=0, h0=None, cs=None):
 
 def oracle_prefill(oracle, inp, h0=None, cs=None):
     return oracle.prefill(inp["x"].astype(np.float64), f64(inp["params"]), inp["H"], c=inp["c"], h0=h0, conv_state_in=cs)
+
+
+class Guarded:
+    """Output buffers carved out of a larger allocation with canary bytes before and after each: the device code builds
+    addresses by hand (swizzled tiles, clipped tiled stores), and the memory checker is closed on this machine, so every call
+    that writes an output is followed by a check that the bytes around it are untouched."""
+    PAD = 4096   # bytes on each side; a multiple of every alignment the library asks for
+    FILL = 0xA5
+
+    def __init__(self, device="cuda"):
+        self.device = device
+        self.items = []
+
+    def empty(self, shape, dtype):
+        import torch
+        n = int(np.prod(shape)) * torch.empty(0, dtype=dtype).element_size()
+        body = (n + 255) // 256 * 256
+        raw = torch.full((self.PAD + body + self.PAD,), self.FILL, dtype=torch.uint8, device=self.device)
+        view = raw[self.PAD:self.PAD + n].view(dtype).view(*shape)
+        self.items.append((raw, n))
+        return view
+
+    def check(self):
+        import torch
+        torch.cuda.synchronize()
+        for k, (raw, n) in enumerate(self.items):
+            head, tail = raw[:self.PAD], raw[self.PAD + n:]
+            assert bool((head == self.FILL).all()), f"guard bytes before output {k} were overwritten"
+            assert bool((tail == self.FILL).all()), f"guard bytes after output {k} were overwritten"

@@ -4,7 +4,7 @@
  * The library computes the temporal core of the Griffin/Hawk recurrent block:
  * a causal depthwise Conv1D of temporal width 4 (Section 2.3, "Recurrent block"),
  * followed by the RG-LRU layer (Section 2.4, Eq. 1-4) with the decay evaluated in
- * log space (Appendix A) and block-diagonal gate matrices (Section 3.1):
+ * log space (Appendix A) and block-diagonal gate matrices (Section 4.1, "Model parallelism", paragraph "Recurrent Block"):
  *
  *     u_t = b_c + sum_{j=0..3} w[j] * x_{t-j}                 (Conv1D, tap j hits x_{t-j})
  *     r_t = sigmoid(W_a u_t + b_a)                            (Eq. 1)
@@ -97,7 +97,7 @@ size_t rglru_workspace_bytes(const rglru_shape_t *shape, int32_t op);
 
 /*
  * Forward over T tokens (Conv1D + Eq. 1-4), also the inference prefill: returns the state
- * that a later rglru_prefill or rglru_decode_step continues from (Appendix E.4.2: the
+ * that a later rglru_prefill or rglru_decode_step continues from (Appendix F.4, "Cache sizes": the
  * recurrent state has size D_RNN, the convolution state (4-1) D_RNN per sequence).
  *   x              [B,T,D] io, in
  *   h0             [B,D] fp32, in, or NULL for a zero state
@@ -111,12 +111,18 @@ int32_t rglru_prefill(const rglru_shape_t *shape, const rglru_params_t *params, 
                       size_t workspace_bytes, void *cuda_stream);
 
 /*
- * One decode step for B sequences (Section 3.3 / Appendix E.4.2): the T = 1 case of the
+ * One decode step for B sequences (Section 5.1, "A simple model of the decode step", and Appendix F.4): the T = 1 case of the
  * forward with the state updated in place.
  *   x          [B,D] io, in
  *   h          [B,D] fp32, in/out
  *   conv_state [B,3,D] io, in/out: rows shift by one (bit-exact) and x becomes row 2
  *   y          [B,D] io, out
+ * The tensor-core kernel is launched so that it may start while the preceding kernel on the stream is still finishing
+ * (programmatic dependent launch): it reads the parameters (conv_w, conv_b, W_a, b_a, W_x, b_x, lambda) before it waits
+ * for that kernel, and x, h and conv_state after.  A kernel that writes the parameters (a cast, an optimiser step) must
+ * therefore not be the one directly before this call on the stream; put any other work, or an event, in between.
+ * After RGLRU_ERR_TIMEOUT (rglru_query_status) h and conv_state are undefined: conv_state may already hold the shifted rows
+ * while h has not been advanced.
  */
 int32_t rglru_decode_step(const rglru_shape_t *shape, const rglru_params_t *params, const void *x, float *h,
                           void *conv_state, void *y, void *workspace, size_t workspace_bytes, void *cuda_stream);
@@ -144,7 +150,9 @@ int32_t rglru_backward(const rglru_shape_t *shape, const rglru_params_t *params,
  * conv_state_out are copied back to the host pointers; the call returns without synchronising and work
  * enqueued on `cuda_stream` afterwards sees the results.  The batch is cut into chunks of sequences whose
  * host-to-device copy, forward and device-to-host copy overlap on two internal streams (created on first use
- * per device); calls on one device must not be made from several host threads at once.
+ * per device); calls on one device must not be made from several host threads at once.  These two streams and the
+ * events that tie them to `cuda_stream` are the one thing the library creates and keeps (per device, until the process
+ * exits): the rule above that nothing is allocated or retained holds for device memory, not for them.
  * params, h0, conv_state_in, staging and workspace are device pointers.
  *   staging : device scratch of at least rglru_host_staging_bytes(shape) bytes, 256-byte aligned.
  */

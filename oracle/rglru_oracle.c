@@ -5,7 +5,7 @@
  * Griffin/Hawk recurrent block: causal depthwise Conv1D of temporal width 4
  * (Section 2.3, "Recurrent block") followed by the RG-LRU layer (Section 2.4,
  * Eq. 1-4), with the decay evaluated in log space (Appendix A) and the gate
- * matrices block-diagonal per head (Section 3.1, "Recurrent Block").
+ * matrices block-diagonal per head (Section 4.1, paragraph "Recurrent Block").
  *
  * Only the tests, the smoke check and the benchmark's CPU-baseline leg may
  * load this file.  It shares no code, header, table or helper with the CUDA
@@ -146,7 +146,7 @@ int oracle_prefill(int B, int T, int D, int H, double c, const double *x, const 
 }
 
 /*
- * One decode step for B sequences (Appendix E.4.2: the carried state is h, size D_RNN,
+ * One decode step for B sequences (Appendix F.4, "Cache sizes": the carried state is h, size D_RNN,
  * and the last 4-1 = 3 conv inputs).  Written from the state definition, not by calling
  * the prefill: h [B,D] and conv_state [B,3,D] are updated in place, y [B,D] is written.
  */

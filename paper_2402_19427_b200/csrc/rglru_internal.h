@@ -7,9 +7,31 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "rglru.h"
 
 namespace rglru {
+
+// Function attributes belong to a device's context, so the opt-in to more than 48 KB of dynamic shared memory has to be made
+// once per device (with that device current), not once per process.  Thread-safe; `T` is a kernel function pointer type.
+struct PerDeviceOptIn {
+    std::mutex mutex;
+    bool done[64] = {};
+    template <typename T> cudaError_t ensure(T kernel, int smem_bytes) {
+        int dev = -1;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+        std::lock_guard<std::mutex> lock(mutex);
+        if (!done[dev]) {
+            e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+            if (e != cudaSuccess) return e;
+            done[dev] = true;
+        }
+        return cudaSuccess;
+    }
+};
 
 // The first 256 bytes of every workspace hold the device-side status: word 0 carries
 // STATUS_MAGIC | code once a kernel has recorded a condition.  A word without the magic

@@ -600,13 +600,9 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
     const int B = q.B, T = q.T, D = q.D, H = q.H;
     const BwdLayout L = bwd_layout(B, T, D, H);
     if (ws_body_bytes < L.total) return cudaErrorInvalidValue;
-    static bool attr_set = false;
-    cudaError_t e;
-    if (!attr_set) {
-        e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_ALLOC);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static PerDeviceOptIn opt_in;
+    cudaError_t e = opt_in.ensure(tc_gemm_kernel, (int)GEMM_SMEM_ALLOC);
+    if (e != cudaSuccess) return e;
     char *ws = (char *)ws_body;
     __half *u = (__half *)(ws + L.off_u), *uT = (__half *)(ws + L.off_uT), *z = (__half *)(ws + L.off_z);
     __half *dz = (__half *)(ws + L.off_dz), *dzT = (__half *)(ws + L.off_dzT), *WT = (__half *)(ws + L.off_wt), *W16 = (__half *)(ws + L.off_w16);

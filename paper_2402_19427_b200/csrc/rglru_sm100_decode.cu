@@ -299,13 +299,9 @@ int num_sms() {
 bool sm100_decode_supported(int B, int D, int H, int io) { return io == RGLRU_BF16 && B > 0 && H > 0 && D == H * DH; }
 
 cudaError_t sm100_decode(const FwdArgs &a, cudaStream_t st) {
-    static bool attr_set = false;
-    cudaError_t e;
-    if (!attr_set) {
-        e = cudaFuncSetAttribute(sm100_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static PerDeviceOptIn opt_in;
+    cudaError_t e = opt_in.ensure(sm100_decode_kernel, (int)SMEM_ALLOC);
+    if (e != cudaSuccess) return e;
     DecArgs p;
     if (!encode_bf16_map_3d(&p.tm_wa, a.W_a, DH, DH, (uint64_t)a.H, 64, CH, true) ||
         !encode_bf16_map_3d(&p.tm_wx, a.W_x, DH, DH, (uint64_t)a.H, 64, CH, true))

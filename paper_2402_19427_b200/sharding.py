@@ -1,6 +1,6 @@
 """Partitioning of the temporal core across ranks.  No data-path collective exists: sequences are independent,
 and channels are independent outside a gate block (block-diagonal W_a / W_x, depthwise conv, diagonal recurrence;
-Section 3.1 of the paper), so a rank owns whole sequences or whole heads and never exchanges activations.
+Section 4.1 of the paper, "Model parallelism"), so a rank owns whole sequences or whole heads and never exchanges activations.
 The only reductions are bookkeeping (the maximum of the per-rank step time).  numpy / torch.distributed only.
 """
 from __future__ import annotations

@@ -41,7 +41,7 @@ def _load():
         lib.oracle_prefill.restype = ctypes.c_int
         lib.oracle_decode_step.argtypes = [ctypes.c_int] * 3 + [ctypes.c_double] + [_dp] * 11
         lib.oracle_decode_step.restype = ctypes.c_int
-        lib.oracle_backward.argtypes = [ctypes.c_int] * 4 + [ctypes.c_double] + [_dp] * 19
+        lib.oracle_backward.argtypes = [ctypes.c_int] * 4 + [ctypes.c_double] + [_dp] * 23
         lib.oracle_backward.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -114,8 +114,9 @@ def decode_step(x, params, H, h, conv_state, c=8.0):
     return y, h, cs
 
 
-def backward(x, params, H, dy, c=8.0, h0=None, conv_state_in=None):
-    """Gradients of sum(dy*y) w.r.t. x and every parameter; returns a dict keyed like ``params`` plus 'x'."""
+def backward(x, params, H, dy, c=8.0, h0=None, conv_state_in=None, dh_T=None, dconv_state_out=None, state_grads=False):
+    """Gradients of sum(dy*y) [+ sum(dh_T*h_T) + sum(dconv_state_out*conv_state_out)] w.r.t. x and every parameter; returns
+    a dict keyed like ``params`` plus 'x', and with ``state_grads`` also 'h0' [B,D] and 'conv_state' [B,3,D]."""
     x = np.ascontiguousarray(x, dtype=np.float64)
     B, T, D = x.shape
     Dh = D // H
@@ -126,9 +127,14 @@ def backward(x, params, H, dy, c=8.0, h0=None, conv_state_in=None):
     out = {"x": np.empty((B, T, D)), "conv_w": np.empty((4, D)), "conv_b": np.empty((D,)),
            "W_a": np.empty((H, Dh, Dh)), "b_a": np.empty((D,)), "W_x": np.empty((H, Dh, Dh)),
            "b_x": np.empty((D,)), "lam": np.empty((D,))}
+    if state_grads:
+        out["h0"] = np.empty((B, D)); out["conv_state"] = np.empty((B, 3, D))
     P = {k: v.ctypes.data_as(_dp) for k, v in out.items()}
+    dha, dhp = _in(dh_T, (B, D))
+    dca, dcp = _in(dconv_state_out, (B, 3, D))
     rc = _load().oracle_backward(B, T, D, H, float(c), x.ctypes.data_as(_dp), cw, cb, Wa, ba, Wx, bx, lam, h0p, csp, dyp,
-                                 P["x"], P["conv_w"], P["conv_b"], P["W_a"], P["b_a"], P["W_x"], P["b_x"], P["lam"])
+                                 P["x"], P["conv_w"], P["conv_b"], P["W_a"], P["b_a"], P["W_x"], P["b_x"], P["lam"],
+                                 dhp, dcp, P.get("h0"), P.get("conv_state"))
     if rc != 0:
         raise ValueError("oracle_backward: bad shape")
     return out

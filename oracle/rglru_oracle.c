@@ -189,11 +189,14 @@ int oracle_decode_step(int B, int D, int H, double c, const double *x, const dou
 }
 
 /*
- * Backward of oracle_prefill for the scalar  loss = sum(dy * y)  (upstream gradient dy only;
- * no gradient arrives through h_T or conv_state_out).  The paper gives no backward; this is
- * reverse-mode differentiation of Eq. 1-4 and of the Conv1D, written out:
+ * Backward of oracle_prefill for the scalar
+ *     loss = sum(dy * y) + sum(dh_T * h_T) + sum(dconv_state_out * conv_state_out)
+ * (the last two terms only when the pointers are given: they are what flows back from a later segment of the same sequence
+ * through the state this segment handed on, so that a sequence can be differentiated segment by segment).  The paper gives
+ * no backward; this is reverse-mode differentiation of Eq. 1-4 and of the Conv1D, written out:
  *
- *   g_t   = dy_t + a_{t+1} g_{t+1}                     (adjoint of h_t; g beyond T is 0)
+ *   g_t   = dy_t + a_{t+1} g_{t+1}                     (adjoint of h_t; beyond the last token g is dh_T, carried with factor 1
+ *                                                       because h_T = h_{T-1}; 0 when dh_T is not given)
  *   dL_t  = g_t (a_t h_{t-1} - a_t^2 v_t / m_t)        (L_t = log a_t, v_t = i_t u_t, m_t = sqrt(1-a_t^2);
  *                                                       the second term is taken as 0 when m_t = 0)
  *   dv_t  = g_t m_t ;  di_t = dv_t u_t ;  du_t += dv_t i_t
@@ -201,14 +204,20 @@ int oracle_decode_step(int B, int D, int H, double c, const double *x, const dou
  *   dz_a  = dr r (1-r) ;  dz_x = di i (1-i) ;  db += dz ;  dW[k][o][n] += dz[o] u[n]
  *   du_t += W_a[k]^T dz_a + W_x[k]^T dz_x
  *   dx_t  = sum_j w[j] du_{t+j} (t+j < T) ;  dw[j] += du_t x_{t-j} ;  db_c += du_t
+ *   dh0   = a_0 g_0                                    (h_{-1} = h0 enters Eq. 4 only at t = 0)
+ *   dconv_state_in[r] = sum_j w[j] du_{r-3+j} (0 <= r-3+j < T)      (row r is x_{r-3}: the same formula as dx, at t < 0)
+ *   conv_state_out is a copy of the last three rows of concat(conv_state_in, x): dconv_state_out[k] is added to the
+ *   gradient of that row (dx_{T-3+k}, or dconv_state_in[T+k] when T+k < 3).
  *
  * All parameter gradients are overwritten (summed over batch and time).
  *   dx [B,T,D]; dconv_w [4,D]; dconv_b [D] (or NULL to skip); dW_a, dW_x [H,Dh,Dh]; db_a, db_x, dlambda [D].
+ *   dh_T [B,D], dconv_state_out [B,3,D]: in, or NULL for zero.  dh0 [B,D], dconv_state_in [B,3,D]: out, or NULL to skip.
  */
 int oracle_backward(int B, int T, int D, int H, double c, const double *x, const double *conv_w, const double *conv_b,
                     const double *W_a, const double *b_a, const double *W_x, const double *b_x, const double *lambda,
                     const double *h0, const double *conv_state_in, const double *dy, double *dx, double *dconv_w,
-                    double *dconv_b, double *dW_a, double *db_a, double *dW_x, double *db_x, double *dlambda) {
+                    double *dconv_b, double *dW_a, double *db_a, double *dW_x, double *db_x, double *dlambda,
+                    const double *dh_T, const double *dconv_state_out, double *dh0, double *dconv_state_in) {
     if (B <= 0 || T <= 0 || D <= 0 || H <= 0 || D % H != 0) return -1;
     const int Dh = D / H;
     memset(dconv_w, 0, sizeof(double) * 4 * D);
@@ -247,13 +256,13 @@ int oracle_backward(int B, int T, int D, int H, double c, const double *x, const
                 }
             }
             /* reverse sweep */
-            for (int n = 0; n < Dh; ++n) g[n] = 0.0;
+            for (int n = 0; n < Dh; ++n) g[n] = dh_T ? dh_T[(size_t)b * D + d0 + n] : 0.0;
             for (int t = T - 1; t >= 0; --t) {
                 double *ut = u + (size_t)t * Dh, *dut = du + (size_t)t * Dh;
                 for (int n = 0; n < Dh; ++n) {
                     size_t e = (size_t)t * Dh + n;
                     int d = d0 + n;
-                    double a_next = (t + 1 < T) ? a[e + Dh] : 0.0;
+                    double a_next = (t + 1 < T) ? a[e + Dh] : 1.0;   /* past the end g holds dh_T (or 0) */
                     g[n] = dy[((size_t)b * T + t) * D + d] + a_next * g[n];
                     double v = gi[e] * ut[n];
                     double dm_term = (m[e] > 0.0) ? a[e] * a[e] * v / m[e] : 0.0;
@@ -279,6 +288,8 @@ int oracle_backward(int B, int T, int D, int H, double c, const double *x, const
                     }
                 }
             }
+            if (dh0)
+                for (int n = 0; n < Dh; ++n) dh0[(size_t)b * D + d0 + n] = a[n] * g[n];   /* a_0 g_0 */
             /* Conv1D backward */
             for (int t = 0; t < T; ++t) {
                 for (int n = 0; n < Dh; ++n) {
@@ -290,6 +301,29 @@ int oracle_backward(int B, int T, int D, int H, double c, const double *x, const
                     for (int j = 0; j < CONV_WIDTH; ++j) dconv_w[(size_t)j * D + d] += dut * x_at(x, conv_state_in, T, D, b, t - j, d);
                     if (dconv_b) dconv_b[d] += dut;
                 }
+            }
+            /* the carried inputs x_{-3..-1}, and what arrives through the copies in conv_state_out */
+            if (dconv_state_in) {
+                for (int r = 0; r < CONV_WIDTH - 1; ++r)
+                    for (int n = 0; n < Dh; ++n) {
+                        int d = d0 + n;
+                        double acc = 0.0;
+                        for (int j = 0; j < CONV_WIDTH; ++j) {
+                            int t = r - (CONV_WIDTH - 1) + j;
+                            if (t >= 0 && t < T) acc += conv_w[(size_t)j * D + d] * du[(size_t)t * Dh + n];
+                        }
+                        dconv_state_in[((size_t)b * (CONV_WIDTH - 1) + r) * D + d] = acc;
+                    }
+            }
+            if (dconv_state_out) {
+                for (int k2 = 0; k2 < CONV_WIDTH - 1; ++k2)
+                    for (int n = 0; n < Dh; ++n) {
+                        int d = d0 + n;
+                        double gk = dconv_state_out[((size_t)b * (CONV_WIDTH - 1) + k2) * D + d];
+                        int row = T + k2;                       /* row of concat(conv_state_in, x) that was copied */
+                        if (row >= CONV_WIDTH - 1) dx[((size_t)b * T + (row - (CONV_WIDTH - 1))) * D + d] += gk;
+                        else if (dconv_state_in) dconv_state_in[((size_t)b * (CONV_WIDTH - 1) + row) * D + d] += gk;
+                    }
             }
         }
         free(u);

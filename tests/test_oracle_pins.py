@@ -323,6 +323,77 @@ def test_backward_overwrites_and_is_additive_in_batch(oracle):
     np.testing.assert_allclose(g["x"], np.concatenate([q["x"] for q in parts], 0), rtol=0, atol=0)
 
 
+def loss_with_state(oracle, x, p, H, dy, h0, cs, dhT, dcs):
+    y, hT, cso = oracle.prefill(x, p, H=H, h0=h0, conv_state_in=cs)
+    return float(np.sum(dy * y) + np.sum(dhT * hT) + np.sum(dcs * cso))
+
+
+@pytest.mark.parametrize("shape", [dict(B=2, T=33, D=16, H=2), dict(B=1, T=2, D=6, H=3), dict(B=2, T=1, D=4, H=1)])
+def test_backward_state_gradients_central_differences(oracle, shape):
+    """dh0 and d conv_state_in, with gradient arriving through h_T and conv_state_out as well (the terms a later segment of
+    the sequence sends back): central differences of loss = <dy,y> + <dh_T,h_T> + <dcs_out,cs_out> in fp64.  T = 1, 2: the
+    conv state is partly a copy of the incoming one, so part of dcs_out passes straight through."""
+    rng = np.random.default_rng(21)
+    B, T, D, H = shape["B"], shape["T"], shape["D"], shape["H"]
+    x, p, h0, cs = rand_problem(22, B=B, T=T, D=D, H=H, scale_w=1.0 / math.sqrt(D // H))
+    p["lam"] = rng.uniform(0.5, 5.0, size=D)
+    dy = rng.normal(size=(B, T, D)); dhT = rng.normal(size=(B, D)); dcs = rng.normal(size=(B, 3, D))
+    g = oracle.backward(x, p, H, dy, h0=h0, conv_state_in=cs, dh_T=dhT, dconv_state_out=dcs, state_grads=True)
+    eps = 1e-6
+
+    def fd(arr, idx):
+        old = arr[idx]
+        arr[idx] = old + eps; lp = loss_with_state(oracle, x, p, H, dy, h0, cs, dhT, dcs)
+        arr[idx] = old - eps; lm = loss_with_state(oracle, x, p, H, dy, h0, cs, dhT, dcs)
+        arr[idx] = old
+        return (lp - lm) / (2 * eps)
+
+    for name, arr, grad in (("h0", h0, g["h0"]), ("conv_state", cs, g["conv_state"]), ("x", x, g["x"]), ("lam", p["lam"], g["lam"]),
+                            ("conv_w", p["conv_w"], g["conv_w"]), ("W_a", p["W_a"], g["W_a"])):
+        scale = np.abs(grad).max() + 1e-30
+        for fi in rng.choice(arr.size, size=min(8, arr.size), replace=False):
+            idx = np.unravel_index(fi, arr.shape)
+            num = fd(arr, idx)
+            assert abs(num - grad[idx]) <= 2e-6 * scale + 1e-7 * abs(num), (name, idx, num, grad[idx])
+    # every row of the carried conv inputs, first and last channel
+    for idx in [(0, 0, 0), (0, 1, D - 1), (B - 1, 2, 0)]:
+        assert abs(fd(cs, idx) - g["conv_state"][idx]) <= 2e-6 * (np.abs(g["conv_state"]).max() + 1e-30)
+
+
+def test_backward_without_incoming_state_gradient_is_unchanged_and_dh0_is_the_decay_product(oracle):
+    rng = np.random.default_rng(23)
+    x, p, h0, cs = rand_problem(24, B=2, T=12, D=8, H=2)
+    dy = rng.normal(size=x.shape)
+    g0 = oracle.backward(x, p, 2, dy, h0=h0, conv_state_in=cs)
+    g1 = oracle.backward(x, p, 2, dy, h0=h0, conv_state_in=cs, state_grads=True)
+    for k in g0:
+        assert np.array_equal(g0[k], g1[k])
+    # gates do not see h (Eq. 1-3), so y_t depends on h0 only through prod_{k<=t} a_k: dh0 = sum_t dy_t prod_{k<=t} a_k
+    y1, _, _ = oracle.prefill(x, p, H=2, h0=h0 + 1.0, conv_state_in=cs)
+    y0, _, _ = oracle.prefill(x, p, H=2, h0=h0, conv_state_in=cs)
+    np.testing.assert_allclose(g1["h0"], np.sum(dy * (y1 - y0), axis=1), rtol=1e-10, atol=1e-12)
+
+
+@pytest.mark.parametrize("T1,T2", [(7, 9), (1, 5), (2, 2), (6, 1)])
+def test_backward_of_two_chained_segments_equals_one_segment(oracle, T1, T2):
+    """Truncated segments compose: the second segment's dh0 and d conv_state_in are the first segment's dh_T and
+    d conv_state_out; dx concatenates, parameter gradients add, and the first segment's state gradients are the whole's."""
+    rng = np.random.default_rng(25)
+    B, D, H = 2, 8, 2
+    x, p, h0, cs = rand_problem(26, B=B, T=T1 + T2, D=D, H=H)
+    dy = rng.normal(size=x.shape); dhT = rng.normal(size=(B, D)); dcs = rng.normal(size=(B, 3, D))
+    whole = oracle.backward(x, p, H, dy, h0=h0, conv_state_in=cs, dh_T=dhT, dconv_state_out=dcs, state_grads=True)
+    _, h1, cs1 = oracle.prefill(x[:, :T1], p, H=H, h0=h0, conv_state_in=cs)
+    g2 = oracle.backward(x[:, T1:], p, H, dy[:, T1:], h0=h1, conv_state_in=cs1, dh_T=dhT, dconv_state_out=dcs, state_grads=True)
+    g1 = oracle.backward(x[:, :T1], p, H, dy[:, :T1], h0=h0, conv_state_in=cs, dh_T=g2["h0"], dconv_state_out=g2["conv_state"],
+                         state_grads=True)
+    np.testing.assert_allclose(np.concatenate([g1["x"], g2["x"]], 1), whole["x"], rtol=1e-10, atol=1e-12)
+    for k in p:
+        np.testing.assert_allclose(g1[k] + g2[k], whole[k], rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(g1["h0"], whole["h0"], rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(g1["conv_state"], whole["conv_state"], rtol=1e-10, atol=1e-12)
+
+
 # ---------------------------------------------------------------- the synthetic input recipe
 def test_input_generator_is_seeded_and_bf16_exact():
     a = synth.make_inputs(2, 16, 32, 2, io="bf16", seed=5, long_memory_frac=0.25, with_dy=True, with_state=True)

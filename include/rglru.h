@@ -130,19 +130,35 @@ int32_t rglru_decode_step(const rglru_shape_t *shape, const rglru_params_t *para
 /*
  * Backward of rglru_prefill for an upstream gradient dy on y (the paper states no backward;
  * this is reverse-mode differentiation of Eq. 1-4 and the Conv1D: a reverse-time scan
- * g_t = dy_t + a_{t+1} g_{t+1} followed by the gate and convolution adjoints).  No gradient
- * flows in through h_T or conv_state_out, none is returned for h0 or conv_state_in.
+ * g_t = dy_t + a_{t+1} g_{t+1} followed by the gate and convolution adjoints).  With
+ * `state` given, the call also differentiates through the carried state, so that a sequence cut
+ * into segments (truncated back-propagation through time, Section 7) is differentiated segment by
+ * segment, last segment first: what a segment returns in dh0 and dconv_state_in is what the segment
+ * before it takes as dh_T and dconv_state_out.
  *   x, h0, conv_state_in : as given to the forward
  *   y              [B,T,D] io, the forward output, or NULL (the state is then recomputed)
  *   dy             [B,T,D] io, in
  *   dx             [B,T,D] io, out; must not overlap x, y or dy
  *   dconv_w [4,D], dconv_b [D] (may be NULL), dW_a, dW_x [H,D_h,D_h], db_a, db_x, dlambda [D]:
  *                  fp32, out, overwritten (not accumulated), summed over batch and time.
+ *   state          NULL (no gradient through the state), or a struct of four device pointers, each of which may be NULL:
+ *       dh_T            [B,D] fp32, in: gradient arriving on h_T
+ *       dconv_state_out [B,3,D] io, in: gradient arriving on conv_state_out (a copy of the last three rows of
+ *                       concat(conv_state_in, x), so it is added to the gradient of the rows it copies)
+ *       dh0             [B,D] fp32, out: gradient of h0 (= a_0 g_0)
+ *       dconv_state_in  [B,3,D] io, out: gradient of the three carried inputs x_{-3..-1}
  */
+typedef struct rglru_state_grads {
+    const float *dh_T;
+    const void *dconv_state_out;
+    float *dh0;
+    void *dconv_state_in;
+} rglru_state_grads_t;
+
 int32_t rglru_backward(const rglru_shape_t *shape, const rglru_params_t *params, const void *x, const float *h0,
                        const void *conv_state_in, const void *y, const void *dy, void *dx, float *dconv_w,
                        float *dconv_b, float *dW_a, float *db_a, float *dW_x, float *db_x, float *dlambda,
-                       void *workspace, size_t workspace_bytes, void *cuda_stream);
+                       const rglru_state_grads_t *state, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * rglru_prefill for callers whose activations live in HOST memory (pinned memory makes the

@@ -65,7 +65,7 @@ def load() -> ctypes.CDLL:
         lib.rglru_prefill.restype = i32
         lib.rglru_decode_step.argtypes = [sp, pp] + [vp] * 5 + [sz, vp]
         lib.rglru_decode_step.restype = i32
-        lib.rglru_backward.argtypes = [sp, pp] + [vp] * 14 + [sz, vp]
+        lib.rglru_backward.argtypes = [sp, pp] + [vp] * 15 + [sz, vp]
         lib.rglru_backward.restype = i32
         lib.rglru_host_staging_bytes.argtypes = [sp]
         lib.rglru_host_staging_bytes.restype = sz
@@ -218,8 +218,14 @@ def decode_step(x, params: Params, h, conv_state, c=8.0, flags=0, y=None, worksp
     return y
 
 
-def backward(x, params: Params, dy, h0=None, conv_state_in=None, y=None, c=8.0, flags=0, workspace=None, out=None):
-    """Gradients of sum(dy*y) (rglru_backward): dict with x (io dtype) and fp32 conv_w, conv_b, W_a, b_a, W_x, b_x, lam."""
+class StateGrads(ctypes.Structure):
+    _fields_ = [("dh_T", ctypes.c_void_p), ("dconv_state_out", ctypes.c_void_p), ("dh0", ctypes.c_void_p), ("dconv_state_in", ctypes.c_void_p)]
+
+
+def backward(x, params: Params, dy, h0=None, conv_state_in=None, y=None, c=8.0, flags=0, workspace=None, out=None,
+             dh_T=None, dconv_state_out=None, state_grads=False):
+    """Gradients of sum(dy*y) [+ sum(dh_T*h_T) + sum(dconv_state_out*conv_state_out)] (rglru_backward): dict with x (io dtype)
+    and fp32 conv_w, conv_b, W_a, b_a, W_x, b_x, lam; with ``state_grads`` also h0 [B,D] fp32 and conv_state [B,3,D] io."""
     lib = load()
     B, T, D = x.shape
     H, Dh = params.H, D // params.H
@@ -237,9 +243,17 @@ def backward(x, params: Params, dy, h0=None, conv_state_in=None, y=None, c=8.0, 
             _chk(out[k], tuple(g[k].shape), g[k].dtype, "out[" + k + "]", dev)
         g = out
     ws = alloc_workspace(shape, OP_BACKWARD, dev) if workspace is None else workspace
+    _chk(dh_T, (B, D), torch.float32, "dh_T", dev); _chk(dconv_state_out, (B, 3, D), x.dtype, "dconv_state_out", dev)
+    sg = None
+    if state_grads or dh_T is not None or dconv_state_out is not None:
+        if state_grads and (out is None or "h0" not in out):
+            g["h0"] = torch.empty(B, D, **f32); g["conv_state"] = torch.empty(B, 3, D, dtype=x.dtype, device=dev)
+        vp = lambda t: None if t is None else t.data_ptr()
+        sg = StateGrads(vp(dh_T), vp(dconv_state_out), vp(g.get("h0")), vp(g.get("conv_state")))
     rc = lib.rglru_backward(ctypes.byref(shape), ctypes.byref(params.ptrs), _ptr(x), _ptr(h0), _ptr(conv_state_in),
                             _ptr(y), _ptr(dy), _ptr(g["x"]), _ptr(g["conv_w"]), _ptr(g["conv_b"]), _ptr(g["W_a"]),
-                            _ptr(g["b_a"]), _ptr(g["W_x"]), _ptr(g["b_x"]), _ptr(g["lam"]), _ptr(ws), ws.numel(), _stream())
+                            _ptr(g["b_a"]), _ptr(g["W_x"]), _ptr(g["b_x"]), _ptr(g["lam"]),
+                            ctypes.byref(sg) if sg is not None else None, _ptr(ws), ws.numel(), _stream())
     if rc != OK:
         raise RglruError(rc, "rglru_backward")
     return g

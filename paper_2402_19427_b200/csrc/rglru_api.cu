@@ -90,7 +90,7 @@ FwdArgs make_fwd(const rglru_shape_t *s, const rglru_params_t *p) {
 
 extern "C" {
 
-int32_t rglru_abi_version(void) { return 100; }
+int32_t rglru_abi_version(void) { return 101; }
 
 const char *rglru_status_string(int32_t status) {
     switch (status) {
@@ -178,7 +178,7 @@ int32_t rglru_decode_step(const rglru_shape_t *s, const rglru_params_t *p, const
 int32_t rglru_backward(const rglru_shape_t *s, const rglru_params_t *p, const void *x, const float *h0,
                        const void *conv_state_in, const void *y, const void *dy, void *dx, float *dconv_w,
                        float *dconv_b, float *dW_a, float *db_a, float *dW_x, float *db_x, float *dlambda,
-                       void *workspace, size_t workspace_bytes, void *cuda_stream) {
+                       const rglru_state_grads_t *state, void *workspace, size_t workspace_bytes, void *cuda_stream) {
     int32_t rc = check_shape(s, true);
     if (rc != RGLRU_OK) return rc;
     if ((rc = check_params(p)) != RGLRU_OK) return rc;
@@ -186,6 +186,9 @@ int32_t rglru_backward(const rglru_shape_t *s, const rglru_params_t *p, const vo
     if (!aligned(x, 16) || !aligned(dy, 16) || !aligned(dx, 16) || !aligned(y, 16) || !aligned(h0, 16) ||
         !aligned(conv_state_in, 16) || !aligned(dconv_w, 16) || !aligned(dconv_b, 16) || !aligned(dW_a, 16) ||
         !aligned(db_a, 16) || !aligned(dW_x, 16) || !aligned(db_x, 16) || !aligned(dlambda, 16) || !aligned(workspace, 256))
+        return RGLRU_ERR_ALIGN;
+    if (state && (!aligned(state->dh_T, 16) || !aligned(state->dconv_state_out, 16) || !aligned(state->dh0, 16) ||
+                  !aligned(state->dconv_state_in, 16)))
         return RGLRU_ERR_ALIGN;
     if (workspace_bytes < rglru_workspace_bytes(s, RGLRU_OP_BACKWARD)) return RGLRU_ERR_WORKSPACE;
     const size_t nbytes = (size_t)s->B * s->T * s->D * io_bytes(s->io);
@@ -199,6 +202,7 @@ int32_t rglru_backward(const rglru_shape_t *s, const rglru_params_t *p, const vo
     q.x = x; q.conv_w = p->conv_w; q.W_a = p->W_a; q.W_x = p->W_x; q.cs_in = conv_state_in; q.dy = dy;
     q.lambda = p->lambda; q.dx = dx;
     q.dconv_w = dconv_w; q.dconv_b = dconv_b; q.dW_a = dW_a; q.db_a = db_a; q.dW_x = dW_x; q.db_x = db_x; q.dlambda = dlambda;
+    if (state) { q.dh_T = state->dh_T; q.dcs_out = state->dconv_state_out; q.dh0 = state->dh0; q.dcs_in = state->dconv_state_in; }
     cudaError_t e;
     if (use_sm100_backward(s))
         e = sm100_backward(f, q, y, (char *)workspace + WS_HEADER_BYTES, workspace_bytes - WS_HEADER_BYTES, (uint32_t *)workspace,

@@ -4,6 +4,7 @@
 // backward.  One block walks one (sequence, head) pair through time; the gate products
 // W_a u, W_x u (Eq. 1-2) run on FP32 FMAs with the weights staged through shared memory.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "rglru_internal.h"
 
@@ -229,7 +230,8 @@ __global__ void __launch_bounds__(NT) generic_bwd_scan_kernel(BwdArgs q) {
     const float lam = q.lambda[d];
     const float s = decay_rate(lam, q.c);
     const float dsdlam_neg = q.c * sigmoid_acc(-lam);  // dL/dLambda = c r sigmoid(-Lambda)
-    float g = 0.0f, a_next = 0.0f, s_lam = 0.0f, s_ba = 0.0f, s_bx = 0.0f;
+    // past the last token g holds the gradient arriving on h_T (h_T = h_{T-1}, so it is carried with factor 1)
+    float g = q.dh_T ? q.dh_T[(size_t)b * D + d] : 0.0f, a_next = 1.0f, s_lam = 0.0f, s_ba = 0.0f, s_bx = 0.0f;
     for (int t = T - 1; t >= 0; --t) {
         size_t e = ((size_t)b * T + t) * D + d;
         float r = q.r[e], gi = q.gi[e], u = q.u[e], hp = q.hp[e], at, mt;
@@ -250,6 +252,7 @@ __global__ void __launch_bounds__(NT) generic_bwd_scan_kernel(BwdArgs q) {
         q.hp[e] = dv * gi;
         a_next = at;
     }
+    if (q.dh0) q.dh0[(size_t)b * D + d] = a_next * g;   // a_0 g_0: h0 enters Eq. 4 only at t = 0
     q.part_vec[((size_t)b * 3 + 0) * D + d] = s_lam;
     q.part_vec[((size_t)b * 3 + 1) * D + d] = s_ba;
     q.part_vec[((size_t)b * 3 + 2) * D + d] = s_bx;
@@ -365,6 +368,42 @@ __global__ void __launch_bounds__(NT) generic_bwd_conv_kernel(BwdArgs q) {
     p[(size_t)4 * D] = sb;
 }
 
+// Gradient through the carried conv inputs and through the copies in conv_state_out.  One thread per (b, d); grid (ceil(D/NT), B).
+template <typename IOT, typename DUT>
+__global__ void __launch_bounds__(NT) state_conv_grads_kernel(BwdArgs q, const DUT *du) {
+    const int d = blockIdx.x * NT + threadIdx.x, b = blockIdx.y;
+    if (d >= q.D) return;
+    const int T = q.T, D = q.D;
+    const IOT *cw = (const IOT *)q.conv_w, *dcs_out = (const IOT *)q.dcs_out;
+    IOT *dx = (IOT *)q.dx, *dcs_in = (IOT *)q.dcs_in;
+    float w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) w[j] = ldf(cw, (size_t)j * D + d);
+    auto du_at = [&](int t) -> float { return (t >= 0 && t < T) ? (float)du[((size_t)b * T + t) * D + d] : 0.0f; };
+    auto dxin = [&](int t) -> float {   // gradient of the conv input at time t (t may be negative): sum_j w[j] du_{t+j}
+        float acc = 0.0f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc = fmaf(w[j], du_at(t + j), acc);
+        return acc;
+    };
+    float in_grad[3];
+#pragma unroll
+    for (int r = 0; r < 3; ++r) in_grad[r] = dxin(r - 3);
+    if (dcs_out) {
+#pragma unroll
+        for (int k = 0; k < 3; ++k) {
+            const float gk = ldf(dcs_out, ((size_t)b * 3 + k) * D + d);
+            const int row = T + k;   // row of concat(conv_state_in, x) that conv_state_out[k] copies
+            if (row >= 3) stf(dx, ((size_t)b * T + (row - 3)) * D + d, dxin(row - 3) + gk);
+            else in_grad[row] += gk;
+        }
+    }
+    if (dcs_in) {
+#pragma unroll
+        for (int r = 0; r < 3; ++r) stf(dcs_in, ((size_t)b * 3 + r) * D + d, in_grad[r]);
+    }
+}
+
 // out[i] = sum_p in[p * stride + i], p ascending (fixed order => run-to-run identical results)
 __global__ void reduce_partials_kernel(const float *in, int nparts, size_t stride, float *out, size_t n) {
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -448,6 +487,15 @@ cudaError_t generic_decode(const FwdArgs &a, int io, cudaStream_t st) {
     return cudaGetLastError();
 }
 
+cudaError_t state_conv_grads(const BwdArgs &q, int io, const void *du, bool du_is_half, cudaStream_t st) {
+    if (!q.dcs_in && !q.dcs_out) return cudaSuccess;
+    dim3 grid((q.D + NT - 1) / NT, q.B);
+    if (io == RGLRU_F32) state_conv_grads_kernel<float, float><<<grid, NT, 0, st>>>(q, (const float *)du);
+    else if (du_is_half) state_conv_grads_kernel<__nv_bfloat16, __half><<<grid, NT, 0, st>>>(q, (const __half *)du);
+    else state_conv_grads_kernel<__nv_bfloat16, float><<<grid, NT, 0, st>>>(q, (const float *)du);
+    return cudaGetLastError();
+}
+
 cudaError_t reduce_partials(const float *in, int nparts, size_t stride, float *out, size_t n, cudaStream_t st) {
     if (out == nullptr || n == 0) return cudaSuccess;
     reduce_partials_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(in, nparts, stride, out, n);
@@ -516,6 +564,7 @@ cudaError_t generic_backward(const FwdArgs &fwd_in, BwdArgs &q, int io, void *ws
     dim3 g5((D + NT - 1) / NT, q.nchunk, B);
     if (io == RGLRU_F32) generic_bwd_conv_kernel<float><<<g5, NT, 0, st>>>(q);
     else generic_bwd_conv_kernel<__nv_bfloat16><<<g5, NT, 0, st>>>(q);
+    if ((e = state_conv_grads(q, io, q.hp, false, st)) != cudaSuccess) return e;   // after dx: it rewrites the rows conv_state_out copies
     // 6. deterministic reductions of the per-channel partial sums
     const unsigned gd = (D + 255) / 256;
     reduce_partials_kernel<<<gd, 256, 0, st>>>(q.part_vec, B, (size_t)3 * D, q.dlambda, D);

@@ -65,6 +65,11 @@ struct BwdArgs {
     const float *lambda;
     void *dx;
     float *dconv_w, *dconv_b, *dW_a, *db_a, *dW_x, *db_x, *dlambda;
+    // gradient through the carried state (each may be null): in dh_T [B,D], dcs_out [B,3,D] io; out dh0 [B,D], dcs_in [B,3,D] io
+    const float *dh_T;
+    const void *dcs_out;
+    float *dh0;
+    void *dcs_in;
     // workspace arrays, each [B,T,D] fp32: u, r -> dz_a, i -> dz_x, hprev -> du
     float *u, *r, *gi, *hp;
     float *part_vec;   // [B][3][D]        partial sums of dlambda, db_a, db_x
@@ -101,6 +106,10 @@ bool sm100_backward_supported(int B, int T, int D, int H, int io);
 size_t sm100_backward_workspace_bytes(int B, int T, int D, int H);
 cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &b, const void *y_saved, void *ws_body, size_t ws_body_bytes, uint32_t *status,
                            cudaStream_t st);
+// Gradient of the three carried conv inputs, dcs_in[r] = sum_j w[j] du_{r-3+j} (0 <= r-3+j < T), and the gradient that arrives
+// on conv_state_out added to the rows it copies (dx_{T-3+k} is recomputed from du with the term added, so it is rounded once;
+// rows of conv_state_in when T < 3).  du is [B,T,D] of DUT (float or __half); io tensors are IOT.  No-op without dcs_in / dcs_out.
+cudaError_t state_conv_grads(const BwdArgs &q, int io, const void *du, bool du_is_half, cudaStream_t st);
 // out[i] = sum over p of in[p * stride + i] in ascending p (fixed order: run-to-run identical results)
 cudaError_t reduce_partials(const float *in, int nparts, size_t stride, float *out, size_t n, cudaStream_t st);
 // A row of n0 + n1 + n2 values summed over the parts and split over up to three output arrays (any of them may be null or

@@ -252,6 +252,8 @@ struct EwArgs {
     float2 *fold;                     // [B][nchunk][D]: (prod a_t, carry out of the chunk for zero carry in)
     float *xin;                       // [B][nchunk][D]: a_{t+1} g_{t+1} entering the chunk from later tokens
     float *part_vec;                  // [B*nchunk][3][D]
+    const float *dh_T;                // [B][D] gradient arriving on h_T, or null
+    float *dh0;                       // [B][D] gradient of h0, or null
 };
 
 // fp16 copies of the gate weights: W16[g][h][o][n] = W_g[h][o][n] and WT[h][n][g*256 + o] = W_g[h][o][n]
@@ -376,7 +378,8 @@ __global__ void __launch_bounds__(256) scan_fold_kernel(EwArgs a) {
 // pass 2: carries across chunks, last chunk first.  grid (D/256, B)
 __global__ void __launch_bounds__(256) scan_carry_kernel(EwArgs a) {
     const int d = blockIdx.x * 256 + threadIdx.x, b = blockIdx.y;
-    float X = 0.0f;
+    // what later tokens hand to the last chunk: the gradient arriving on h_T (h_T = h_{T-1}, factor 1), else nothing
+    float X = a.dh_T ? a.dh_T[(size_t)b * a.D + d] : 0.0f;
     // sixteen folds are requested at once (loads interleaved with the stores below would go out one at a time)
     for (int c1 = a.nchunk; c1 > 0; c1 -= 16) {
         float2 f[16];
@@ -394,6 +397,7 @@ __global__ void __launch_bounds__(256) scan_carry_kernel(EwArgs a) {
             }
         }
     }
+    if (a.dh0) a.dh0[(size_t)b * a.D + d] = X;   // what the first chunk hands on is a_0 g_0, the gradient of h0
 }
 
 // pass 3: the scan with its carry and every element-wise adjoint (derived from Eq. 1-4):
@@ -631,6 +635,7 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
     a.conv_b = fwd.conv_b; a.b_a = fwd.b_a; a.b_x = fwd.b_x; a.lambda = q.lambda; a.h0 = fwd.h0;
     a.u = u; a.uT = uT; a.dz = dz; a.dzT = dzT; a.z = z; a.du = du;
     a.fold = (float2 *)(ws + L.off_fold); a.xin = (float *)(ws + L.off_xin); a.part_vec = (float *)(ws + L.off_pvec);
+    a.dh_T = q.dh_T; a.dh0 = q.dh0;
 
     // 1. W^T for the du contraction, conv output
     convert_w_kernel<<<dim3(DH / 32, DH / 32, 2 * H), dim3(32, 8), 0, st>>>((const __nv_bfloat16 *)q.W_a, (const __nv_bfloat16 *)q.W_x, W16, WT, H);
@@ -693,6 +698,7 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
     cb.x = a.x; cb.conv_w = a.conv_w; cb.cs_in = a.cs_in; cb.du = du; cb.dx = (__nv_bfloat16 *)q.dx;
     cb.part_conv = (float *)(ws + L.off_pconv);
     conv_backward_kernel<<<grid_ew, 256, 0, st>>>(cb);
+    if ((e = state_conv_grads(q, RGLRU_BF16, du, true, st)) != cudaSuccess) return e;   // after dx: it rewrites the rows conv_state_out copies
     if ((e = reduce_partials3(cb.part_conv, nparts, (size_t)5 * D, q.dconv_w, (size_t)4 * D, q.dconv_b, D, nullptr, 0, st)) != cudaSuccess) return e;
     return cudaGetLastError();
 }

@@ -29,7 +29,7 @@ def test_every_declared_symbol_is_exported(lib):
     for n in names:
         assert getattr(lib, n) is not None, n
     assert sorted(binding.EXPORTED) == names
-    assert lib.rglru_abi_version() == 100
+    assert lib.rglru_abi_version() == 101
 
 
 def test_status_strings(lib):
@@ -91,10 +91,10 @@ def test_argument_errors_are_return_codes(lib):
     rc = lib.rglru_decode_step(ctypes.byref(sh), ctypes.byref(pp), vp(good), vp(good), vp(good), vp(good), vp(good), 1 << 20, None)
     assert rc == b.ERR_ALIAS
     args = [vp(good)] * 3 + [None, vp(good)] + [vp(good + 0x100000)] + [vp(good)] * 7
-    rc = lib.rglru_backward(ctypes.byref(sh), ctypes.byref(pp), *args, vp(good), 16, None)
+    rc = lib.rglru_backward(ctypes.byref(sh), ctypes.byref(pp), *args, None, vp(good), 16, None)
     assert rc == b.ERR_WORKSPACE
     args[5] = vp(good)
-    rc = lib.rglru_backward(ctypes.byref(sh), ctypes.byref(pp), *args, vp(good), 1 << 30, None)
+    rc = lib.rglru_backward(ctypes.byref(sh), ctypes.byref(pp), *args, None, vp(good), 1 << 30, None)
     assert rc == b.ERR_ALIAS
     rc = lib.rglru_prefill_host(ctypes.byref(sh), ctypes.byref(pp), vp(good), None, None, vp(good), vp(good), vp(good),
                                 vp(good), 16, vp(good), 1 << 20, None)

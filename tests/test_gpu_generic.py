@@ -132,3 +132,54 @@ def test_recorded_timeout_is_reported_once_and_wait_limit_knob_round_trips():
     assert prev == 2_000_000_000
     assert binding.set_wait_limit_ns(0) == 123456789
     assert binding.set_wait_limit_ns(0) == 2_000_000_000
+
+
+@pytest.mark.parametrize("B,T,D,H,io,flags", [(2, 33, 32, 2, "f32", 1), (1, 2, 16, 2, "f32", 1), (2, 1, 8, 1, "f32", 1),
+                                               (2, 64, 512, 2, "bf16", 0), (1, 200, 256, 1, "bf16", 0), (2, 70, 256, 2, "bf16", 1)])
+def test_backward_through_the_carried_state(oracle, B, T, D, H, io, flags):
+    """dh0 and d conv_state_in, with gradient arriving on h_T and conv_state_out, against the oracle: CUDA-core kernels
+    (fp32, and bf16 forced generic) and the tensor-core backward (bf16, head width 256, T a multiple of 8)."""
+    import torch
+    from paper_2402_19427_b200 import binding
+    inp = synth.make_inputs(B, T, D, H, io=io, seed=71 + T, with_dy=True, with_state=True, bias_scale=0.2)
+    rng = np.random.default_rng(5)
+    dhT = rng.normal(size=(B, D)).astype(np.float32)
+    dcs = rng.normal(size=(B, 3, D)).astype(np.float32)
+    if io == "bf16":
+        dcs = synth.round_to_bf16(dcs)
+    params = binding.Params.from_numpy(inp["params"], io)
+    g = binding.backward(to_dev(inp["x"], io), params, to_dev(inp["dy"], io), h0=to_dev(inp["h0"]),
+                         conv_state_in=to_dev(inp["conv_state"], io), flags=flags, dh_T=to_dev(dhT), dconv_state_out=to_dev(dcs, io),
+                         state_grads=True)
+    torch.cuda.synchronize()
+    gr = oracle.backward(inp["x"].astype(np.float64), f64(inp["params"]), H, inp["dy"].astype(np.float64), h0=inp["h0"].astype(np.float64),
+                         conv_state_in=inp["conv_state"].astype(np.float64), dh_T=dhT.astype(np.float64),
+                         dconv_state_out=dcs.astype(np.float64), state_grads=True)
+    for k in gr:
+        scale = max(1.0, float(np.abs(gr[k]).max())) if io == "f32" else 1.0
+        assert_close("d" + k, to_np(g[k]), gr[k], io, scale=scale)
+
+
+def test_backward_of_two_chained_segments_on_the_gpu_matches_the_whole(oracle):
+    """Truncated segments compose on the GPU as they do in the oracle: last segment first, its dh0 / d conv_state_in fed to
+    the segment before it.  Compared with the oracle's backward of the whole sequence."""
+    import torch
+    from paper_2402_19427_b200 import binding
+    B, T1, T2, D, H = 2, 128, 72, 256, 1
+    inp = synth.make_inputs(B, T1 + T2, D, H, io="bf16", seed=88, with_dy=True, with_state=True)
+    params = binding.Params.from_numpy(inp["params"], "bf16")
+    x = to_dev(inp["x"], "bf16"); dy = to_dev(inp["dy"], "bf16")
+    x1, x2 = x[:, :T1].contiguous(), x[:, T1:].contiguous()
+    h0 = to_dev(inp["h0"]); cs0 = to_dev(inp["conv_state"], "bf16")
+    y1, h1, cs1 = binding.prefill(x1, params, h0=h0, conv_state_in=cs0)
+    g2 = binding.backward(x2, params, dy[:, T1:].contiguous(), h0=h1, conv_state_in=cs1, state_grads=True)
+    g1 = binding.backward(x1, params, dy[:, :T1].contiguous(), h0=h0, conv_state_in=cs0, y=y1, dh_T=g2["h0"],
+                          dconv_state_out=g2["conv_state"], state_grads=True)
+    torch.cuda.synchronize()
+    gr = oracle.backward(inp["x"].astype(np.float64), f64(inp["params"]), H, inp["dy"].astype(np.float64), h0=inp["h0"].astype(np.float64),
+                         conv_state_in=inp["conv_state"].astype(np.float64), state_grads=True)
+    assert_close("dx", np.concatenate([to_np(g1["x"]), to_np(g2["x"])], 1), gr["x"], "bf16")
+    for k in ("conv_w", "conv_b", "W_a", "b_a", "W_x", "b_x", "lam"):
+        assert_close("d" + k, to_np(g1[k]) + to_np(g2[k]), gr[k], "bf16")
+    assert_close("dh0", to_np(g1["h0"]), gr["h0"], "bf16")
+    assert_close("dconv_state", to_np(g1["conv_state"]), gr["conv_state"], "bf16")

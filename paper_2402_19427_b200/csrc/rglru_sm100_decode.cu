@@ -6,17 +6,19 @@
 //   * its 2 x 128 rows of W_a, W_x arrive by tiled TMA in the 128-byte-swizzled K-major layout tcgen05.mma reads
 //     (the copy runs while the conv phase works);
 //   * all threads do the conv phase for the CTA's own 128 channels: one thread per (sequence, 8 channels) reads
-//     x and the three conv-state rows with 16-byte loads, writes the shifted conv state back (bit-exact copies),
-//     and stores the bf16 conv output u as one 16-byte swizzle chunk of the U tile, both into its own shared
-//     memory and into the peer CTA's (distributed shared memory), so that after one cluster barrier each CTA
-//     holds u for all 256 input channels.  Every conv-state element is read and written by exactly one thread.
+//     x and the three conv-state rows with 16-byte loads, stores the bf16 conv output u as one 16-byte swizzle chunk
+//     of the U tile in its own shared memory and writes the shifted conv state back (bit-exact copies) after the
+//     hand-over.  Every conv-state element is read and written by exactly one thread.  The CTA's half of the U tile
+//     (two K blocks of NB rows x 128 bytes) then goes to the peer CTA as two bulk shared-to-shared copies counted on a
+//     barrier of the peer, which only the peer's MMA-issuing thread waits for; a last barrier tells the sender that
+//     its copies have been received before it leaves.
 //     The rounding remainder u - bf16(u) is kept beside it (own channels only): the gate products take the
 //     bf16 value, the term i_t * u_t of Eq. 4 takes bf16(u) + remainder, which is u to 16 mantissa bits;
 //   * one thread issues Z^T = W U^T for both gates (M = 128 channels, N = sequences of the tile, K = 256) with
 //     fp32 accumulators in tensor memory;
 //   * all sixteen warps run the epilogue: channel on the TMEM lane, sequences along the columns; gates, log-space
 //     decay and h <- a h + sqrt(1 - a^2) (i u) in fp32, h and y written with lane-contiguous stores.
-// Waits on the two mbarriers are bounded and end in RGLRU_ERR_TIMEOUT; the only cluster barriers come before them.
+// Waits on the mbarriers are bounded and end in RGLRU_ERR_TIMEOUT; the only cluster barrier comes before them.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -38,8 +40,8 @@ constexpr uint32_t SMEM_WA = 0;
 constexpr uint32_t SMEM_WX = SMEM_WA + 4 * KBLOCK_BYTES;
 constexpr uint32_t SMEM_U = SMEM_WX + 4 * KBLOCK_BYTES;
 constexpr uint32_t SMEM_R = SMEM_U + 4 * KBLOCK_BYTES;    // bf16 r_s[NB_MAX][CH]: u - bf16(u) for this CTA's channels
-constexpr uint32_t SMEM_BAR = SMEM_R + NB_MAX * CH * 2;   // two mbarriers
-constexpr uint32_t SMEM_MISC = SMEM_BAR + 16;             // tmem base
+constexpr uint32_t SMEM_BAR = SMEM_R + NB_MAX * CH * 2;   // four mbarriers
+constexpr uint32_t SMEM_MISC = SMEM_BAR + 32;             // tmem base
 constexpr uint32_t SMEM_TOTAL = SMEM_MISC + 16;
 constexpr uint32_t SMEM_ALLOC = SMEM_TOTAL + 1024;
 constexpr uint32_t TMEM_COLS = 256;                        // z_a in columns [0, NB), z_x in [128, 128 + NB)
@@ -65,7 +67,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;   // the same offset in both CTAs of the cluster
     uint8_t *smem = smem_raw + (base - raw_addr);
-    const uint32_t BAR_W = base + SMEM_BAR, BAR_ACC = BAR_W + 8;
+    // BAR_W: weight bytes; BAR_ACC: accumulators complete; BAR_U: the peer's half of the U tile has landed here;
+    // BAR_SENT: the peer has received this CTA's half (nothing of this CTA's shared memory is still being read)
+    const uint32_t BAR_W = base + SMEM_BAR, BAR_ACC = BAR_W + 8, BAR_U = BAR_W + 16, BAR_SENT = BAR_W + 24;
     uint32_t *tmem_base_s = (uint32_t *)(smem + SMEM_MISC);
 
     const FwdArgs &f = p.f;
@@ -85,6 +89,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     if (tid == 0) {
         mbar_init(BAR_W, 1);
         mbar_init(BAR_ACC, 1);
+        mbar_init(BAR_U, 1);
+        mbar_init(BAR_SENT, 1);
+        mbar_expect_tx(BAR_U, 2u * (uint32_t)NB * 128u);   // two K blocks of NB rows x 128 bytes, sent by the peer
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) { tmem_alloc(smem_u32(tmem_base_s), TMEM_COLS); tmem_relinquish(); }
@@ -113,11 +120,21 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     const int c_own = q * 32 + lane;
     const int dl = (int)rank * CH + c_own;
     const size_t d = (size_t)head * DH + dl;
-    const float lam = f.lambda[d];
-    const float zl = -lam;
-    const float s = f.c * (zl > 0.0f ? zl + log1pf(expf(-zl)) : log1pf(expf(zl)));
-    const bool poly = __all_sync(0xffffffffu, s <= S_POLY);
-    const f32x2 hba2 = pack2(0.5f * f.b_a[d], 0.5f * f.b_a[d]), hbx2 = pack2(0.5f * f.b_x[d], 0.5f * f.b_x[d]), s2 = pack2(s, s);
+    const float lam = f.lambda[d], ba = f.b_a[d], bx = f.b_x[d];   // used after the conv phase: nothing waits on them here
+
+    // ---- gate products: the K blocks this CTA convolved itself are multiplied while the peer's half is still on its way
+    const uint32_t idesc = make_idesc(128, NB);
+    auto issue_kblocks = [&](int kb_first, bool first) {   // two K blocks = 8 K steps of 16, both gates
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t koff = (uint32_t)(kb_first + (j >> 2)) * KBLOCK_BYTES + (uint32_t)(j & 3) * 32u;
+            const uint64_t bd = make_desc_sw128(base + SMEM_U + koff);
+            const uint32_t accum = (first && j == 0) ? 0u : 1u;
+            mma_ss(tmem, make_desc_sw128(base + SMEM_WA + koff), bd, idesc, accum);
+            mma_ss(tmem + 128, make_desc_sw128(base + SMEM_WX + koff), bd, idesc, accum);
+        }
+    };
+    bool w_ok = true;
 
     // ---- conv phase: thread = (8-channel chunk c, sequences n = tid/16, tid/16 + 32, ...)
     {
@@ -151,8 +168,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
                 r2[i] = *(const uint4 *)(cs + ((size_t)b * 3 + 2) * D + cd);
             }
         }
-        cluster_wait();
-        const uint32_t peer_base = map_to_cta(base, rank ^ 1u);
+        cluster_wait();   // the peer has set up its barriers
         const uint32_t w0[4] = {w[0].x, w[0].y, w[0].z, w[0].w}, w1[4] = {w[1].x, w[1].y, w[1].z, w[1].w},
                        w2[4] = {w[2].x, w[2].y, w[2].z, w[2].w}, w3[4] = {w[3].x, w[3].y, w[3].z, w[3].w};
 #pragma unroll
@@ -176,20 +192,46 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
                 }
                 uo = make_uint4(o[0], o[1], o[2], o[3]);
                 *(uint4 *)(smem + SMEM_R + (uint32_t)n * (CH * 2) + (uint32_t)c * 16u) = make_uint4(rem[0], rem[1], rem[2], rem[3]);
-                // the conv state moves up by one row: bit-exact copies
+            }
+            *(uint4 *)(smem + u_kb + (uint32_t)n * 128u + ((chunk ^ (uint32_t)(n & 7)) << 4)) = uo;
+        }
+        fence_async_all();   // generic-proxy writes before the tensor core and the bulk copies read them
+        __syncthreads();     // this CTA's half of the U tile is complete in its own shared memory
+        // ... and goes to the peer as two bulk copies (one per K block: NB rows of 128 bytes, contiguous), counted on the
+        // peer's barrier: nobody but the peer's MMA issuer waits for them
+        if (tid == 32) {
+            const uint32_t peer_bar = map_to_cta(BAR_U, rank ^ 1u);
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const uint32_t off = SMEM_U + (uint32_t)((int)rank * 2 + k) * KBLOCK_BYTES;
+                bulk_s2peer(map_to_cta(base + off, rank ^ 1u), base + off, (uint32_t)NB * 128u, peer_bar);
+            }
+        }
+        if (tid == 0) {
+            w_ok = mbar_wait(BAR_W, 0, spin, &no_abort);
+            if (w_ok) {
+                tc_fence_after();
+                issue_kblocks((int)rank * 2, true);
+            } else {
+                atomicExch(f.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
+            }
+        }
+        // the conv state moves up by one row: bit-exact copies, stored after the hand-over so that nothing waits on them
+#pragma unroll
+        for (int i = 0; i < NIT; ++i) {
+            const int n = (tid >> 4) + 32 * i, b = b0 + n;
+            if (n < NB && b < B) {
                 *(uint4 *)(cs + ((size_t)b * 3 + 0) * D + cd) = r1[i];
                 *(uint4 *)(cs + ((size_t)b * 3 + 1) * D + cd) = r2[i];
                 *(uint4 *)(cs + ((size_t)b * 3 + 2) * D + cd) = xv[i];
             }
-            const uint32_t off = u_kb + (uint32_t)n * 128u + ((chunk ^ (uint32_t)(n & 7)) << 4);
-            *(uint4 *)(smem + off) = uo;
-            st_cluster_v4(peer_base + off, uo);
         }
     }
-    fence_async_all();   // generic-proxy writes (local and remote) before the tensor core reads them
-    __syncthreads();     // this CTA's half of the U tile is complete in its own shared memory
-    cluster_arrive();    // ... and, once the peer has waited, in the peer's
 
+    const float zl = -lam;
+    const float s = f.c * (zl > 0.0f ? zl + log1pf(expf(-zl)) : log1pf(expf(zl)));
+    const bool poly = __all_sync(0xffffffffu, s <= S_POLY);
+    const f32x2 hba2 = pack2(0.5f * ba, 0.5f * ba), hbx2 = pack2(0.5f * bx, 0.5f * bx), s2 = pack2(s, s);
     const uint8_t *u_col = smem + SMEM_U + (uint32_t)(dl >> 6) * KBLOCK_BYTES + (uint32_t)(dl & 7) * 2u;
     const uint32_t u_chunk = (uint32_t)(dl & 63) >> 3;
     const uint8_t *r_col = smem + SMEM_R + (uint32_t)c_own * 2u;
@@ -205,34 +247,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
         hv[j] = (j < nq && b < B) ? h[(size_t)b * D + d] : 0.0f;
     }
 
-    // ---- gate products: the K blocks this CTA convolved itself are multiplied while the peer's half is still on its way
-    const uint32_t idesc = make_idesc(128, NB);
-    auto issue_kblocks = [&](int kb_first, bool first) {   // two K blocks = 8 K steps of 16, both gates
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const uint32_t koff = (uint32_t)(kb_first + (j >> 2)) * KBLOCK_BYTES + (uint32_t)(j & 3) * 32u;
-            const uint64_t bd = make_desc_sw128(base + SMEM_U + koff);
-            const uint32_t accum = (first && j == 0) ? 0u : 1u;
-            mma_ss(tmem, make_desc_sw128(base + SMEM_WA + koff), bd, idesc, accum);
-            mma_ss(tmem + 128, make_desc_sw128(base + SMEM_WX + koff), bd, idesc, accum);
-        }
-    };
-    bool w_ok = true;
     if (tid == 0) {
-        w_ok = mbar_wait(BAR_W, 0, spin, &no_abort);
-        if (w_ok) {
+        // the peer's half of the U tile (waited for even when the weights failed: the peer's copies must have landed
+        // before this CTA may leave)
+        const bool u_ok = mbar_wait(BAR_U, 0, spin, &no_abort);
+        if (u_ok) mbar_arrive_at(BAR_SENT, rank ^ 1u);
+        if (u_ok && w_ok) {
             tc_fence_after();
-            issue_kblocks((int)rank * 2, true);
-        } else {
+            issue_kblocks((int)(rank ^ 1u) * 2, false);
+            tc_commit(BAR_ACC);
+        } else if (!u_ok) {
             atomicExch(f.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
         }
-    }
-    __syncwarp();
-    cluster_wait();      // both halves of the U tile are in place in both CTAs
-    if (tid == 0 && w_ok) {
-        fence_async_all();
-        issue_kblocks((int)(rank ^ 1u) * 2, false);
-        tc_commit(BAR_ACC);
     }
     __syncwarp();
 
@@ -283,6 +309,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
         while (gtimer() - tw < 50000ull) __nanosleep(1000);
     }
 
+    // the peer has received this CTA's half of the U tile: its bulk copies no longer read this shared memory
+    if (tid == 0 && !timed_out) mbar_wait(BAR_SENT, 0, spin, &no_abort);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);

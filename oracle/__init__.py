@@ -37,8 +37,10 @@ def _load():
         lib.oracle_num_threads.restype = ctypes.c_int
         lib.oracle_decay.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double, _dp, _dp]
         lib.oracle_decay.restype = None
-        lib.oracle_prefill.argtypes = [ctypes.c_int] * 4 + [ctypes.c_double] + [_dp] * 13
+        lib.oracle_prefill.argtypes = [ctypes.c_int] * 4 + [ctypes.c_double] + [_dp] * 15
         lib.oracle_prefill.restype = ctypes.c_int
+        lib.oracle_gelu.argtypes = [ctypes.c_double]
+        lib.oracle_gelu.restype = ctypes.c_double
         lib.oracle_decode_step.argtypes = [ctypes.c_int] * 3 + [ctypes.c_double] + [_dp] * 11
         lib.oracle_decode_step.restype = ctypes.c_int
         lib.oracle_backward.argtypes = [ctypes.c_int] * 4 + [ctypes.c_double] + [_dp] * 23
@@ -82,19 +84,29 @@ def _params(p, D, H):
     return keep, ptrs
 
 
-def prefill(x, params, H, c=8.0, h0=None, conv_state_in=None):
-    """Conv1D(4) + RG-LRU over T tokens (Eq. 1-4).  Returns (y[B,T,D], h_T[B,D], conv_state_out[B,3,D])."""
+def gelu(v: float) -> float:
+    """GeLU(v) = v Phi(v) (Section 2.3: the non-linearity on the recurrent block's second branch)."""
+    return float(_load().oracle_gelu(float(v)))
+
+
+def prefill(x, params, H, c=8.0, h0=None, conv_state_in=None, gate_branch=None, with_a_prod=False):
+    """Conv1D(4) + RG-LRU over T tokens (Eq. 1-4).  Returns (y[B,T,D], h_T[B,D], conv_state_out[B,3,D]), and with
+    ``with_a_prod`` a fourth array prod_t a_t [B,D].  With ``gate_branch`` [B,T,D], y_t = h_t * GeLU(gate_branch_t)
+    (Section 2.3) while h_T stays the raw state."""
     x = np.ascontiguousarray(x, dtype=np.float64)
     B, T, D = x.shape
     keep, (cw, cb, Wa, ba, Wx, bx, lam) = _params(params, D, H)
     h0a, h0p = _in(h0, (B, D))
     csa, csp = _in(conv_state_in, (B, 3, D))
+    gba, gbp = _in(gate_branch, (B, T, D))
     y = np.empty((B, T, D)); hT = np.empty((B, D)); cso = np.empty((B, 3, D))
+    ap = np.empty((B, D)) if with_a_prod else None
     rc = _load().oracle_prefill(B, T, D, H, float(c), x.ctypes.data_as(_dp), cw, cb, Wa, ba, Wx, bx, lam, h0p, csp,
-                                y.ctypes.data_as(_dp), hT.ctypes.data_as(_dp), cso.ctypes.data_as(_dp))
+                                y.ctypes.data_as(_dp), hT.ctypes.data_as(_dp), cso.ctypes.data_as(_dp), gbp,
+                                ap.ctypes.data_as(_dp) if with_a_prod else None)
     if rc != 0:
         raise ValueError("oracle_prefill: bad shape")
-    return y, hT, cso
+    return (y, hT, cso, ap) if with_a_prod else (y, hT, cso)
 
 
 def decode_step(x, params, H, h, conv_state, c=8.0):

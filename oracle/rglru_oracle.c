@@ -107,37 +107,51 @@ static void write_conv_state(const double *x, const double *cs_in, int B, int T,
     free(tmp);
 }
 
+/* GeLU(v) = v Phi(v) with Phi the standard normal distribution function: the definition of the non-linearity the
+ * recurrent block applies to its second branch (Section 2.3). */
+double oracle_gelu(double v) { return 0.5 * v * (1.0 + erf(v / sqrt(2.0))); }
+
 /*
  * Prefill / forward over T tokens.  Returns 0, or -1 on a bad shape.
  *   x [B,T,D]; conv_w [4,D]; conv_b [D] or NULL; W_a, W_x [H,Dh,Dh]; b_a, b_x, lambda [D];
  *   h0 [B,D] or NULL (zero); conv_state_in [B,3,D] or NULL (zero);
- *   y [B,T,D]; h_T [B,D] (may alias h0); conv_state_out [B,3,D] (may alias conv_state_in).
+ *   y [B,T,D]; h_T [B,D] (may alias h0); conv_state_out [B,3,D] (may alias conv_state_in);
+ *   gate_branch [B,T,D] or NULL: the second branch of the recurrent block (Section 2.3: GeLU on that branch, then the
+ *       two branches are merged by element-wise multiplication).  With it y_t = h_t * GeLU(gate_branch_t); the
+ *       carried state h_T stays the raw h;
+ *   a_prod [B,D] or NULL, out: prod_t a_t over the T tokens.  Eq. 4 is affine in the incoming state, so
+ *       h_T = a_prod * h0 + (h_T from a zero state): (a_prod, h_T from zero) describes the whole call as one step.
  */
 int oracle_prefill(int B, int T, int D, int H, double c, const double *x, const double *conv_w, const double *conv_b,
                    const double *W_a, const double *b_a, const double *W_x, const double *b_x, const double *lambda,
-                   const double *h0, const double *conv_state_in, double *y, double *h_T, double *conv_state_out) {
+                   const double *h0, const double *conv_state_in, double *y, double *h_T, double *conv_state_out,
+                   const double *gate_branch, double *a_prod) {
     if (B <= 0 || T <= 0 || D <= 0 || H <= 0 || D % H != 0) return -1;
     const int Dh = D / H;
 #pragma omp parallel for collapse(2) schedule(dynamic)
     for (int b = 0; b < B; ++b) {
         for (int k = 0; k < H; ++k) {
             const int d0 = k * Dh;
-            double *u = (double *)malloc(sizeof(double) * Dh * 4);
-            double *za = u + Dh, *zx = u + 2 * Dh, *h = u + 3 * Dh;
-            for (int n = 0; n < Dh; ++n) h[n] = h0 ? h0[(size_t)b * D + d0 + n] : 0.0;
+            double *u = (double *)malloc(sizeof(double) * Dh * 5);
+            double *za = u + Dh, *zx = u + 2 * Dh, *h = u + 3 * Dh, *ap = u + 4 * Dh;
+            for (int n = 0; n < Dh; ++n) { h[n] = h0 ? h0[(size_t)b * D + d0 + n] : 0.0; ap[n] = 1.0; }
             for (int t = 0; t < T; ++t) {
                 conv_row(x, conv_state_in, conv_w, conv_b, T, D, b, t, d0, Dh, u);
                 gate_preact(W_a + (size_t)k * Dh * Dh, b_a + d0, u, Dh, za); /* Eq. 1 */
                 gate_preact(W_x + (size_t)k * Dh * Dh, b_x + d0, u, Dh, zx); /* Eq. 2 */
                 for (int n = 0; n < Dh; ++n) {
                     double r = logistic(za[n]), i = logistic(zx[n]), a, m;
+                    const size_t at = ((size_t)b * T + t) * D + d0 + n;
                     oracle_decay(lambda[d0 + n], r, c, &a, &m);  /* Eq. 3 */
                     h[n] = a * h[n] + m * (i * u[n]);            /* Eq. 4 */
-                    y[((size_t)b * T + t) * D + d0 + n] = h[n];  /* y_t = h_t */
+                    ap[n] *= a;
+                    y[at] = gate_branch ? h[n] * oracle_gelu(gate_branch[at]) : h[n];  /* y_t = h_t [merged, Section 2.3] */
                 }
             }
             /* h_T may alias h0: each (b, head) slice is read above before it is written here */
             for (int n = 0; n < Dh; ++n) h_T[(size_t)b * D + d0 + n] = h[n];
+            if (a_prod)
+                for (int n = 0; n < Dh; ++n) a_prod[(size_t)b * D + d0 + n] = ap[n];
             free(u);
         }
     }

@@ -394,6 +394,63 @@ def test_backward_of_two_chained_segments_equals_one_segment(oracle, T1, T2):
     np.testing.assert_allclose(g1["conv_state"], whole["conv_state"], rtol=1e-10, atol=1e-12)
 
 
+# ---------------------------------------------------------------- the call as one affine step, and the merged output
+def test_decay_product_describes_the_call_as_one_step(oracle):
+    """Eq. 4 is affine in the incoming state: h_T(h0) = (prod_t a_t) h0 + h_T(0).  The product must reproduce that for any
+    h0, equal the closed form for constant gates, and compose over a split in time like the monoid (a2 a1, a2 b1 + b2)."""
+    x, p, h0, cs = rand_problem(31, T=17)
+    _, hz, _, ap = oracle.prefill(x, p, H=3, conv_state_in=cs, with_a_prod=True)
+    _, h1, _, ap1 = oracle.prefill(x, p, H=3, h0=h0, conv_state_in=cs, with_a_prod=True)
+    assert np.array_equal(ap, ap1)                                  # the product does not depend on the state
+    assert np.all(ap > 0) and np.all(ap < 1)
+    np.testing.assert_allclose(h1, ap * h0 + hz, rtol=1e-12, atol=1e-14)
+    # constant gates: a_t = sigmoid(Lambda)^(c sigmoid(b_a)) for every t
+    D, T = 5, 23
+    lam = np.linspace(-1, 4, D)
+    pc = const_gate_params(D, 1, lam, 0.7, 0.1)
+    rng = np.random.default_rng(2)
+    _, _, _, apc = oracle.prefill(rng.standard_normal((2, T, D)), pc, H=1, with_a_prod=True)
+    np.testing.assert_allclose(apc, np.broadcast_to(sigmoid(lam) ** (8.0 * sigmoid(0.7) * T), (2, D)), rtol=1e-12)
+    # two segments: the halo of the second is the conv state of the first; aggregates combine as (a2 a1, a2 b1 + b2)
+    for T1 in (1, 3, 9):
+        _, b1, c1, a1 = oracle.prefill(x[:, :T1], p, H=3, conv_state_in=cs, with_a_prod=True)
+        _, b2, _, a2 = oracle.prefill(x[:, T1:], p, H=3, conv_state_in=c1, with_a_prod=True)
+        np.testing.assert_allclose(a2 * a1, ap, rtol=1e-12)
+        np.testing.assert_allclose(a2 * b1 + b2, hz, rtol=1e-12, atol=1e-14)
+
+
+def test_gelu_merge(oracle):
+    """Section 2.3: GeLU on the second branch, then element-wise multiplication.  GeLU(v) = v Phi(v): GeLU(0) = 0,
+    GeLU(v) - GeLU(-v) = v, GeLU(v) -> v for large v, its minimum is about -0.17 near v = -0.75, and Phi is the normal
+    distribution function (checked against a numerical integral of the density).  The state is not touched by the merge."""
+    assert oracle.gelu(0.0) == 0.0
+    for v in (0.1, 0.5, 1.0, 2.5, 7.0):
+        assert abs(oracle.gelu(v) - oracle.gelu(-v) - v) < 1e-15 * max(1.0, v)
+    assert abs(oracle.gelu(12.0) - 12.0) < 1e-15 and abs(oracle.gelu(-12.0)) < 1e-15
+    grid = np.linspace(-3, 0, 3001)
+    vals = np.array([oracle.gelu(v) for v in grid])
+    assert abs(vals.min() - (-0.16997)) < 1e-4 and abs(grid[vals.argmin()] - (-0.7518)) < 2e-3
+    for v in (-1.3, 0.4, 2.0):   # Phi(v) by Simpson's rule on the normal density
+        t = np.linspace(-12.0, v, 200001)
+        dens = np.exp(-0.5 * t * t) / math.sqrt(2 * math.pi)
+        hstep = t[1] - t[0]
+        phi = hstep / 3 * (dens[0] + dens[-1] + 4 * dens[1:-1:2].sum() + 2 * dens[2:-1:2].sum())
+        assert abs(oracle.gelu(v) - v * phi) < 1e-10
+    x, p, h0, cs = rand_problem(32, T=11)
+    rng = np.random.default_rng(5)
+    g = rng.standard_normal(x.shape) * 2
+    y, hT, cso = oracle.prefill(x, p, H=3, h0=h0, conv_state_in=cs)
+    ym, hTm, csm = oracle.prefill(x, p, H=3, h0=h0, conv_state_in=cs, gate_branch=g)
+    assert np.array_equal(hT, hTm) and np.array_equal(cso, csm)
+    gel = np.vectorize(oracle.gelu)(g)
+    np.testing.assert_allclose(ym, y * gel, rtol=1e-15, atol=0)
+    # a branch that is a large constant passes h through scaled by that constant; a zero branch gives zero
+    yb, _, _ = oracle.prefill(x, p, H=3, h0=h0, conv_state_in=cs, gate_branch=np.full(x.shape, 20.0))
+    np.testing.assert_allclose(yb, 20.0 * y, rtol=1e-14)
+    y0, _, _ = oracle.prefill(x, p, H=3, h0=h0, conv_state_in=cs, gate_branch=np.zeros(x.shape))
+    assert np.all(y0 == 0)
+
+
 # ---------------------------------------------------------------- the synthetic input recipe
 def test_input_generator_is_seeded_and_bf16_exact():
     a = synth.make_inputs(2, 16, 32, 2, io="bf16", seed=5, long_memory_frac=0.25, with_dy=True, with_state=True)

@@ -111,6 +111,29 @@ int32_t rglru_prefill(const rglru_shape_t *shape, const rglru_params_t *params, 
                       size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * rglru_prefill with optional extras (NULL, or a struct whose members may each be NULL; with all of them NULL the call is
+ * rglru_prefill):
+ *   gate_branch [B,T,D] io, in: the second branch of the recurrent block (Section 2.3: a GeLU on that branch, then the two
+ *               branches are merged by element-wise multiplication).  The call then writes
+ *               y_t = h_t * GeLU(gate_branch_t), GeLU(v) = v Phi(v), the merge as the epilogue of the scan, so that h is
+ *               not written and read again by a separate kernel; h_T stays the raw state.  Must not overlap y.
+ *   a_prod      [B,D] fp32, out: prod_t a_t over the T tokens of the call (Eq. 3).  Eq. 4 is affine in the incoming state,
+ *               h_T = a_prod * h0 + (h_T from a zero state), so with h0 = NULL the pair (a_prod, h_T) describes the whole call
+ *               as one step of the recurrence: what ranks that split a sequence in time exchange (Section 4.1 shards the
+ *               recurrent block over heads without communication; along time one exchange of this pair per rank suffices).
+ * Other arguments, ownership, asynchrony and errors as for rglru_prefill; RGLRU_ERR_ALIGN also for an extra that is not
+ * 16-byte aligned, RGLRU_ERR_ALIAS also when gate_branch overlaps y.
+ */
+typedef struct {
+    const void *gate_branch;
+    float *a_prod;
+} rglru_prefill_extras_t;
+
+int32_t rglru_prefill_ex(const rglru_shape_t *shape, const rglru_params_t *params, const void *x, const float *h0,
+                         const void *conv_state_in, void *y, float *h_T, void *conv_state_out,
+                         const rglru_prefill_extras_t *extras, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * One decode step for B sequences (Section 5.1, "A simple model of the decode step", and Appendix F.4): the T = 1 case of the
  * forward with the state updated in place.
  *   x          [B,D] io, in

@@ -90,7 +90,7 @@ FwdArgs make_fwd(const rglru_shape_t *s, const rglru_params_t *p) {
 
 extern "C" {
 
-int32_t rglru_abi_version(void) { return 101; }
+int32_t rglru_abi_version(void) { return 102; }
 
 const char *rglru_status_string(int32_t status) {
     switch (status) {
@@ -127,20 +127,29 @@ size_t rglru_workspace_bytes(const rglru_shape_t *s, int32_t op) {
 int32_t rglru_prefill(const rglru_shape_t *s, const rglru_params_t *p, const void *x, const float *h0,
                       const void *conv_state_in, void *y, float *h_T, void *conv_state_out, void *workspace,
                       size_t workspace_bytes, void *cuda_stream) {
+    return rglru_prefill_ex(s, p, x, h0, conv_state_in, y, h_T, conv_state_out, nullptr, workspace, workspace_bytes, cuda_stream);
+}
+
+int32_t rglru_prefill_ex(const rglru_shape_t *s, const rglru_params_t *p, const void *x, const float *h0,
+                         const void *conv_state_in, void *y, float *h_T, void *conv_state_out, const rglru_prefill_extras_t *extras,
+                         void *workspace, size_t workspace_bytes, void *cuda_stream) {
     int32_t rc = check_shape(s, true);
     if (rc != RGLRU_OK) return rc;
     if ((rc = check_params(p)) != RGLRU_OK) return rc;
     if (!x || !y || !h_T || !conv_state_out || !workspace) return RGLRU_ERR_NULL;
+    const void *gate_branch = extras ? extras->gate_branch : nullptr;
+    float *a_prod = extras ? extras->a_prod : nullptr;
     if (!aligned(x, 16) || !aligned(y, 16) || !aligned(h_T, 16) || !aligned(conv_state_out, 16) || !aligned(h0, 16) ||
-        !aligned(conv_state_in, 16) || !aligned(workspace, 256))
+        !aligned(conv_state_in, 16) || !aligned(workspace, 256) || !aligned(gate_branch, 16) || !aligned(a_prod, 16))
         return RGLRU_ERR_ALIGN;
     const size_t need = rglru_workspace_bytes(s, RGLRU_OP_PREFILL);
     if (workspace_bytes < need) return RGLRU_ERR_WORKSPACE;
     const size_t nbytes = (size_t)s->B * s->T * s->D * io_bytes(s->io);
-    if (overlap(x, nbytes, y, nbytes)) return RGLRU_ERR_ALIAS;
+    if (overlap(x, nbytes, y, nbytes) || (gate_branch && overlap(gate_branch, nbytes, y, nbytes))) return RGLRU_ERR_ALIAS;
 
     FwdArgs a = make_fwd(s, p);
     a.x = x; a.h0 = h0; a.cs_in = conv_state_in; a.y = y; a.h_T = h_T; a.cs_out = conv_state_out;
+    a.gate_branch = gate_branch; a.a_prod = a_prod;
     a.status = (uint32_t *)workspace;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     cudaError_t e;

@@ -21,6 +21,8 @@ __device__ __forceinline__ void stf(float *p, size_t i, float v) { p[i] = v; }
 __device__ __forceinline__ void stf(__nv_bfloat16 *p, size_t i, float v) { p[i] = __float2bfloat16_rn(v); }
 
 __device__ __forceinline__ float sigmoid_acc(float z) { return 1.0f / (1.0f + expf(-z)); }
+// GeLU(v) = v Phi(v), the non-linearity on the second branch of the recurrent block (Section 2.3)
+__device__ __forceinline__ float gelu(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678f)); }
 
 // s = c * softplus(-Lambda) = -c log sigmoid(Lambda)   (Appendix A, with a = sigmoid(Lambda))
 __device__ __forceinline__ float decay_rate(float lambda, float c) {
@@ -101,6 +103,7 @@ __global__ void __launch_bounds__(NT) generic_prefill_kernel(FwdArgs a) {
     const IOT *x = (const IOT *)a.x, *cw = (const IOT *)a.conv_w, *cs_in = (const IOT *)a.cs_in;
     const IOT *Wa = (const IOT *)a.W_a + (size_t)k * Dh * Dh, *Wx = (const IOT *)a.W_x + (size_t)k * Dh * Dh;
     IOT *y = (IOT *)a.y;
+    const IOT *gb = (const IOT *)a.gate_branch;
     const int nob = (Dh + NT - 1) / NT;
 
     for (int n = tid; n < Dh; n += NT) h_s[n] = a.h0 ? a.h0[(size_t)b * D + d0 + n] : 0.0f;
@@ -129,6 +132,8 @@ __global__ void __launch_bounds__(NT) generic_prefill_kernel(FwdArgs a) {
                 const int d = d0 + o;
                 const float s = decay_rate(a.lambda[d], a.c), ba = a.b_a[d], bx = a.b_x[d];
                 float h = h_s[o];
+                // prod_t a_t of the call, carried from one time group to the next in the output itself (same thread each time)
+                float ap = (a.a_prod && t0 > 0) ? a.a_prod[(size_t)b * D + d] : 1.0f;
 #pragma unroll
                 for (int tt = 0; tt < GT; ++tt) {
                     if (tt < len) {
@@ -137,10 +142,13 @@ __global__ void __launch_bounds__(NT) generic_prefill_kernel(FwdArgs a) {
                         size_t e = ((size_t)b * T + t0 + tt) * D + d;
                         if (SAVE) { a.save_r[e] = r; a.save_i[e] = g; a.save_hprev[e] = h; }
                         h = fmaf(at, h, mt * (g * u_s[tt * Dh + o]));
-                        if (!SAVE) stf(y, e, h);
+                        ap *= at;
+                        // merged output of the recurrent block (Section 2.3): GeLU on the second branch, then the product
+                        if (!SAVE) stf(y, e, gb ? h * gelu(ldf(gb, e)) : h);
                     }
                 }
                 h_s[o] = h;
+                if (!SAVE && a.a_prod) a.a_prod[(size_t)b * D + d] = ap;
             }
         }
     }

@@ -56,6 +56,8 @@ struct FwdArgs {
     float *save_u, *save_r, *save_i, *save_hprev;
     uint32_t *status;         // workspace header
     uint32_t flags;           // RGLRU_FLAG_* of the call
+    const void *gate_branch;  // [B,T,D] io or null: y_t = h_t * GeLU(gate_branch_t) (prefill only)
+    float *a_prod;            // [B,D] or null: prod_t a_t over the call (prefill only)
 };
 
 struct BwdArgs {

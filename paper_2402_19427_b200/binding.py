@@ -23,7 +23,7 @@ FLAG_TEST_CARRY_NEVER_ARRIVES = 0x40000000   # failure-path test hook of the ten
 
 EXPORTED = ["rglru_abi_version", "rglru_status_string", "rglru_workspace_bytes", "rglru_prefill",
             "rglru_decode_step", "rglru_backward", "rglru_host_staging_bytes", "rglru_prefill_host",
-            "rglru_query_status", "rglru_prefill_static_scratch", "rglru_set_wait_limit_ns"]
+            "rglru_query_status", "rglru_prefill_static_scratch", "rglru_set_wait_limit_ns", "rglru_prefill_ex"]
 
 
 class Shape(ctypes.Structure):
@@ -63,6 +63,8 @@ def load() -> ctypes.CDLL:
         lib.rglru_workspace_bytes.restype = sz
         lib.rglru_prefill.argtypes = [sp, pp] + [vp] * 7 + [sz, vp]
         lib.rglru_prefill.restype = i32
+        lib.rglru_prefill_ex.argtypes = [sp, pp] + [vp] * 8 + [sz, vp]
+        lib.rglru_prefill_ex.restype = i32
         lib.rglru_decode_step.argtypes = [sp, pp] + [vp] * 5 + [sz, vp]
         lib.rglru_decode_step.restype = i32
         lib.rglru_backward.argtypes = [sp, pp] + [vp] * 15 + [sz, vp]
@@ -153,9 +155,14 @@ def alloc_workspace(shape: Shape, op: int, device) -> torch.Tensor:
     return torch.zeros(n, dtype=torch.uint8, device=device)
 
 
+class PrefillExtras(ctypes.Structure):
+    _fields_ = [("gate_branch", ctypes.c_void_p), ("a_prod", ctypes.c_void_p)]
+
+
 def prefill(x, params: Params, h0=None, conv_state_in=None, c=8.0, flags=0, y=None, h_T=None, conv_state_out=None,
-            workspace=None):
-    """y, h_T, conv_state_out = Conv1D(4) + RG-LRU over x[B,T,D] (rglru_prefill)."""
+            workspace=None, gate_branch=None, a_prod=None):
+    """y, h_T, conv_state_out = Conv1D(4) + RG-LRU over x[B,T,D] (rglru_prefill; rglru_prefill_ex when an extra is given).
+    ``gate_branch`` [B,T,D]: y_t = h_t * GeLU(gate_branch_t); ``a_prod`` [B,D] fp32 receives prod_t a_t."""
     lib = load()
     B, T, D = x.shape
     shape = make_shape(B, T, D, params.H, x.dtype, c, flags)
@@ -167,9 +174,15 @@ def prefill(x, params: Params, h0=None, conv_state_in=None, c=8.0, flags=0, y=No
     conv_state_out = torch.empty(B, 3, D, dtype=x.dtype, device=dev) if conv_state_out is None else conv_state_out
     _chk(y, (B, T, D), x.dtype, "y", dev); _chk(h_T, (B, D), torch.float32, "h_T", dev)
     _chk(conv_state_out, (B, 3, D), x.dtype, "conv_state_out", dev)
+    _chk(gate_branch, (B, T, D), x.dtype, "gate_branch", dev); _chk(a_prod, (B, D), torch.float32, "a_prod", dev)
     ws = alloc_workspace(shape, OP_PREFILL, dev) if workspace is None else workspace
-    rc = lib.rglru_prefill(ctypes.byref(shape), ctypes.byref(params.ptrs), _ptr(x), _ptr(h0), _ptr(conv_state_in),
-                           _ptr(y), _ptr(h_T), _ptr(conv_state_out), _ptr(ws), ws.numel(), _stream())
+    if gate_branch is None and a_prod is None:
+        rc = lib.rglru_prefill(ctypes.byref(shape), ctypes.byref(params.ptrs), _ptr(x), _ptr(h0), _ptr(conv_state_in),
+                               _ptr(y), _ptr(h_T), _ptr(conv_state_out), _ptr(ws), ws.numel(), _stream())
+    else:
+        ex = PrefillExtras(_ptr(gate_branch), _ptr(a_prod))
+        rc = lib.rglru_prefill_ex(ctypes.byref(shape), ctypes.byref(params.ptrs), _ptr(x), _ptr(h0), _ptr(conv_state_in),
+                                  _ptr(y), _ptr(h_T), _ptr(conv_state_out), ctypes.byref(ex), _ptr(ws), ws.numel(), _stream())
     if rc != OK:
         raise RglruError(rc, "rglru_prefill")
     return y, h_T, conv_state_out

@@ -57,7 +57,7 @@ constexpr uint32_t Y_BUF_BYTES = TILE * 32 * 2;            // 4096: one scan war
 constexpr uint32_t SMEM_Y = SMEM_X + XS * X_SLAB_BYTES;    // bf16 y_s[4 warps][2 buffers][64][32], staged for tiled stores
 constexpr uint32_t SMEM_AGG = SMEM_Y + 4 * 2 * Y_BUF_BYTES;   // float2 agg_s[2 buffers][2 half tiles][128 channels]
 constexpr uint32_t SMEM_BAR = SMEM_AGG + 2 * 2 * CH * 8;
-constexpr int NUM_BARS = 2 * XS + 2 * US + 4 + 8 + 1;
+constexpr int NUM_BARS = 2 * XS + 2 * US + 4 + 8 + 1 + 4;
 constexpr uint32_t SMEM_MISC = SMEM_BAR + NUM_BARS * 8;    // tmem base, abort flag
 constexpr uint32_t SMEM_TOTAL = SMEM_MISC + 16;
 constexpr uint32_t SMEM_ALLOC = SMEM_TOTAL + 1024;         // slack for 1024-byte alignment
@@ -66,10 +66,29 @@ constexpr uint32_t SMEM_ALLOC = SMEM_TOTAL + 1024;         // slack for 1024-byt
 constexpr uint32_t TM_W_A = 256, TM_W_X = 384;
 __host__ __device__ constexpr uint32_t tm_acc(int bf, int gate) { return (uint32_t)(bf * 128 + gate * 64); }
 
+// y * GeLU(g) for two tokens at once, GeLU(v) = v Phi(v) = v (1 + erf(v / sqrt 2)) / 2 (Section 2.3).  erf by the rational
+// approximation 7.1.26 of Abramowitz & Stegun (|error| < 1.5e-7):
+// 1 - erf(z) = t (a1 + t (a2 + t (a3 + t (a4 + t a5)))) exp(-z^2), t = 1 / (1 + p z), z >= 0.
+__device__ __forceinline__ f32x2 gelu_times2(f32x2 y, float g0, float g1) {
+    const f32x2 g = pack2(g0, g1);
+    const f32x2 z = mul2(pack2(fabsf(g0), fabsf(g1)), pack2(0.70710678f, 0.70710678f));
+    const f32x2 den = fma2(z, pack2(0.3275911f, 0.3275911f), pack2(1.0f, 1.0f));
+    const f32x2 t = pack2(__fdividef(1.0f, lo2(den)), __fdividef(1.0f, hi2(den)));
+    f32x2 q = fma2(t, pack2(1.061405429f, 1.061405429f), pack2(-1.453152027f, -1.453152027f));
+    q = fma2(q, t, pack2(1.421413741f, 1.421413741f));
+    q = fma2(q, t, pack2(-0.284496736f, -0.284496736f));
+    q = fma2(q, t, pack2(0.254829592f, 0.254829592f));
+    const f32x2 ez = mul2(mul2(z, z), pack2(-1.44269504f, -1.44269504f));
+    q = mul2(mul2(q, t), pack2(ex2_approx(lo2(ez)), ex2_approx(hi2(ez))));   // 1 - erf(z)
+    const f32x2 two_phi = pack2(g0 >= 0.0f ? 2.0f - lo2(q) : lo2(q), g1 >= 0.0f ? 2.0f - hi2(q) : hi2(q));   // 1 + erf(g / sqrt 2)
+    return mul2(y, mul2(mul2(g, pack2(0.5f, 0.5f)), two_phi));
+}
+
 struct Sm100Args {
     // x as [B][T][D] with a box of SLAB_ROWS token rows x one head; y with a box of TILE rows x 32 channels
     alignas(64) CUtensorMap tm_x;
     alignas(64) CUtensorMap tm_y;
+    alignas(64) CUtensorMap tm_g;   // gate branch, same geometry as y (encoded only when the call has one)
     FwdArgs f;
     int S;             // pairs per head (time split factor)
     int tps;           // tiles per sequence
@@ -82,6 +101,9 @@ struct Sm100Args {
 
 using namespace ptx;
 
+// MERGED: the call has a gate branch and writes y_t = h_t GeLU(branch_t); a separate instantiation so that the plain forward
+// carries none of its code.
+template <bool MERGED>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm100_prefill_kernel(const __grid_constant__ Sm100Args p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -97,6 +119,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
     auto BAR_ACCEMPTY = [&](int bf) { return bar0 + 8u * (2 * XS + 2 * US + 2 + bf); };   // leader CTA only
     auto BAR_GDONE = [&](int bf, int q) { return bar0 + 8u * (2 * XS + 2 * US + 4 + bf * 4 + q); };
     const uint32_t BAR_WREADY = bar0 + 8u * (2 * XS + 2 * US + 12);               // leader CTA only: both CTAs' weights are in tensor memory
+    auto BAR_BRANCH = [&](int q) { return bar0 + 8u * (2 * XS + 2 * US + 13 + q); };   // scan warp q's block of the gate branch has landed
     uint32_t *tmem_base_s = (uint32_t *)(smem + SMEM_MISC);
     volatile int *abort_flag = (volatile int *)(smem + SMEM_MISC + 4);
 
@@ -152,6 +175,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
             for (int q = 0; q < 4; ++q) mbar_init(BAR_GDONE(bf, q), 2);
         }
         mbar_init(BAR_WREADY, 16);
+        for (int q = 0; q < 4; ++q) mbar_init(BAR_BRANCH(q), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -436,6 +460,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
         const __nv_bfloat16 *x = (const __nv_bfloat16 *)f.x;
         const __nv_bfloat16 *cs_in = (const __nv_bfloat16 *)f.cs_in;
         float h_prev_own = 0.0f;  // state at the end of this pair's previous tile
+        float P_prev_own = 1.0f;  // prod of a_t from the start of the sequence to the end of this pair's previous tile
+        constexpr bool merged = MERGED;
         bool ok = true;
         int b, ti;
         tile_first(b, ti);
@@ -444,6 +470,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
             const int gidx = (b - B_whole) * p.tps + ti;   // index of the tile's carry record (shared tiles only)
             const int t0 = ti * TILE;
             const int bf = it & 1;
+            const uint32_t y_off = y_warp_off + (uint32_t)bf * Y_BUF_BYTES;
+            if constexpr (merged) {
+                // The warp's 64 x 32 block of the gate branch is fetched into the y staging buffer of this tile (free once
+                // the store of two tiles ago has read it) while the gate warps still work; y then overwrites it in place.
+                if (lane == 0) {
+                    bulk_wait_read1();
+                    mbar_expect_tx(BAR_BRANCH(q), Y_BUF_BYTES);
+                    tma_load_3d(base + y_off, &p.tm_g, head * DH + (int)rank * CH + q * 32, t0, b, BAR_BRANCH(q));
+                }
+                __syncwarp();
+            }
             ok = warp_wait(BAR_GDONE(bf, q), (it >> 1) & 1, spin, abort_flag);
             if (!ok) break;
             tc_fence_after();
@@ -451,9 +488,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
             const float2 e0 = agg_s[(bf * 2 + 0) * CH], e1 = agg_s[(bf * 2 + 1) * CH];
             // ---- incoming state of the tile: the state this pair reached at the end of its previous tile, or h0 near the
             //      start of a sequence, advanced by the aggregates that the other pairs published for the tiles in between
-            float h;
+            float h, P;
             if (!shared) {
                 h = ti == 0 ? (f.h0 ? f.h0[(size_t)b * D + d] : 0.0f) : h_prev_own;
+                P = ti == 0 ? 1.0f : P_prev_own;
             } else {
                 // publish the tile's aggregate before waiting for anyone
                 uint4 rec;
@@ -461,8 +499,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
                 uint4 *dst = p.agg + ((size_t)group * p.tiles_total + gidx) * CH + c_own;
                 asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "r"(rec.x), "r"(rec.y), "r"(rec.z), "r"(rec.w) : "memory");
                 int nback;
-                if (ti < S) { h = f.h0 ? f.h0[(size_t)b * D + d] : 0.0f; nback = ti; }
-                else { h = h_prev_own; nback = S - 1; }
+                if (ti < S) { h = f.h0 ? f.h0[(size_t)b * D + d] : 0.0f; P = 1.0f; nback = ti; }
+                else { h = h_prev_own; P = P_prev_own; nback = S - 1; }
                 if (nback > 0) {
                     // All records are requested at once, then polled until every lane sees this call's tag in
                     // both halves of each record (8-byte words are written atomically).
@@ -494,16 +532,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
                     if (!ok) break;
 #pragma unroll
                     for (int j = MAX_S - 1; j >= 1; --j)
-                        if (j <= nback) h = fmaf(__uint_as_float(r[j - 1].x), h, __uint_as_float(r[j - 1].z));
+                        if (j <= nback) { h = fmaf(__uint_as_float(r[j - 1].x), h, __uint_as_float(r[j - 1].z)); P *= __uint_as_float(r[j - 1].x); }
                 }
             }
             const float h_mid = fmaf(e0.x, h, e0.y);      // state after the first half tile
             h_prev_own = fmaf(e1.x, h_mid, e1.y);         // state after the tile
+            P_prev_own = P * (e0.x * e1.x);
             // ---- the y block written two tiles ago must have been read out by its tiled store
             if (lane == 0) bulk_wait_read1();
             __syncwarp();
             // ---- y_t = h_t = (h_t from zero) + (prod a up to t) h_in  (Eq. 4 unrolled over the half tile), 16 tokens at a time
-            const uint32_t y_off = y_warp_off + (uint32_t)bf * Y_BUF_BYTES;
             uint16_t *y_s = (uint16_t *)(smem + y_off) + lane;   // this thread's column of the warp's y block [64 tokens][32 channels]
             // The whole tile is pulled into registers and the accumulator buffer handed back before any arithmetic: the buffer's
             // round trip (MMA -> gate warps -> here -> MMA) is what paces the kernel.
@@ -515,14 +553,30 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_at(BAR_ACCEMPTY(bf), 0);
+            if constexpr (merged) {
+                // merged output of the recurrent block (Section 2.3): y_t = h_t GeLU(branch_t); the state is not touched
+                ok = warp_wait(BAR_BRANCH(q), it & 1, spin, abort_flag);
+                if (!ok) break;
 #pragma unroll
-            for (int j = 0; j < TILE; j += 2) {
-                const float hb = j < HALF ? h : h_mid;
-                const float y0 = fmaf(C[j], hb, H[j]), y1 = fmaf(C[j + 1], hb, H[j + 1]);
-                const __nv_bfloat162 o = __floats2bfloat162_rn(y0, y1);
-                const uint32_t ow = *(const uint32_t *)&o;
-                y_s[j * 32] = (uint16_t)(ow & 0xFFFFu);             // row of the warp's block: 32 channels x 2 bytes
-                y_s[(j + 1) * 32] = (uint16_t)(ow >> 16);
+                for (int j = 0; j < TILE; j += 2) {
+                    const float hb = j < HALF ? h : h_mid;
+                    const float g0 = __uint_as_float((uint32_t)y_s[j * 32] << 16), g1 = __uint_as_float((uint32_t)y_s[(j + 1) * 32] << 16);
+                    const f32x2 ym = gelu_times2(fma2(pack2(C[j], C[j + 1]), pack2(hb, hb), pack2(H[j], H[j + 1])), g0, g1);
+                    const __nv_bfloat162 o = __floats2bfloat162_rn(lo2(ym), hi2(ym));
+                    const uint32_t ow = *(const uint32_t *)&o;
+                    y_s[j * 32] = (uint16_t)(ow & 0xFFFFu);
+                    y_s[(j + 1) * 32] = (uint16_t)(ow >> 16);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < TILE; j += 2) {
+                    const float hb = j < HALF ? h : h_mid;
+                    const float y0 = fmaf(C[j], hb, H[j]), y1 = fmaf(C[j + 1], hb, H[j + 1]);
+                    const __nv_bfloat162 o = __floats2bfloat162_rn(y0, y1);
+                    const uint32_t ow = *(const uint32_t *)&o;
+                    y_s[j * 32] = (uint16_t)(ow & 0xFFFFu);             // row of the warp's block: 32 channels x 2 bytes
+                    y_s[(j + 1) * 32] = (uint16_t)(ow >> 16);
+                }
             }
             fence_async_smem();   // y rows become visible to the bulk-copy engine
             __syncwarp();
@@ -534,6 +588,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
             if (ti == p.tps - 1) {
                 // end of a sequence: h_T (unrounded state) and the last three raw inputs, bit-exact
                 f.h_T[(size_t)b * D + d] = h_prev_own;
+                if (f.a_prod) f.a_prod[(size_t)b * D + d] = P_prev_own;
                 __nv_bfloat16 keep[3];
 #pragma unroll
                 for (int kk = 0; kk < 3; ++kk) {
@@ -581,7 +636,9 @@ cudaError_t device_info(DeviceInfo *out) {
     DeviceInfo &di = g_dev[dev];
     if (!di.ready) {
         // opt in to the large dynamic shared memory once per device (function attributes are per context)
-        e = cudaFuncSetAttribute(sm100_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC);
+        e = cudaFuncSetAttribute(sm100_prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(sm100_prefill_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC);
         if (e != cudaSuccess) return e;
         int n = 0;
         if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) di.sms = n;
@@ -589,7 +646,7 @@ cudaError_t device_info(DeviceInfo *out) {
         q.gridDim = dim3(2 * di.sms); q.blockDim = dim3(NUM_THREADS); q.dynamicSmemBytes = SMEM_ALLOC;
         int np = 0;
         // a pair needs two free SMs of one cluster-capable group, so fewer than sms / 2 pairs may fit
-        di.max_pairs = (cudaOccupancyMaxActiveClusters(&np, sm100_prefill_kernel, &q) == cudaSuccess && np > 0) ? np : di.sms / 2 - 4;
+        di.max_pairs = (cudaOccupancyMaxActiveClusters(&np, sm100_prefill_kernel<false>, &q) == cudaSuccess && np > 0) ? np : di.sms / 2 - 4;
         di.ready = true;
     }
     *out = di;
@@ -683,6 +740,11 @@ cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes,
     Sm100Args p;
     if (!make_activation_map(&p.tm_x, a.x, a.B, a.T, a.D, DH, SLAB_ROWS) || !make_activation_map(&p.tm_y, a.y, a.B, a.T, a.D, 32, TILE))
         return cudaErrorNotSupported;
+    if (a.gate_branch) {
+        if (!make_activation_map(&p.tm_g, a.gate_branch, a.B, a.T, a.D, 32, TILE)) return cudaErrorNotSupported;
+    } else {
+        p.tm_g = p.tm_y;   // never used by the kernel
+    }
     p.f = a;
     p.tps = (a.T + TILE - 1) / TILE;
     const int pairs = di.max_pairs < di.sms / 2 ? di.max_pairs : di.sms / 2;
@@ -713,7 +775,7 @@ cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes,
     attr[0].id = cudaLaunchAttributeCooperative;   // pairs wait on one another's aggregates: they must all be resident
     attr[0].val.cooperative = 1;
     cfg.attrs = attr; cfg.numAttrs = (S > 1 && a.B % S != 0) ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, sm100_prefill_kernel, p);
+    return a.gate_branch ? cudaLaunchKernelEx(&cfg, sm100_prefill_kernel<true>, p) : cudaLaunchKernelEx(&cfg, sm100_prefill_kernel<false>, p);
 }
 
 }  // namespace rglru

@@ -1,7 +1,13 @@
-"""Partitioning of the temporal core across ranks.  No data-path collective exists: sequences are independent,
-and channels are independent outside a gate block (block-diagonal W_a / W_x, depthwise conv, diagonal recurrence;
-Section 4.1 of the paper, "Model parallelism"), so a rank owns whole sequences or whole heads and never exchanges activations.
-The only reductions are bookkeeping (the maximum of the per-rank step time).  numpy / torch.distributed only.
+"""Partitioning of the temporal core across ranks.  Sequences are independent, and channels are independent outside a
+gate block (block-diagonal W_a / W_x, depthwise conv, diagonal recurrence; Section 4.1 of the paper, "Model parallelism"),
+so a rank that owns whole sequences or whole heads never exchanges activations; the only reduction there is bookkeeping
+(the maximum of the per-rank step time).
+
+A sequence may also be split along time, rank r owning tokens [t_r, t_r + T_r).  Eq. 4 is affine in the incoming state, so a
+rank's share of the sequence acts on the state as one step h_out = A_r h_in + b_r with A_r = prod_t a_t and b_r its final
+state from a zero start; these steps compose as (A_2 A_1, A_2 b_1 + b_2).  Two small messages per rank suffice: the last
+three raw inputs of the share (the Conv1D history of the next rank), and the pair (A_r, b_r).  Every rank then knows its
+incoming state and runs the real forward.  numpy / torch.distributed only; no arithmetic of Eq. 1-3 lives here.
 """
 from __future__ import annotations
 
@@ -42,3 +48,41 @@ def max_over_ranks(value: float, dist=None, device=None) -> float:
     t = torch.tensor([float(value)], dtype=torch.float64, device=device if device is not None else "cpu")
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def combine_steps(first, second):
+    """Composition of two affine steps h -> A h + b applied in this order: (A_2 A_1, A_2 b_1 + b_2).  Works on numpy arrays
+    and torch tensors alike; associative, with identity (1, 0)."""
+    a1, b1 = first
+    a2, b2 = second
+    return a2 * a1, a2 * b1 + b2
+
+
+def exchange_conv_history(x_tail, dist, conv_state_in=None):
+    """The Conv1D history of this rank's time share: the last three raw inputs [B,3,D] of the rank before it
+    (`conv_state_in`, or zeros, for rank 0).  `x_tail` is this rank's own last three rows; every share must hold at
+    least three tokens.  One all-gather of [B,3,D] per rank."""
+    import torch
+    if x_tail.shape[1] != 3:
+        raise ValueError("x_tail must be the last three token rows of this rank's share")
+    rank, world = dist.get_rank(), dist.get_world_size()
+    tails = [torch.empty_like(x_tail) for _ in range(world)]
+    dist.all_gather(tails, x_tail.contiguous())
+    if rank > 0:
+        return tails[rank - 1]
+    return conv_state_in if conv_state_in is not None else torch.zeros_like(x_tail)
+
+
+def exchange_time_steps(a_prod, h_end, dist, h0=None):
+    """Incoming recurrent state [B,D] of this rank's time share.  `a_prod`, `h_end` [B,D]: the rank's share as one affine
+    step (prod_t a_t, and the final state of a forward from a zero state with the right Conv1D history).  One all-gather of
+    [B,2,D] per rank, then the exclusive scan over ranks of `combine_steps`, applied to `h0` (zeros if None)."""
+    import torch
+    rank, world = dist.get_rank(), dist.get_world_size()
+    mine = torch.stack([a_prod, h_end], dim=1).contiguous()
+    steps = [torch.empty_like(mine) for _ in range(world)]
+    dist.all_gather(steps, mine)
+    h = h0.clone() if h0 is not None else torch.zeros_like(h_end)
+    for r in range(rank):
+        h = steps[r][:, 0] * h + steps[r][:, 1]
+    return h

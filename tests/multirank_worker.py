@@ -30,6 +30,19 @@ def main():
                               conv_state_in=sl["conv_state"].astype(np.float64))
     hparts = [None] * world
     dist.all_gather_object(hparts, yh)
+    # time sharding: the sequence is cut along time; one message carries the Conv1D history, one the share as an affine step
+    g = synth.make_inputs(3, 45, 64, 2, io="bf16", seed=78, with_state=True)
+    gp = f64(g["params"])
+    ts, tc = sharding.split_range(45, world, rank)
+    xs = g["x"][:, ts:ts + tc].astype(np.float64)
+    hist = sharding.exchange_conv_history(torch.from_numpy(np.ascontiguousarray(xs[:, -3:])), dist,
+                                          conv_state_in=torch.from_numpy(g["conv_state"].astype(np.float64))).numpy()
+    _, b_r, _, a_r = oracle.prefill(xs, gp, 2, conv_state_in=hist, with_a_prod=True)
+    h_in = sharding.exchange_time_steps(torch.from_numpy(a_r), torch.from_numpy(b_r), dist,
+                                        h0=torch.from_numpy(g["h0"].astype(np.float64))).numpy()
+    yt, hTt, cst = oracle.prefill(xs, gp, 2, h0=h_in, conv_state_in=hist)
+    tparts = [None] * world
+    dist.all_gather_object(tparts, (yt, hTt, cst))
     slowest = sharding.max_over_ranks(10.0 + rank, dist)
     seeds = [None] * world
     dist.all_gather_object(seeds, sharding.rank_seed(synth.BASE_SEED, rank))
@@ -40,6 +53,11 @@ def main():
         assert np.array_equal(np.concatenate([p[1] for p in parts], 0), hf)
         assert np.array_equal(np.concatenate([p[2] for p in parts], 0), cf)
         assert np.array_equal(np.concatenate(hparts, 2), yf)
+        yg, hg, cg = oracle.prefill(g["x"].astype(np.float64), gp, 2, h0=g["h0"].astype(np.float64),
+                                    conv_state_in=g["conv_state"].astype(np.float64))
+        np.testing.assert_allclose(np.concatenate([p[0] for p in tparts], 1), yg, rtol=1e-12, atol=1e-14)
+        np.testing.assert_allclose(tparts[-1][1], hg, rtol=1e-12, atol=1e-14)      # the last rank ends in the final state
+        assert np.array_equal(tparts[-1][2], cg)
         assert slowest == 10.0 + world - 1
         assert len(set(seeds)) == world
         print("MULTIRANK_OK")

@@ -29,7 +29,7 @@ def test_every_declared_symbol_is_exported(lib):
     for n in names:
         assert getattr(lib, n) is not None, n
     assert sorted(binding.EXPORTED) == names
-    assert lib.rglru_abi_version() == 101
+    assert lib.rglru_abi_version() == 102
 
 
 def test_status_strings(lib):

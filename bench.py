@@ -462,7 +462,16 @@ def measure_extras(binding, dev, peaks):
 
 
 def run_only(args):
-    """One op a few times on a seeded synthetic workload of the given shape; meant to be wrapped in a profiler."""
+    """One op a few times on a seeded synthetic workload of the given shape; meant to be wrapped in a profiler.  Prints the
+    median CUDA-event time of the calls after the first.  With --impl reference (prefill only) the CPU oracle is timed on
+    one head of the same shape instead, which is 1/H of the work."""
+    if args.impl == "reference":
+        cfg = dict(synth.CONFIGS[1])
+        cfg.update(B=args.B or cfg["B"], T=args.T or cfg["T"], D=args.D or cfg["D"], H=args.H or cfg["H"])
+        tps, dt, cores, what = time_oracle(cfg, synth.BASE_SEED, 1)
+        print(json.dumps({"only": "prefill", "impl": "reference", "B": cfg["B"], "T": cfg["T"], "D": cfg["D"], "H": cfg["H"],
+                          "tokens_per_s": tps, "seconds": dt, "cores": cores, "sample": what}))
+        return
     import torch
     from paper_2402_19427_b200 import binding, build
     build.build()
@@ -475,12 +484,14 @@ def run_only(args):
     pr = synth.make_inputs(1, 4, D, H, io="bf16", seed=1)["params"]
     params = binding.Params.from_numpy(pr, "bf16", device=dev)
     g = torch.Generator(device=dev); g.manual_seed(0)
+    ev = []
     if args.only == "decode":
         x = torch.randn(B, D, device=dev, generator=g).to(dt)
         h = torch.randn(B, D, device=dev, generator=g)
         cs = torch.randn(B, 3, D, device=dev, generator=g).to(dt)
         for _ in range(args.iters):
-            binding.decode_step(x, params, h, cs)
+            ev.append((torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)))
+            ev[-1][0].record(); binding.decode_step(x, params, h, cs); ev[-1][1].record()
     else:
         xs = [torch.randn(B, T, D, device=dev, generator=g).to(dt) for _ in range(2)]
         ys = [torch.empty_like(xs[0]) for _ in range(2)]
@@ -488,14 +499,19 @@ def run_only(args):
             shape = binding.make_shape(B, T, D, H, dt)
             ws = binding.alloc_workspace(shape, binding.OP_PREFILL, dev)
             for i in range(args.iters):
-                binding.prefill(xs[i % 2], params, y=ys[i % 2], workspace=ws)
+                ev.append((torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)))
+                ev[-1][0].record(); binding.prefill(xs[i % 2], params, y=ys[i % 2], workspace=ws); ev[-1][1].record()
             if binding.query_status(ws) != binding.OK:
                 raise RuntimeError("device status")
         else:
             for i in range(args.iters):
-                binding.backward(xs[i % 2], params, ys[0].normal_())
+                dy = ys[0].normal_()
+                ev.append((torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)))
+                ev[-1][0].record(); binding.backward(xs[i % 2], params, dy); ev[-1][1].record()
     torch.cuda.synchronize()
-    print(json.dumps({"only": args.only, "B": B, "T": T, "D": D, "H": H, "iters": args.iters}))
+    us = sorted(a.elapsed_time(b) * 1e3 for a, b in ev[1:]) or [float("nan")]
+    print(json.dumps({"only": args.only, "B": B, "T": T, "D": D, "H": H, "iters": args.iters, "us_per_call_median": us[len(us) // 2],
+                      "us_per_call_min": us[0], "tokens_per_s": B * T * 1e6 / us[len(us) // 2]}))
 
 
 def launch_command(args, argv):

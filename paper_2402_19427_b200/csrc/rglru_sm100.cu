@@ -46,7 +46,8 @@ constexpr int SLAB_ROWS = HALF + 3;
 constexpr int XS = 4;              // x slab ring depth
 constexpr int US = 6;              // U tile stages
 constexpr int NUM_THREADS = 640;
-constexpr int MAX_S = 8;           // at most this many pairs share one head's time axis
+constexpr int MAX_S = 16;          // at most this many pairs share one head's time axis
+constexpr int LOOKBACK_BATCH = 8;  // carry records requested at once by the look-back
 constexpr uint32_t U_STAGE_BYTES = HALF * DH * 2;          // 16384
 constexpr uint32_t U_KBLOCK_BYTES = HALF * 128;            // 4096: one 64-channel K block
 constexpr uint32_t X_ROW_BYTES = DH * 2;                   // 512
@@ -501,25 +502,26 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
                 int nback;
                 if (ti < S) { h = f.h0 ? f.h0[(size_t)b * D + d] : 0.0f; P = 1.0f; nback = ti; }
                 else { h = h_prev_own; P = P_prev_own; nback = S - 1; }
-                if (nback > 0) {
-                    // All records are requested at once, then polled until every lane sees this call's tag in
-                    // both halves of each record (8-byte words are written atomically).
-                    const uint4 *src = p.agg + ((size_t)group * p.tiles_total + gidx) * CH + c_own;
-                    uint4 r[MAX_S - 1];
+                // The records are taken oldest first, up to eight at a time: all of a batch are requested at once, then polled
+                // until every lane sees this call's tag in both halves of each record (8-byte words are written atomically).
+                const uint4 *src = p.agg + ((size_t)group * p.tiles_total + gidx) * CH + c_own;
+                for (int jb = nback; jb > 0 && ok; jb -= LOOKBACK_BATCH) {
+                    const int cnt = jb < LOOKBACK_BATCH ? jb : LOOKBACK_BATCH;   // records jb, jb - 1, ..., jb - cnt + 1 tiles back
+                    uint4 r[LOOKBACK_BATCH];
                     uint64_t tstart = 0;
                     for (uint32_t npoll = 0;; ++npoll) {
                         bool ready = true;
 #pragma unroll
-                        for (int j = 1; j < MAX_S; ++j) {
-                            if (j <= nback) {
-                                const uint4 *sj = src - (size_t)j * CH;
+                        for (int k = 0; k < LOOKBACK_BATCH; ++k) {
+                            if (k < cnt) {
+                                const uint4 *sj = src - (size_t)(jb - k) * CH;
                                 asm volatile("ld.volatile.global.v4.b32 {%0, %1, %2, %3}, [%4];"
-                                             : "=r"(r[j - 1].x), "=r"(r[j - 1].y), "=r"(r[j - 1].z), "=r"(r[j - 1].w) : "l"(sj) : "memory");
+                                             : "=r"(r[k].x), "=r"(r[k].y), "=r"(r[k].z), "=r"(r[k].w) : "l"(sj) : "memory");
                             }
                         }
 #pragma unroll
-                        for (int j = 1; j < MAX_S; ++j)
-                            if (j <= nback) ready = ready && r[j - 1].y == p.tag_wait && r[j - 1].w == p.tag_wait;
+                        for (int k = 0; k < LOOKBACK_BATCH; ++k)
+                            if (k < cnt) ready = ready && r[k].y == p.tag_wait && r[k].w == p.tag_wait;
                         if (__all_sync(0xffffffffu, ready)) break;
                         if ((npoll & 15u) == 15u) {
                             const uint64_t tnow = gtimer();
@@ -529,11 +531,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
                         __nanosleep(32);
                     }
                     ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
+                    if (ok) {
 #pragma unroll
-                    for (int j = MAX_S - 1; j >= 1; --j)
-                        if (j <= nback) { h = fmaf(__uint_as_float(r[j - 1].x), h, __uint_as_float(r[j - 1].z)); P *= __uint_as_float(r[j - 1].x); }
+                        for (int k = 0; k < LOOKBACK_BATCH; ++k)
+                            if (k < cnt) { h = fmaf(__uint_as_float(r[k].x), h, __uint_as_float(r[k].z)); P *= __uint_as_float(r[k].x); }
+                    }
                 }
+                if (!ok) break;
             }
             const float h_mid = fmaf(e0.x, h, e0.y);      // state after the first half tile
             h_prev_own = fmaf(e1.x, h_mid, e1.y);         // state after the tile
@@ -711,12 +715,23 @@ bool sm100_prefill_supported(int B, int T, int D, int H, int io) {
 
 namespace {
 inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
-// Carry records exist for the sequences that are split in time: at most MAX_S - 1 of them (B mod S with S <= MAX_S).
+// Pairs that share a head's time axis: as many as fit beside the other heads, at most MAX_S.  The host-only workspace
+// size has to agree with the launch, so both count with at most MAX_PAIRS pairs whatever the device reports.
+constexpr int MAX_PAIRS = 74;
+inline int pairs_per_head(int H, int pairs) {
+    if (pairs > MAX_PAIRS) pairs = MAX_PAIRS;
+    int S = pairs / H;
+    return S < 1 ? 1 : (S > MAX_S ? MAX_S : S);
+}
+// Carry records exist for the sequences that are split in time: B mod S of them, at most S - 1 with S <= pairs_per_head(H, MAX_PAIRS).
 // Record (sequence slot, tile, half-head, channel) is indexed as [half-head][slot * tps + tile][channel].
-inline int record_slots(int B) { return B < MAX_S - 1 ? B : MAX_S - 1; }
+inline int record_slots(int B, int H) {
+    const int most = pairs_per_head(H, MAX_PAIRS) - 1;
+    return B < most ? B : most;
+}
 size_t agg_bytes(int B, int T, int H) {
     const size_t tps = (T + TILE - 1) / TILE;
-    return up256((size_t)H * 2 * record_slots(B) * tps * CH * sizeof(uint4));
+    return up256((size_t)H * 2 * record_slots(B, H) * tps * CH * sizeof(uint4));
 }
 inline bool ranges_overlap(const void *a, const void *b, size_t n) {
     if (!a || !b) return false;
@@ -748,12 +763,10 @@ cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes,
     p.f = a;
     p.tps = (a.T + TILE - 1) / TILE;
     const int pairs = di.max_pairs < di.sms / 2 ? di.max_pairs : di.sms / 2;
-    int S = pairs / a.H;
-    if (S < 1) S = 1;
-    if (S > MAX_S) S = MAX_S;
+    int S = pairs_per_head(a.H, pairs);
     if (S > a.B * p.tps) S = a.B * p.tps;
     p.S = S;
-    p.tiles_total = record_slots(a.B) * p.tps;
+    p.tiles_total = record_slots(a.B, a.H) * p.tps;
     p.tag = next_tag();
     p.tag_wait = (a.flags & RGLRU_FLAG_TEST_CARRY_NEVER_ARRIVES) ? ~p.tag : p.tag;
     p.agg = (uint4 *)ws_body;

@@ -27,6 +27,10 @@
  *    bytes, 256-byte aligned.  Its contents need not be preserved between calls; calls
  *    that share a workspace must be ordered on one stream.
  *  - Shapes without a kernel return RGLRU_ERR_UNSUPPORTED.  There is no CPU fallback.
+ *  - Kernels.  bf16 io with head width D_h = 256 runs on tensor-core kernels (prefill, decode step, backward).  The
+ *    tensor-core prefill also takes D_h = 128 and 64 when D is a multiple of 256 (Appendix C: the layers have 16 blocks, so
+ *    smaller models have narrower heads): two or four heads then share one 256 x 256 block-diagonal weight tile.  Every other
+ *    shape with D_h <= 1024, fp32 or bf16, runs on shape-generic CUDA-core kernels.
  */
 #ifndef RGLRU_H_
 #define RGLRU_H_
@@ -212,7 +216,7 @@ int32_t rglru_prefill_host(const rglru_shape_t *shape, const rglru_params_t *par
  *   - status_word: optional device pointer to a 4-byte-aligned uint32 owned by the caller, zero before the
  *     first use.  A device-side wait that runs out is recorded there, and the pointer may be given to
  *     rglru_query_status in place of a workspace.  NULL: such a condition is not reported.
- *   - Only shapes served by the tensor-core kernel (bf16 io, head width 256) are accepted; others return
+ *   - Only shapes served by the tensor-core prefill (bf16 io, head width 256, or 128 / 64 with D a multiple of 256) are accepted; others return
  *     RGLRU_ERR_UNSUPPORTED.  A shape whose scratch (256 bytes + rglru_workspace_bytes(shape, PREFILL))
  *     exceeds RGLRU_STATIC_SCRATCH_BYTES returns RGLRU_ERR_WORKSPACE; nothing is launched.
  *   - Every GPU on which the library is loaded holds the array until the process exits.

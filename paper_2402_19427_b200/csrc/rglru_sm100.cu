@@ -1,4 +1,5 @@
-// sm_100a fused prefill for the RG-LRU temporal core (bf16 io, head width 256).
+// sm_100a fused prefill for the RG-LRU temporal core (bf16 io, head width 256; heads of width 128 or 64 run as groups of
+// two or four that fill a 256-channel block whose weight matrix is block-diagonal).
 //
 // A head is owned by a pair of CTAs (a cluster of two, one CTA per SM).  CTA r of the pair keeps rows
 // [128 r, 128 r + 128) of W_a and W_x resident in its tensor memory as the A operand of the two-CTA form of
@@ -91,6 +92,7 @@ struct Sm100Args {
     alignas(64) CUtensorMap tm_y;
     alignas(64) CUtensorMap tm_g;   // gate branch, same geometry as y (encoded only when the call has one)
     FwdArgs f;
+    int dh;            // width of a head of the layer: 256, or 128 / 64 (then a "head" below is a group of 2 / 4 layer heads)
     int S;             // pairs per head (time split factor)
     int tps;           // tiles per sequence
     int tiles_total;   // B * tps
@@ -196,12 +198,19 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
     if (warp >= 8 && warp < 16) {
         const int q = warp & 3, g = (warp - 8) >> 2;  // g = 0: W_a, 1: W_x
         const __nv_bfloat16 *W = (const __nv_bfloat16 *)(g ? f.W_x : f.W_a);
-        const uint4 *row = (const uint4 *)(W + ((size_t)head * DH + rank * CH + q * 32 + lane) * DH);
+        // Narrower heads (128 or 64 channels) run as groups of 2 or 4 heads that fill the 256 x 256 block: the block is then
+        // block-diagonal, and a row holds its own head's weights in that head's input channels and zeros elsewhere.
+        const int dh = p.dh, row_in_group = (int)rank * CH + q * 32 + lane;
+        const int sub = row_in_group / dh;                     // head of the group this output channel belongs to
+        const uint4 *row = (const uint4 *)(W + ((size_t)head * DH + row_in_group) * dh);   // (head * 256 / dh + sub) * dh + row_in_group % dh rows of dh
+        const int c_first = sub * (dh >> 3), c_count = dh >> 3;   // the 16-byte chunks of the 256 input channels that are this head's
         const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (g ? TM_W_X : TM_W_A);
         auto cvt2 = [](uint32_t w) { return pack_f16_sat(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u)); };
+        const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll 4
         for (int c = 0; c < 16; ++c) {
-            uint4 lo = __ldg(row + 2 * c), hi = __ldg(row + 2 * c + 1);
+            const int c0 = 2 * c - c_first, c1 = c0 + 1;
+            uint4 lo = (c0 >= 0 && c0 < c_count) ? __ldg(row + c0) : zero4, hi = (c1 >= 0 && c1 < c_count) ? __ldg(row + c1) : zero4;
             lo.x = cvt2(lo.x); lo.y = cvt2(lo.y); lo.z = cvt2(lo.z); lo.w = cvt2(lo.w);
             hi.x = cvt2(hi.x); hi.y = cvt2(hi.y); hi.z = cvt2(hi.z); hi.w = cvt2(hi.w);
             tmem_st8(taddr + c * 8, lo, hi);
@@ -709,8 +718,11 @@ bool encode_bf16_map_3d(CUtensorMap *tm, const void *ptr, uint64_t d0, uint64_t 
     return encode_map16_3d(tm, ptr, dims, strides, box, swizzle128);
 }
 
+// Head width 256, or 128 / 64 with the heads filling whole 256-channel groups (the kernel then works on D / 256 groups).
 bool sm100_prefill_supported(int B, int T, int D, int H, int io) {
-    return io == RGLRU_BF16 && B > 0 && T > 0 && H > 0 && D == H * DH;
+    if (io != RGLRU_BF16 || B <= 0 || T <= 0 || H <= 0 || D % H != 0 || D % DH != 0) return false;
+    const int dh = D / H;
+    return dh == 256 || dh == 128 || dh == 64;
 }
 
 namespace {
@@ -745,6 +757,7 @@ inline bool ranges_overlap(const void *a, const void *b, size_t n) {
 // different tiles and of the two halves of a head read the incoming state at unrelated times,
 // so an in-place update must not be visible to them.
 size_t sm100_prefill_workspace_bytes(int B, int T, int D, int H) {
+    H = D / DH;   // the kernel's unit is a 256-channel group of heads
     return agg_bytes(B, T, H) + up256((size_t)B * D * sizeof(float)) + up256((size_t)B * 3 * D * sizeof(__nv_bfloat16));
 }
 
@@ -761,19 +774,22 @@ cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes,
         p.tm_g = p.tm_y;   // never used by the kernel
     }
     p.f = a;
+    const int G = a.D / DH;   // 256-channel groups of heads: the kernel's "heads"
+    p.f.H = G;
+    p.dh = a.D / a.H;
     p.tps = (a.T + TILE - 1) / TILE;
     const int pairs = di.max_pairs < di.sms / 2 ? di.max_pairs : di.sms / 2;
-    int S = pairs_per_head(a.H, pairs);
+    int S = pairs_per_head(G, pairs);
     if (S > a.B * p.tps) S = a.B * p.tps;
     p.S = S;
-    p.tiles_total = record_slots(a.B, a.H) * p.tps;
+    p.tiles_total = record_slots(a.B, G) * p.tps;
     p.tag = next_tag();
     p.tag_wait = (a.flags & RGLRU_FLAG_TEST_CARRY_NEVER_ARRIVES) ? ~p.tag : p.tag;
     p.agg = (uint4 *)ws_body;
     p.spin_ns = g_spin_limit_ns;
     if (ws_body_bytes < sm100_prefill_workspace_bytes(a.B, a.T, a.D, a.H)) return cudaErrorInvalidValue;
     const size_t h_bytes = (size_t)a.B * a.D * sizeof(float), cs_bytes = (size_t)a.B * 3 * a.D * sizeof(__nv_bfloat16);
-    char *h0_copy = (char *)ws_body + agg_bytes(a.B, a.T, a.H), *cs_copy = h0_copy + up256(h_bytes);
+    char *h0_copy = (char *)ws_body + agg_bytes(a.B, a.T, G), *cs_copy = h0_copy + up256(h_bytes);
     if (ranges_overlap(a.h0, a.h_T, h_bytes)) {
         if ((e = cudaMemcpyAsync(h0_copy, a.h0, h_bytes, cudaMemcpyDeviceToDevice, st)) != cudaSuccess) return e;
         p.f.h0 = (const float *)h0_copy;
@@ -783,7 +799,7 @@ cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes,
         p.f.cs_in = cs_copy;
     }
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(2 * a.H * S); cfg.blockDim = dim3(NUM_THREADS); cfg.dynamicSmemBytes = SMEM_ALLOC; cfg.stream = st;
+    cfg.gridDim = dim3(2 * G * S); cfg.blockDim = dim3(NUM_THREADS); cfg.dynamicSmemBytes = SMEM_ALLOC; cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeCooperative;   // pairs wait on one another's aggregates: they must all be resident
     attr[0].val.cooperative = 1;

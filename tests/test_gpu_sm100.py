@@ -214,3 +214,23 @@ def test_prefill_host_pipelined_chunks_match_device_prefill(oracle, B, T, H):
         assert_close("y", to_np(y_pin), yr, "bf16"); assert_close("h_T", to_np(hT_pin), hr, "bf16")
         assert np.array_equal(to_np(cs_pin), cr)
         y_pin.zero_()
+
+
+@pytest.mark.parametrize("Dh,B,T,H", [(128, 2, 130, 2), (128, 3, 257, 4), (64, 2, 130, 4), (64, 1, 1000, 8), (128, 9, 200, 2)])
+def test_narrower_heads_on_the_tensor_core_path(oracle, Dh, B, T, H):
+    """Heads of width 128 and 64 (the paper's 16-block layers at smaller model sizes, Appendix C) run on the same kernel as
+    groups of two or four heads whose block-diagonal weights fill a 256 x 256 block; a workspace larger than the bare
+    status header shows that the tensor-core path was chosen.  The last case splits a sequence in time."""
+    D = Dh * H
+    assert D % 256 == 0 and uses_sm100(B, T, D, H)
+    inp = synth.make_inputs(B, T, D, H, io="bf16", seed=800 + Dh + T, with_state=True, bias_scale=0.5)
+    y, hT, cso = gpu_prefill(inp, h0=inp["h0"], cs=inp["conv_state"])
+    yr, hr, cr = oracle_prefill(oracle, inp, h0=inp["h0"].astype(np.float64), cs=inp["conv_state"].astype(np.float64))
+    assert_close("y", y, yr, "bf16"); assert_close("h_T", hT, hr, "bf16")
+    assert np.array_equal(cso, cr)
+    # heads stay independent: changing one head's weights changes only that head's channels
+    inp2 = {**inp, "params": dict(inp["params"])}
+    W = inp2["params"]["W_a"].copy(); W[1] = -W[1]; inp2["params"]["W_a"] = W
+    y2, _, _ = gpu_prefill(inp2, h0=inp["h0"], cs=inp["conv_state"])
+    other = np.ones(D, bool); other[Dh:2 * Dh] = False
+    assert np.array_equal(y2[:, :, other], y[:, :, other]) and not np.array_equal(y2[:, :, ~other], y[:, :, ~other])

@@ -218,7 +218,7 @@ def test_prefill_host_pipelined_chunks_match_device_prefill(oracle, B, T, H):
 
 @pytest.mark.parametrize("Dh,B,T,H", [(128, 2, 130, 2), (128, 3, 257, 4), (64, 2, 130, 4), (64, 1, 1000, 8), (128, 9, 200, 2)])
 def test_narrower_heads_on_the_tensor_core_path(oracle, Dh, B, T, H):
-    """Heads of width 128 and 64 (the paper's 16-block layers at smaller model sizes, Appendix C) run on the same kernel as
+    """Heads of width 128 and 64 (the 16 blocks of Section 4.1 at smaller D_RNN) run on the same kernel as
     groups of two or four heads whose block-diagonal weights fill a 256 x 256 block; a workspace larger than the bare
     status header shows that the tensor-core path was chosen.  The last case splits a sequence in time."""
     D = Dh * H

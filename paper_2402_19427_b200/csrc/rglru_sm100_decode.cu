@@ -1,4 +1,5 @@
-// sm_100a batched decode step of the RG-LRU temporal core (bf16 io, head width 256): one new token for each
+// sm_100a batched decode step of the RG-LRU temporal core (bf16 io, head width 256; 128 and 64 as groups of heads, see the
+// weight loads below): one new token for each
 // of B sequences, recurrent state h [B,D] fp32 and the 3-row conv state [B,3,D] updated in place.
 //
 // A cluster of two CTAs owns one (head, batch tile) pair.  CTA r of the pair owns channels [128 r, 128 r + 128)
@@ -50,6 +51,7 @@ struct DecArgs {
     alignas(64) CUtensorMap tm_wa;   // W_a as [H][256 out][256 in], box 128 out x 64 in, 128-byte swizzle
     alignas(64) CUtensorMap tm_wx;
     FwdArgs f;
+    int dh;       // head width of the layer: 256, or 128 / 64 (a "head" of the kernel is then a group of 2 / 4 heads, H their number)
     int NB;       // sequences per batch tile (multiple of 16)
     int ntile;    // batch tiles
     unsigned long long spin_ns;
@@ -104,15 +106,48 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     // ---- this CTA's gate weights: 2 gates x 4 K blocks of [128 out rows x 64 in channels], issued by the last warp so
     //      that the descriptor fetch of the first tiled copy delays nobody's global loads; they are the longest latency
     //      of the step (128 KB per CTA out of L2) and overlap the whole conv phase
+    //      Narrower heads (128 or 64 channels) run as groups of 2 or 4 that fill the 256 channels: the group's weight matrix is
+    //      block-diagonal, so this CTA's 128 output rows only see K blocks 2 rank and 2 rank + 1 -- the channels it convolves
+    //      itself -- and nothing is exchanged with the peer.  With 64-wide heads each of those K blocks holds one head's 64 rows;
+    //      the other 64 rows of the block are zeroed by the threads below.
+    const int dh = p.dh;
     if (tid == NTHREADS - 32) {
-        mbar_expect_tx(BAR_W, 8 * KBLOCK_BYTES);
+        if (dh == DH) {
+            mbar_expect_tx(BAR_W, 8 * KBLOCK_BYTES);
 #pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-            tma_load_3d(base + SMEM_WA + kb * KBLOCK_BYTES, &p.tm_wa, kb * 64, (int)rank * CH, head, BAR_W);
-            tma_load_3d(base + SMEM_WX + kb * KBLOCK_BYTES, &p.tm_wx, kb * 64, (int)rank * CH, head, BAR_W);
+            for (int kb = 0; kb < 4; ++kb) {
+                tma_load_3d(base + SMEM_WA + kb * KBLOCK_BYTES, &p.tm_wa, kb * 64, (int)rank * CH, head, BAR_W);
+                tma_load_3d(base + SMEM_WX + kb * KBLOCK_BYTES, &p.tm_wx, kb * 64, (int)rank * CH, head, BAR_W);
+            }
+        } else if (dh == 128) {
+            mbar_expect_tx(BAR_W, 4 * KBLOCK_BYTES);
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const uint32_t off = (uint32_t)(2 * (int)rank + j) * KBLOCK_BYTES;
+                tma_load_3d(base + SMEM_WA + off, &p.tm_wa, j * 64, 0, 2 * head + (int)rank, BAR_W);
+                tma_load_3d(base + SMEM_WX + off, &p.tm_wx, j * 64, 0, 2 * head + (int)rank, BAR_W);
+            }
+        } else {
+            mbar_expect_tx(BAR_W, 2 * KBLOCK_BYTES);
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const uint32_t off = (uint32_t)(2 * (int)rank + j) * KBLOCK_BYTES + (uint32_t)j * (KBLOCK_BYTES / 2);
+                tma_load_3d(base + SMEM_WA + off, &p.tm_wa, 0, 0, 4 * head + 2 * (int)rank + j, BAR_W);
+                tma_load_3d(base + SMEM_WX + off, &p.tm_wx, 0, 0, 4 * head + 2 * (int)rank + j, BAR_W);
+            }
         }
     }
     __syncwarp();
+    if (dh == 64) {
+        // rows of the two K blocks that belong to the other head of this CTA: zero (generic stores; the fence and barrier after
+        // the conv phase order them before the MMAs)
+        for (int i = tid; i < 4 * (int)(KBLOCK_BYTES / 2 / 16); i += NTHREADS) {
+            const int blk = i / (int)(KBLOCK_BYTES / 2 / 16), w16 = i % (int)(KBLOCK_BYTES / 2 / 16);   // blk: gate * 2 + j
+            const int j = blk & 1;
+            const uint32_t off = (blk >> 1 ? SMEM_WX : SMEM_WA) + (uint32_t)(2 * (int)rank + j) * KBLOCK_BYTES + (uint32_t)(1 - j) * (KBLOCK_BYTES / 2) + (uint32_t)w16 * 16u;
+            *(uint4 *)(smem + off) = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
 
     // ---- epilogue constants (parameters only, fetched early): warp (q, kq) owns channels 32 q .. 32 q + 31 and quarter kq
     //      of the tile's sequences
@@ -199,7 +234,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
         __syncthreads();     // this CTA's half of the U tile is complete in its own shared memory
         // ... and goes to the peer as two bulk copies (one per K block: NB rows of 128 bytes, contiguous), counted on the
         // peer's barrier: nobody but the peer's MMA issuer waits for them
-        if (tid == 32) {
+        if (tid == 32 && dh == DH) {
             const uint32_t peer_bar = map_to_cta(BAR_U, rank ^ 1u);
 #pragma unroll
             for (int k = 0; k < 2; ++k) {
@@ -250,11 +285,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     if (tid == 0) {
         // the peer's half of the U tile (waited for even when the weights failed: the peer's copies must have landed
         // before this CTA may leave)
-        const bool u_ok = mbar_wait(BAR_U, 0, spin, &no_abort);
-        if (u_ok) mbar_arrive_at(BAR_SENT, rank ^ 1u);
+        const bool u_ok = dh != DH || mbar_wait(BAR_U, 0, spin, &no_abort);
+        if (u_ok && dh == DH) mbar_arrive_at(BAR_SENT, rank ^ 1u);
         if (u_ok && w_ok) {
             tc_fence_after();
-            issue_kblocks((int)(rank ^ 1u) * 2, false);
+            if (dh == DH) issue_kblocks((int)(rank ^ 1u) * 2, false);
             tc_commit(BAR_ACC);
         } else if (!u_ok) {
             atomicExch(f.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
@@ -310,7 +345,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     }
 
     // the peer has received this CTA's half of the U tile: its bulk copies no longer read this shared memory
-    if (tid == 0 && !timed_out) mbar_wait(BAR_SENT, 0, spin, &no_abort);
+    if (tid == 0 && !timed_out && dh == DH) mbar_wait(BAR_SENT, 0, spin, &no_abort);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
@@ -324,20 +359,29 @@ int num_sms() {
 
 }  // namespace
 
-bool sm100_decode_supported(int B, int D, int H, int io) { return io == RGLRU_BF16 && B > 0 && H > 0 && D == H * DH; }
+// Head width 256, or 128 / 64 with the heads filling whole 256-channel groups.
+bool sm100_decode_supported(int B, int D, int H, int io) {
+    if (io != RGLRU_BF16 || B <= 0 || H <= 0 || D % H != 0 || D % DH != 0) return false;
+    const int dh = D / H;
+    return dh == 256 || dh == 128 || dh == 64;
+}
 
 cudaError_t sm100_decode(const FwdArgs &a, cudaStream_t st) {
     static PerDeviceOptIn opt_in;
     cudaError_t e = opt_in.ensure(sm100_decode_kernel, (int)SMEM_ALLOC);
     if (e != cudaSuccess) return e;
     DecArgs p;
-    if (!encode_bf16_map_3d(&p.tm_wa, a.W_a, DH, DH, (uint64_t)a.H, 64, CH, true) ||
-        !encode_bf16_map_3d(&p.tm_wx, a.W_x, DH, DH, (uint64_t)a.H, 64, CH, true))
+    const int dh = a.D / a.H, G = a.D / DH;   // G: 256-channel groups of heads, the kernel's unit
+    const uint32_t box_rows = dh == 64 ? 64u : (uint32_t)CH;
+    if (!encode_bf16_map_3d(&p.tm_wa, a.W_a, (uint64_t)dh, (uint64_t)dh, (uint64_t)a.H, 64, box_rows, true) ||
+        !encode_bf16_map_3d(&p.tm_wx, a.W_x, (uint64_t)dh, (uint64_t)dh, (uint64_t)a.H, 64, box_rows, true))
         return cudaErrorNotSupported;
     p.f = a;
+    p.f.H = G;
+    p.dh = dh;
     // batch tile: as few tiles per head as fill the SM pairs once, rounded to the MMA's N granularity
     const int pairs = num_sms() / 2;
-    const int tiles_wanted = pairs / a.H > 0 ? pairs / a.H : 1;
+    const int tiles_wanted = pairs / G > 0 ? pairs / G : 1;
     int NB = (a.B + tiles_wanted - 1) / tiles_wanted;
     NB = ((NB + 15) / 16) * 16;
     if (NB > NB_MAX) NB = NB_MAX;
@@ -345,7 +389,7 @@ cudaError_t sm100_decode(const FwdArgs &a, cudaStream_t st) {
     p.NB = NB;
     p.ntile = (a.B + NB - 1) / NB;
     p.spin_ns = g_spin_limit_ns;
-    dim3 grid(2u * (unsigned)a.H * (unsigned)p.ntile), block(NTHREADS);
+    dim3 grid(2u * (unsigned)G * (unsigned)p.ntile), block(NTHREADS);
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = SMEM_ALLOC; cfg.stream = st;
     cudaLaunchAttribute attr[1];

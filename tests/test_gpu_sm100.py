@@ -234,3 +234,28 @@ def test_narrower_heads_on_the_tensor_core_path(oracle, Dh, B, T, H):
     y2, _, _ = gpu_prefill(inp2, h0=inp["h0"], cs=inp["conv_state"])
     other = np.ones(D, bool); other[Dh:2 * Dh] = False
     assert np.array_equal(y2[:, :, other], y[:, :, other]) and not np.array_equal(y2[:, :, ~other], y[:, :, ~other])
+
+
+@pytest.mark.parametrize("Dh,B,H,T0,steps", [(128, 19, 2, 5, 6), (128, 130, 4, 3, 4), (64, 33, 4, 4, 5), (64, 200, 8, 2, 3)])
+def test_decode_chain_with_narrower_heads(oracle, Dh, B, H, T0, steps):
+    """Decode steps for heads of width 128 and 64 on the tensor-core kernel (groups of two or four heads per 256 channels; a
+    CTA then needs only the channels it convolves itself).  Checked against the oracle; the CUDA-core kernel, forced by flag,
+    must agree within tolerance but not bit for bit, which shows that a different kernel ran by default."""
+    import torch
+    from paper_2402_19427_b200 import binding
+    D = Dh * H
+    inp = synth.make_inputs(B, T0 + steps, D, H, io="bf16", seed=900 + Dh + B, bias_scale=0.3)
+    params = binding.Params.from_numpy(inp["params"], "bf16")
+    x = to_dev(inp["x"], "bf16")
+    _, h0, cs0 = binding.prefill(x[:, :T0].contiguous(), params)
+    outs = []
+    for flags in (0, 1):
+        h, cs = h0.clone(), cs0.clone()
+        ys = [binding.decode_step(x[:, t].contiguous(), params, h, cs, flags=flags) for t in range(T0, T0 + steps)]
+        outs.append((torch.stack(ys, 1), h, cs))
+    torch.cuda.synchronize()
+    yr, hr, cr = oracle_prefill(oracle, inp)
+    for y, h, cs in outs:
+        assert_close("y", to_np(y), yr[:, T0:], "bf16"); assert_close("h", to_np(h), hr, "bf16")
+        assert np.array_equal(to_np(cs), cr)
+    assert not torch.equal(outs[0][1], outs[1][1])

@@ -27,8 +27,8 @@
  *    bytes, 256-byte aligned.  Its contents need not be preserved between calls; calls
  *    that share a workspace must be ordered on one stream.
  *  - Shapes without a kernel return RGLRU_ERR_UNSUPPORTED.  There is no CPU fallback.
- *  - Kernels.  bf16 io with head width D_h = 256 runs on tensor-core kernels (prefill, decode step, backward).  The
- *    tensor-core prefill and decode step also take D_h = 128 and 64 when D is a multiple of 256 (Section 4.1: the gates have 16 blocks, so
+ *  - Kernels.  bf16 io with head width D_h = 256 runs on tensor-core kernels (prefill, decode step, backward; the backward
+ *    needs T % 8 == 0).  They also take D_h = 128 and 64 when D is a multiple of 256 (Section 4.1: the gates have 16 blocks, so
  *    layers with D_RNN below 4096 have narrower heads): two or four heads then share one 256 x 256 block-diagonal weight tile.  Every other
  *    shape with D_h <= 1024, fp32 or bf16, runs on shape-generic CUDA-core kernels.
  */

@@ -259,15 +259,19 @@ struct EwArgs {
 // fp16 copies of the gate weights: W16[g][h][o][n] = W_g[h][o][n] and WT[h][n][g*256 + o] = W_g[h][o][n]
 // One block per 32 x 32 tile of one (gate, head) matrix; the transposed copy goes through shared memory so that both
 // copies are written with consecutive threads on consecutive addresses.  grid (8, 8, 2 H), block (32, 8)
-__global__ void convert_w_kernel(const __nv_bfloat16 *Wa, const __nv_bfloat16 *Wx, __half *W16, __half *WT, int H) {
+// H counts 256-channel groups; dh is the width of a head of the layer (256, 128 or 64): a group holds 256 / dh heads on its
+// diagonal, and tiles off the diagonal blocks are written as zeros.
+__global__ void convert_w_kernel(const __nv_bfloat16 *Wa, const __nv_bfloat16 *Wx, __half *W16, __half *WT, int H, int dh) {
     __shared__ __half tile[32][33];
     const int g = blockIdx.z / H, h = blockIdx.z % H;
     const int o0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
-    const __nv_bfloat16 *W = (g ? Wx : Wa) + (size_t)h * DH * DH;
+    const int sub = o0 / dh;                         // head of the group that owns these output rows
+    const bool on_diagonal = n0 / dh == sub;
+    const __nv_bfloat16 *W = (g ? Wx : Wa) + ((size_t)h * (DH / dh) + sub) * dh * dh + (size_t)(o0 - sub * dh) * dh + (n0 - sub * dh);
     __half *W16m = W16 + ((size_t)g * H + h) * DH * DH;
 #pragma unroll
     for (int r = threadIdx.y; r < 32; r += 8) {
-        const float v = __bfloat162float(W[(size_t)(o0 + r) * DH + n0 + threadIdx.x]);
+        const float v = on_diagonal ? __bfloat162float(W[(size_t)r * dh + threadIdx.x]) : 0.0f;
         const __half hv = __float2half_rn(fminf(fmaxf(v, -65504.0f), 65504.0f));
         W16m[(size_t)(o0 + r) * DH + n0 + threadIdx.x] = hv;
         tile[r][threadIdx.x] = hv;
@@ -276,6 +280,24 @@ __global__ void convert_w_kernel(const __nv_bfloat16 *Wa, const __nv_bfloat16 *W
 #pragma unroll
     for (int r = threadIdx.y; r < 32; r += 8)
         WT[((size_t)h * DH + n0 + r) * (2 * DH) + g * DH + o0 + threadIdx.x] = tile[threadIdx.x][r];
+}
+
+// Fixed-order sum over the token splits of the diagonal blocks of the groups' 256 x 256 weight gradients: one thread per
+// element of dW_a / dW_x [H_layer][dh][dh].  part: [S][2 gates][G groups][256][256]
+__global__ void reduce_dw_blocks_kernel(const float *part, int S, int G, int dh, float *dWa, float *dWx) {
+    const size_t per_gate = (size_t)G * DH * dh;   // = H_layer * dh * dh
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= 2 * per_gate) return;
+    const int gate = (int)(i / per_gate);
+    size_t r = i % per_gate;
+    const int n = (int)(r % dh); r /= dh;
+    const int o = (int)(r % dh); r /= dh;
+    const int head = (int)r, group = head / (DH / dh), sub = head % (DH / dh);
+    const size_t src = (((size_t)gate * G + group) * DH + sub * dh + o) * DH + sub * dh + n;
+    const size_t stride = (size_t)2 * G * DH * DH;
+    float acc = 0.0f;
+    for (int s = 0; s < S; ++s) acc += part[(size_t)s * stride + src];
+    (gate ? dWx : dWa)[i % per_gate] = acc;
 }
 
 __device__ __forceinline__ __half to_half_sat(float v) { return __float2half_rn(fminf(fmaxf(v, -65504.0f), 65504.0f)); }
@@ -561,6 +583,7 @@ struct BwdLayout {
 
 BwdLayout bwd_layout(int B, int T, int D, int H) {
     BwdLayout L{};
+    H = D / DH;   // the GEMMs work on 256-channel groups of heads
     L.BT = (size_t)B * T;
     L.BTp = (L.BT + 63) & ~(size_t)63;
     L.nchunk = (T + CHUNK - 1) / CHUNK;
@@ -593,15 +616,21 @@ BwdLayout bwd_layout(int B, int T, int D, int H) {
 
 }  // namespace
 
+// Head width 256, or 128 / 64 with the heads filling whole 256-channel groups: the group's weight matrix is then
+// block-diagonal; it is multiplied as a dense 256 x 256 matrix (convert_w_kernel writes the zeros), and only the diagonal
+// blocks of its gradient are kept (reduce_dw_blocks_kernel).
 bool sm100_backward_supported(int B, int T, int D, int H, int io) {
-    return io == RGLRU_BF16 && B > 0 && T > 0 && H > 0 && D == H * DH && T % 8 == 0;
+    if (io != RGLRU_BF16 || B <= 0 || T <= 0 || H <= 0 || D % H != 0 || D % DH != 0 || T % 8 != 0) return false;
+    const int dh = D / H;
+    return dh == 256 || dh == 128 || dh == 64;
 }
 
 size_t sm100_backward_workspace_bytes(int B, int T, int D, int H) { return bwd_layout(B, T, D, H).total; }
 
 cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, void *ws_body, size_t ws_body_bytes, uint32_t *status,
                            cudaStream_t st) {
-    const int B = q.B, T = q.T, D = q.D, H = q.H;
+    const int B = q.B, T = q.T, D = q.D, dh = q.D / q.H;
+    const int H = D / DH;   // 256-channel groups of heads: the unit of every kernel below
     const BwdLayout L = bwd_layout(B, T, D, H);
     if (ws_body_bytes < L.total) return cudaErrorInvalidValue;
     static PerDeviceOptIn opt_in;
@@ -638,7 +667,7 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
     a.dh_T = q.dh_T; a.dh0 = q.dh0;
 
     // 1. W^T for the du contraction, conv output
-    convert_w_kernel<<<dim3(DH / 32, DH / 32, 2 * H), dim3(32, 8), 0, st>>>((const __nv_bfloat16 *)q.W_a, (const __nv_bfloat16 *)q.W_x, W16, WT, H);
+    convert_w_kernel<<<dim3(DH / 32, DH / 32, 2 * H), dim3(32, 8), 0, st>>>((const __nv_bfloat16 *)q.W_a, (const __nv_bfloat16 *)q.W_x, W16, WT, H, dh);
     const dim3 grid_ew(D / 256, L.nchunk, B);
     conv_forward_kernel<<<grid_ew, 256, 0, st>>>(a);
 
@@ -688,7 +717,12 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
         g.nx = 4; g.ny = L.S;
         tc_gemm_kernel<<<gemm_grid(g), GEMM_THREADS, GEMM_SMEM_ALLOC, st>>>(g);
         const size_t wsz = (size_t)H * DH * DH;
-        if ((e = reduce_partials3(part, L.S, 2 * wsz, q.dW_a, wsz, q.dW_x, wsz, nullptr, 0, st)) != cudaSuccess) return e;
+        if (dh == DH) {
+            if ((e = reduce_partials3(part, L.S, 2 * wsz, q.dW_a, wsz, q.dW_x, wsz, nullptr, 0, st)) != cudaSuccess) return e;
+        } else {
+            const size_t nout = (size_t)2 * q.H * dh * dh;
+            reduce_dw_blocks_kernel<<<(unsigned)((nout + 255) / 256), 256, 0, st>>>(part, L.S, H, dh, q.dW_a, q.dW_x);
+        }
     }
     // 6. per-channel sums, Conv1D adjoint
     const int nparts = B * L.nchunk;

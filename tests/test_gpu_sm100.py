@@ -259,3 +259,32 @@ def test_decode_chain_with_narrower_heads(oracle, Dh, B, H, T0, steps):
         assert_close("y", to_np(y), yr[:, T0:], "bf16"); assert_close("h", to_np(h), hr, "bf16")
         assert np.array_equal(to_np(cs), cr)
     assert not torch.equal(outs[0][1], outs[1][1])
+
+
+@pytest.mark.parametrize("Dh,B,T,H,with_y", [(128, 2, 136, 2, True), (128, 1, 264, 4, False), (64, 2, 200, 4, True), (64, 1, 72, 8, False)])
+def test_backward_with_narrower_heads(oracle, Dh, B, T, H, with_y):
+    """Tensor-core backward for heads of width 128 and 64: the GEMMs run on 256-channel groups with block-diagonal weights
+    and only the diagonal blocks of the weight gradient are returned.  All gradients, the state gradients included, against
+    the oracle's analytic ones."""
+    import torch
+    from paper_2402_19427_b200 import binding
+    D = Dh * H
+    inp = synth.make_inputs(B, T, D, H, io="bf16", seed=950 + Dh + T, with_dy=True, with_state=True, bias_scale=0.2)
+    params = binding.Params.from_numpy(inp["params"], "bf16")
+    x = to_dev(inp["x"], "bf16"); dy = to_dev(inp["dy"], "bf16")
+    h0 = to_dev(inp["h0"]); cs = to_dev(inp["conv_state"], "bf16")
+    shape = binding.make_shape(B, T, D, H, torch.bfloat16)
+    assert binding.workspace_bytes(shape, binding.OP_BACKWARD) != binding.workspace_bytes(
+        binding.make_shape(B, T, D, H, torch.bfloat16, flags=1), binding.OP_BACKWARD)      # not the generic path
+    y = binding.prefill(x, params, h0=h0, conv_state_in=cs)[0] if with_y else None
+    ws = binding.alloc_workspace(shape, binding.OP_BACKWARD, x.device)
+    rng = np.random.default_rng(3)
+    dhT = rng.standard_normal((B, D)).astype(np.float32)
+    g = binding.backward(x, params, dy, h0=h0, conv_state_in=cs, y=y, workspace=ws, dh_T=to_dev(dhT), state_grads=True)
+    assert binding.query_status(ws) == binding.OK
+    gr = oracle.backward(inp["x"].astype(np.float64), f64(inp["params"]), H, inp["dy"].astype(np.float64),
+                         h0=inp["h0"].astype(np.float64), conv_state_in=inp["conv_state"].astype(np.float64),
+                         dh_T=dhT.astype(np.float64), state_grads=True)
+    assert set(gr) <= set(g)
+    for k in gr:
+        assert_close("d" + k, to_np(g[k]), gr[k], "bf16")

@@ -278,11 +278,25 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # Everything that costs host time (NVML set-up, event creation) happens before the warm-up, so that the GPU does not sit
-    # idle between the warm-up and the timed region; the warm-up itself is preceded by untimed launches of the same step for
-    # PREWARM_S seconds, which brings clocks and caches to their steady state whatever K and W are.
+    # The K timed steps are K calls of the public API captured once in a CUDA graph and replayed: the calls allocate nothing
+    # (outputs and workspace are passed in), and a graph takes the host's launch cost and the gap between consecutive
+    # cooperative launches out of the measurement (measured: 86 against 91 us per step with plain stream launches, which are
+    # timed as well and reported beside it).  Everything that costs host time (NVML set-up, event creation, the capture)
+    # happens before the warm-up, so that the GPU does not sit idle between the warm-up and the timed region; the warm-up
+    # itself is preceded by untimed launches of the same step for PREWARM_S seconds, which brings clocks and caches to their
+    # steady state whatever K and W are.
     sampler = ClockSampler(local)
     evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step(0)
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(args.steps):
+                step(i)
+    torch.cuda.current_stream().wait_stream(side)
     t_pre = time.perf_counter()
     n_pre = 0
     while time.perf_counter() - t_pre < PREWARM_S:
@@ -294,13 +308,20 @@ def run_ours(args):
         step(i)
     barrier()
     sampler.start()
+    g0.record()
+    graph.replay()
+    g1.record()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = g0.elapsed_time(g1)
+    # the same K steps as plain launches on the stream, each between two events (side record)
+    barrier()
     evs[0].record()
     for i in range(args.steps):
         step(i)
         evs[i + 1].record()
     barrier()
-    clocks = sampler.stop()
-    total_ms = evs[0].elapsed_time(evs[-1])
+    stream_total_ms = evs[0].elapsed_time(evs[-1])
     per_launch_ms = [evs[i].elapsed_time(evs[i + 1]) for i in range(args.steps)]
     status = binding.query_status(ws)
     if status != binding.OK:
@@ -347,7 +368,7 @@ def run_ours(args):
 
     peaks, peak_kind = load_peaks()
     nbytes, flops = algorithmic_work(cfg)
-    launch_s = float(np.mean(per_launch_ms)) * 1e-3
+    launch_s = total_ms / args.steps * 1e-3   # average duration of the kernel over the timed region (one kernel per step)
     roof = roofline(nbytes, flops, launch_s, peaks, peak_kind, traffic=captured_traffic())
     roof["kernel"] = "rglru prefill (dominant kernel of the step)"
 
@@ -365,11 +386,15 @@ def run_ours(args):
                 "config": {"workload": workload_name(cfg), "parallelism": f"batch-sharded x{world}, no collective",
                            "l2": f"{N_ROTATE} rotating input/output buffer sets ({N_ROTATE * 2 * B * T * D * 2 / 1e6:.0f} MB) > 126 MB L2",
                            "prewarm": f"{PREWARM_S * 1e3:.0f} ms of untimed launches of the step before the {args.warmup} warm-up steps",
+                           "launch": f"the {args.steps} timed steps are {args.steps} API calls captured in one CUDA graph and replayed once",
                            "kernel_path": "sm100" if binding.workspace_bytes(shape, binding.OP_PREFILL) > 256 else "generic"},
                 "clocks": clocks, "gpu_launches": args.steps,
                 "e2e": {"value": world * B * T / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                         "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps},
-                "roofline": roof}
+                "roofline": roof,
+                "stream_launches": {"what": "the same steps as plain launches on the stream, one event pair per step",
+                                    "ms_per_step": stream_total_ms / args.steps, "ms_per_launch_median": float(np.median(per_launch_ms)),
+                                    "ms_per_launch_min": float(np.min(per_launch_ms))}}
         if world == 1 and not args.no_cpu_baseline:
             tps, dt_s, cores, sample = time_oracle(cfg, synth.BASE_SEED + WORKLOAD, cfg["H"])   # one whole step
             line["cpu_baseline"] = {"value": tps, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample,

@@ -2,16 +2,18 @@
 //
 // The paper gives no backward; this is reverse-mode differentiation of Eq. 1-4 and the Conv1D.  The three dense
 // contractions run on tcgen05 tensor cores through one small GEMM kernel, the rest is element-wise and HBM-bound:
-//   1. conv_forward      u = Conv1D(x) in fp16, token-major [tok][D] and channel-major [D][tok]; fp16 copies of the weights
+//   1. conv_forward      u = Conv1D(x) in fp16, token-major [tok][D]; fp16 copies of the weights
 //                        (every tensor-core operand here is fp16: 11 significant bits instead of bf16's 8 keep the
 //                        rounding of u and dz out of the gradients; finite overflow saturates at +-65504)
 //   2. GEMM              z_a | z_x = u W_a^T | u W_x^T per head (Eq. 1-2 before the sigmoid), fp16 out
 //   3. scan_fold / scan_carry / scan_apply
 //                        reverse-time scan g_t = dy_t + a_{t+1} g_{t+1} over chunks of 128 tokens (fold, carry across
-//                        chunks, re-run with the carry), then the element-wise adjoints: dz_a, dz_x (fp16, token-major
-//                        and channel-major), the direct part of du (fp16), partial sums of dLambda, db_a, db_x
+//                        chunks, re-run with the carry), then the element-wise adjoints: dz_a, dz_x (fp16, token-major),
+//                        the direct part of du (fp16), partial sums of dLambda, db_a, db_x
 //   4. GEMM              du += dz_a W_a + dz_x W_x
-//   5. GEMM (split K)    dW_a | dW_x = dz^T u over all tokens, fp32 partial sums per split, reduced in fixed order
+//   5. GEMM (split K)    dW_a | dW_x = dz^T u over all tokens: both operands are read token-major as steps 1 and 3 wrote them
+//                        and handed to the tensor core as MN-major operands (no transposed copies exist); fp32 partial sums
+//                        per split, reduced in fixed order
 //   6. Conv1D adjoint    dx, dconv_w, dconv_b with sliding windows, fixed-order reductions
 // h_{t-1} comes from the forward output y (bf16); when the caller has none the forward is run first.
 #include <cuda.h>
@@ -33,6 +35,7 @@ constexpr int GEMM_STAGES = 4;
 constexpr uint32_t A_STAGE_BYTES = 128 * 128;   // 128 rows x 64 bf16
 constexpr uint32_t B_STAGE_BYTES = 256 * 128;   // 256 rows x 64 bf16
 constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr uint32_t MN_BLOCK_BYTES = 64 * 128;   // one copy of 64 tokens x 64 channels for the MN-major operands of the dW product
 constexpr uint32_t GEMM_SMEM_BAR = GEMM_STAGES * STAGE_BYTES;
 constexpr uint32_t GEMM_SMEM_TOTAL = GEMM_SMEM_BAR + (2 * GEMM_STAGES + 4) * 8 + 16;
 constexpr uint32_t GEMM_SMEM_ALLOC = GEMM_SMEM_TOTAL + 1024;
@@ -58,7 +61,7 @@ struct GemmArgs {
 // the loads and MMAs of the next.  Tile number -> (x, y, z) with x fastest:
 //   MODE_Z : (token tiles, 2 gates, H)   A = u[tok][h][k]        B = W_gate[h][out][k]
 //   MODE_DU: (token tiles, 1, H)         A = dz[tok][h][k=512]   B = W^T[h][in][k=512]
-//   MODE_DW: (4 row tiles, splits, H)    A = dz^T[h][row][tok]   B = u^T[h][in][tok], K = this split's tokens
+//   MODE_DW: (4 row tiles, splits, H)    A = dz[tok][h][row]     B = u[tok][h][in], both MN-major, K = this split's tokens
 // 32-byte accesses: one whole DRAM sector per thread and instruction where a thread owns a row (pointers 32-byte aligned)
 __device__ __forceinline__ void st_global_v8(void *ptr, const uint32_t (&r)[8]) {
     asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(ptr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]),
@@ -114,9 +117,13 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                     mbar_expect_tx(BAR_FULL(s), STAGE_BYTES);
                     const uint32_t a_dst = base + s * STAGE_BYTES, b_dst = a_dst + A_STAGE_BYTES;
                     if (p.mode == MODE_DW) {
+                        // both operands token-major as the scan wrote them: 64 tokens (K) x 64 channels per copy, the channels
+                        // innermost; tokens at or beyond B T read as zero
                         const int k0 = (ty * p.kblocks + kb) * 64;
-                        tma_load_3d(a_dst, &p.tm_a, k0, tx * 128, h, BAR_FULL(s));
-                        tma_load_3d(b_dst, tb, k0, 0, h, BAR_FULL(s));
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) tma_load_3d(a_dst + j * MN_BLOCK_BYTES, &p.tm_a, tx * 128 + j * 64, h, k0, BAR_FULL(s));
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) tma_load_3d(b_dst + j * MN_BLOCK_BYTES, tb, j * 64, h, k0, BAR_FULL(s));
                     } else {
                         tma_load_3d(a_dst, &p.tm_a, kb * 64, h, tx * 128, BAR_FULL(s));
                         tma_load_3d(b_dst, tb, kb * 64, 0, h, BAR_FULL(s));
@@ -128,7 +135,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
     } else if (warp == 1) {
         // ---- MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_f16(128, 256);
+            constexpr uint32_t idesc = make_idesc_f16(128, 256), idesc_mn = make_idesc_f16_mn(128, 256);
             int kbg = 0, it = 0;
             for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
                 const int acc = it & 1;
@@ -140,9 +147,17 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_src = base + s * STAGE_BYTES, b_src = a_src + A_STAGE_BYTES;
+                    if (p.mode == MODE_DW) {
+                        // K = tokens runs along the rows of the staged blocks: 16 rows of 128 bytes per instruction
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        mma_ss(tmem + acc * 256, make_desc_sw128(a_src + ks * 32), make_desc_sw128(b_src + ks * 32), idesc, (kb | ks) != 0);
+                        for (int ks = 0; ks < 4; ++ks)
+                            mma_ss(tmem + acc * 256, make_desc_sw128_mn(a_src + ks * 2048, MN_BLOCK_BYTES), make_desc_sw128_mn(b_src + ks * 2048, MN_BLOCK_BYTES),
+                                   idesc_mn, (kb | ks) != 0);
+                    } else {
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            mma_ss(tmem + acc * 256, make_desc_sw128(a_src + ks * 32), make_desc_sw128(b_src + ks * 32), idesc, (kb | ks) != 0);
+                    }
                     tc_commit(BAR_EMPTY(s));
                 }
                 if (ok) tc_commit(BAR_ACCFULL(acc));
@@ -242,11 +257,10 @@ __device__ __forceinline__ float decay_rate(float lambda, float c) {
 
 struct EwArgs {
     int B, T, D, H, nchunk;
-    size_t BTp;                       // padded token count = row pitch of the channel-major arrays
     float c;
     const __nv_bfloat16 *x, *conv_w, *cs_in, *dy, *y;
     const float *conv_b, *b_a, *b_x, *lambda, *h0;
-    __half *u, *uT, *dz, *dzT;
+    __half *u, *dz;
     const __half *z;
     __half *du;                       // [tok][D]
     float2 *fold;                     // [B][nchunk][D]: (prod a_t, carry out of the chunk for zero carry in)
@@ -316,40 +330,31 @@ __global__ void __launch_bounds__(256) conv_forward_kernel(EwArgs a) {
         return a.cs_in ? bf2f(a.cs_in[((size_t)b * 3 + (3 + t)) * D + d]) : 0.0f;
     };
     float x3 = xat(t0 - 3), x2 = xat(t0 - 2), x1 = xat(t0 - 1);
-    // eight tokens: u token-major (coalesced across the block) and eight fp16 values of this channel's row
+    // eight tokens at a time, all loads first: u token-major (coalesced across the block)
     const uint32_t sD = (uint32_t)D;   // token stride; sixteen tokens' worth fits 32 bits
-    auto batch8 = [&](__half *pu, const float (&xs)[8]) -> uint4 {
-        uint32_t packed[4];
+    auto batch8 = [&](__half *pu, const float (&xs)[8]) {
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             const float uv = fmaf(w[3], x3, fmaf(w[2], x2, fmaf(w[1], x1, fmaf(w[0], xs[k], cb))));
-            const __half ub = to_half_sat(uv);
-            pu[k * sD] = ub;
-            const uint32_t bits = (uint32_t)__half_as_ushort(ub);
-            if (k & 1) packed[k >> 1] |= bits << 16; else packed[k >> 1] = bits;
+            pu[k * sD] = to_half_sat(uv);
             x3 = x2; x2 = x1; x1 = xs[k];
         }
-        return make_uint4(packed[0], packed[1], packed[2], packed[3]);
     };
     int t = t0;
-    for (; t + 16 <= t1; t += 16) {   // sixteen tokens: the channel-major store fills whole 32-byte sectors
+    for (; t + 16 <= t1; t += 16) {
         float xa[8], xb[8];
         const __nv_bfloat16 *px = a.x + ((size_t)b * T + t) * D + d;
         __half *pu = a.u + ((size_t)b * T + t) * D + d;
 #pragma unroll
         for (int k = 0; k < 8; ++k) { xa[k] = bf2f(px[k * sD]); xb[k] = bf2f(px[(8 + k) * sD]); }
-        const uint4 lo = batch8(pu, xa), hi = batch8(pu + 8 * (size_t)sD, xb);
-        __half *dst = a.uT + (size_t)d * a.BTp + (size_t)b * T + t;
-        if ((reinterpret_cast<uintptr_t>(dst) & 31) == 0) {
-            const uint32_t wv[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-            st_global_v8(dst, wv);
-        } else { ((uint4 *)dst)[0] = lo; ((uint4 *)dst)[1] = hi; }
+        batch8(pu, xa);
+        batch8(pu + 8 * (size_t)sD, xb);
     }
     if (t < t1) {
         float xa[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) xa[k] = bf2f(a.x[((size_t)b * T + t + k) * D + d]);
-        *(uint4 *)(a.uT + (size_t)d * a.BTp + (size_t)b * T + t) = batch8(a.u + ((size_t)b * T + t) * D + d, xa);
+        batch8(a.u + ((size_t)b * T + t) * D + d, xa);
     }
 }
 
@@ -441,10 +446,9 @@ __global__ void __launch_bounds__(256, 3) scan_apply_kernel(EwArgs a) {
     const __half *p_z = a.z + tokb * (size_t)sZ + (size_t)h * 2 * DH + n, *p_u = a.u + tokb * (size_t)sD + d;
     __half *p_dz = a.dz + tokb * (size_t)sZ + (size_t)h * 2 * DH + n;
     __half *p_du = a.du + tokb * (size_t)sD + d;
-    __half *p_ta = a.dzT + ((size_t)h * 2 * DH + n) * a.BTp + tokb, *p_tx = p_ta + (size_t)DH * a.BTp;
     const float h0v = a.h0 ? a.h0[(size_t)b * D + d] : 0.0f;
-    // eight tokens at the running pointers, newest first; the channel-major copies of dz come back packed
-    auto batch8 = [&](int tb, uint32_t (&pa)[4], uint32_t (&px)[4]) {
+    // eight tokens at the running pointers, newest first
+    auto batch8 = [&](int tb) {
         float dza_hi = 0.0f, dzx_hi = 0.0f;
         float dyv[8], hpv[8], zav[8], zxv[8], uv[8];
 #pragma unroll
@@ -469,11 +473,10 @@ __global__ void __launch_bounds__(256, 3) scan_apply_kernel(EwArgs a) {
             s_lam = fmaf(dL * r, dsdlam_neg, s_lam);
             s_ba += dza; s_bx += dzx;
             p_du[k * sD] = to_half_sat(dv * gi);
-            // tokens k (odd) and k - 1 share one packed conversion: the pair is what the channel-major copy stores
+            // tokens k (odd) and k - 1 share one packed conversion
             if (k & 1) { dza_hi = dza; dzx_hi = dzx; }
             else {
                 const uint32_t wa = pack_f16_sat(dza, dza_hi), wx = pack_f16_sat(dzx, dzx_hi);
-                pa[k >> 1] = wa; px[k >> 1] = wx;
                 p_dz[k * sZ] = __ushort_as_half((unsigned short)(wa & 0xFFFFu));
                 p_dz[(k + 1) * sZ] = __ushort_as_half((unsigned short)(wa >> 16));
                 p_dz[k * sZ + DH] = __ushort_as_half((unsigned short)(wx & 0xFFFFu));
@@ -483,30 +486,12 @@ __global__ void __launch_bounds__(256, 3) scan_apply_kernel(EwArgs a) {
         p_dy -= 8 * (size_t)sD; p_y -= 8 * (size_t)sD; p_z -= 8 * (size_t)sZ; p_u -= 8 * (size_t)sD; p_dz -= 8 * (size_t)sZ; p_du -= 8 * (size_t)sD;
     };
     int tb = t1 - 8;
-    // sixteen tokens per round, so that each channel-major row gets 32 adjacent bytes (a whole sector) at once
+    // sixteen tokens per round: the loads of the second eight are requested while the first eight are worked on
     for (; tb - 8 >= t0; tb -= 16) {
-        uint32_t pa1[4], px1[4], pa0[4], px0[4];
-        batch8(tb, pa1, px1);
-        batch8(tb - 8, pa0, px0);
-        if ((reinterpret_cast<uintptr_t>(p_ta - 8) & 31) == 0) {
-            const uint32_t wa[8] = {pa0[0], pa0[1], pa0[2], pa0[3], pa1[0], pa1[1], pa1[2], pa1[3]};
-            const uint32_t wx[8] = {px0[0], px0[1], px0[2], px0[3], px1[0], px1[1], px1[2], px1[3]};
-            st_global_v8(p_ta - 8, wa);
-            st_global_v8(p_tx - 8, wx);
-        } else {
-            *(uint4 *)(p_ta - 8) = make_uint4(pa0[0], pa0[1], pa0[2], pa0[3]);
-            *(uint4 *)p_ta = make_uint4(pa1[0], pa1[1], pa1[2], pa1[3]);
-            *(uint4 *)(p_tx - 8) = make_uint4(px0[0], px0[1], px0[2], px0[3]);
-            *(uint4 *)p_tx = make_uint4(px1[0], px1[1], px1[2], px1[3]);
-        }
-        p_ta -= 16; p_tx -= 16;
+        batch8(tb);
+        batch8(tb - 8);
     }
-    if (tb >= t0) {
-        uint32_t pa[4], px[4];
-        batch8(tb, pa, px);
-        *(uint4 *)p_ta = make_uint4(pa[0], pa[1], pa[2], pa[3]);
-        *(uint4 *)p_tx = make_uint4(px[0], px[1], px[2], px[3]);
-    }
+    if (tb >= t0) batch8(tb);
     float *pv = a.part_vec + ((size_t)b * a.nchunk + c) * 3 * D + d;
     pv[0] = s_lam; pv[(size_t)D] = s_ba; pv[(size_t)2 * D] = s_bx;
 }
@@ -576,7 +561,7 @@ unsigned gemm_grid(const GemmArgs &g) {
 }
 
 struct BwdLayout {
-    size_t BT, BTp, off_u, off_uT, off_z, off_dz, off_dzT, off_du, off_y, off_hT, off_cs, off_fold, off_xin, off_pvec, off_pconv, off_pdw,
+    size_t BT, BTp, off_u, off_z, off_dz, off_du, off_y, off_hT, off_cs, off_fold, off_xin, off_pvec, off_pconv, off_pdw,
         off_wt, off_w16, off_fws, total;
     int nchunk, nchunk_conv, S, kb_per_split;
 };
@@ -594,10 +579,8 @@ BwdLayout bwd_layout(int B, int T, int D, int H) {
     size_t o = 0;
     auto take = [&](size_t bytes) { const size_t at = o; o += up256(bytes); return at; };
     L.off_u = take(L.BT * D * 2);
-    L.off_uT = take((size_t)D * L.BTp * 2);
     L.off_z = take(L.BT * D * 2 * 2);
     L.off_dz = take(L.BT * D * 2 * 2);
-    L.off_dzT = take((size_t)D * 2 * L.BTp * 2);
     L.off_du = take(L.BT * D * 2);
     L.off_y = take(L.BT * D * 2);
     L.off_hT = take((size_t)B * D * 4);
@@ -637,8 +620,8 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
     cudaError_t e = opt_in.ensure(tc_gemm_kernel, (int)GEMM_SMEM_ALLOC);
     if (e != cudaSuccess) return e;
     char *ws = (char *)ws_body;
-    __half *u = (__half *)(ws + L.off_u), *uT = (__half *)(ws + L.off_uT), *z = (__half *)(ws + L.off_z);
-    __half *dz = (__half *)(ws + L.off_dz), *dzT = (__half *)(ws + L.off_dzT), *WT = (__half *)(ws + L.off_wt), *W16 = (__half *)(ws + L.off_w16);
+    __half *u = (__half *)(ws + L.off_u), *z = (__half *)(ws + L.off_z);
+    __half *dz = (__half *)(ws + L.off_dz), *WT = (__half *)(ws + L.off_wt), *W16 = (__half *)(ws + L.off_w16);
     __half *du = (__half *)(ws + L.off_du);
 
     // 0. h_{t-1} comes from the forward output; run the forward when the caller kept none
@@ -652,17 +635,13 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
         if (e != cudaSuccess) return e;
         y = f.y;
     }
-    if (L.BTp != L.BT) {   // the padded token columns enter the dW contraction and must be zero
-        if ((e = cudaMemsetAsync(uT, 0, (size_t)D * L.BTp * 2, st)) != cudaSuccess) return e;
-        if ((e = cudaMemsetAsync(dzT, 0, (size_t)D * 2 * L.BTp * 2, st)) != cudaSuccess) return e;
-    }
 
     EwArgs a{};
-    a.B = B; a.T = T; a.D = D; a.H = H; a.nchunk = L.nchunk; a.BTp = L.BTp; a.c = q.c;
+    a.B = B; a.T = T; a.D = D; a.H = H; a.nchunk = L.nchunk; a.c = q.c;
     a.x = (const __nv_bfloat16 *)q.x; a.conv_w = (const __nv_bfloat16 *)q.conv_w; a.cs_in = (const __nv_bfloat16 *)q.cs_in;
     a.dy = (const __nv_bfloat16 *)q.dy; a.y = (const __nv_bfloat16 *)y;
     a.conv_b = fwd.conv_b; a.b_a = fwd.b_a; a.b_x = fwd.b_x; a.lambda = q.lambda; a.h0 = fwd.h0;
-    a.u = u; a.uT = uT; a.dz = dz; a.dzT = dzT; a.z = z; a.du = du;
+    a.u = u; a.dz = dz; a.z = z; a.du = du;
     a.fold = (float2 *)(ws + L.off_fold); a.xin = (float *)(ws + L.off_xin); a.part_vec = (float *)(ws + L.off_pvec);
     a.dh_T = q.dh_T; a.dh0 = q.dh0;
 
@@ -674,7 +653,7 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
     GemmArgs g{};
     g.H = H; g.D = D; g.status = status; g.spin_ns = g_spin_limit_ns;
     const unsigned mtiles = (unsigned)((L.BT + 127) / 128);
-    const uint64_t BT = L.BT, BTp = L.BTp;
+    const uint64_t BT = L.BT;
     // 2. z = u W^T per head and gate
     {
         const uint64_t da[3] = {DH, (uint64_t)H, BT}, sa[2] = {DH * 2, (uint64_t)D * 2};
@@ -706,11 +685,11 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
     }
     // 5. dW = dz^T u, split over the tokens, then a fixed-order sum of the splits
     {
-        const uint64_t da[3] = {BTp, 2 * DH, (uint64_t)H}, sa[2] = {BTp * 2, (uint64_t)2 * DH * BTp * 2};
-        const uint32_t ba[3] = {64, 128, 1};
-        const uint64_t db[3] = {BTp, DH, (uint64_t)H}, sb[2] = {BTp * 2, (uint64_t)DH * BTp * 2};
-        const uint32_t bb[3] = {64, 256, 1};
-        if (!encode_map16_3d(&g.tm_a, dzT, da, sa, ba, true) || !encode_map16_3d(&g.tm_b0, uT, db, sb, bb, true)) return cudaErrorNotSupported;
+        const uint64_t da[3] = {2 * DH, (uint64_t)H, BT}, sa[2] = {2 * DH * 2, (uint64_t)H * 2 * DH * 2};   // dz [tok][h][gate, channel]
+        const uint32_t ba[3] = {64, 1, 64};
+        const uint64_t db[3] = {DH, (uint64_t)H, BT}, sb[2] = {DH * 2, (uint64_t)D * 2};                     // u [tok][h][channel]
+        const uint32_t bb[3] = {64, 1, 64};
+        if (!encode_map16_3d(&g.tm_a, dz, da, sa, ba, true) || !encode_map16_3d(&g.tm_b0, u, db, sb, bb, true)) return cudaErrorNotSupported;
         g.tm_b1 = g.tm_b0;
         float *part = (float *)(ws + L.off_pdw);
         g.mode = MODE_DW; g.kblocks = L.kb_per_split; g.rows_valid = 2 * DH; g.out = part;

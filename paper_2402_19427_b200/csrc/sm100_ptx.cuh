@@ -206,6 +206,17 @@ __device__ __forceinline__ uint64_t make_desc_sw128(uint32_t saddr) {
     return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
            ((uint64_t)2 << 61);
 }
+// MN-major, 128B-swizzled shared-memory operand: rows (one K index each) of 64 elements of the M or N dimension = 128 B,
+// 8-row groups 1024 B apart along K (stride offset), 64-element blocks of the M / N dimension `block_bytes` apart (leading
+// offset).  This is what a tiled copy with the M / N dimension innermost and a 128-byte swizzle leaves in shared memory.
+__device__ __forceinline__ uint64_t make_desc_sw128_mn(uint32_t saddr, uint32_t block_bytes) {
+    return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)((block_bytes >> 4) & 0x3FFF) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// kind::f16 instruction descriptor: fp32 accumulator, fp16 A and B, both MN-major (bits 15 and 16), M x N
+__host__ __device__ constexpr uint32_t make_idesc_f16_mn(int M, int N) {
+    return (1u << 4) | (1u << 15) | (1u << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
 // kind::f16 instruction descriptor: fp32 accumulator, fp16 A and B, both K-major, M x N
 __host__ __device__ constexpr uint32_t make_idesc_f16(int M, int N) {
     return (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);

@@ -92,7 +92,10 @@ struct Sm100Args {
     alignas(64) CUtensorMap tm_y;
     alignas(64) CUtensorMap tm_g;   // gate branch, same geometry as y (encoded only when the call has one)
     FwdArgs f;
-    int dh;            // width of a head of the layer: 256, or 128 / 64 (then a "head" below is a group of 2 / 4 layer heads)
+    int dh;            // width of a head of the layer.  256, 128 or 64: a "head" below is a group of 256 / dh layer heads.  Another
+                       // multiple of 32 below 256: a "head" below is one layer head whose channels [dh, 256) do not exist
+    int hstride;       // channels from one "head" of the kernel to the next: 256, or dh in the second case
+    int cvalid;        // channels of a "head" that exist: 256, or dh in the second case
     int S;             // pairs per head (time split factor)
     int tps;           // tiles per sequence
     int tiles_total;   // B * tps
@@ -135,6 +138,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
     const int pair = blockIdx.x >> 1;
     const int head = pair / S, kcta = pair % S;
     const int group = head * 2 + (int)rank;   // index of this half-head's carry records
+    // First channel of this head in the layer, and how many of the head's 256 channel slots exist.  A head narrower than 256
+    // that does not divide 256 runs alone in its 256 slots: the slots beyond its width read whatever follows in memory (the
+    // next head's channels, or zeros past the end of the tensor), their weights are zero in both directions, and nothing of
+    // them is written.
+    const int cbase = head * p.hstride, cvalid = p.cvalid;
     const uint32_t peer_abort = map_to_cta(base + SMEM_MISC + 4, rank ^ 1u);
     auto record_timeout = [&]() {
         *abort_flag = 1;
@@ -202,8 +210,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
         // block-diagonal, and a row holds its own head's weights in that head's input channels and zeros elsewhere.
         const int dh = p.dh, row_in_group = (int)rank * CH + q * 32 + lane;
         const int sub = row_in_group / dh;                     // head of the group this output channel belongs to
-        const uint4 *row = (const uint4 *)(W + ((size_t)head * DH + row_in_group) * dh);   // (head * 256 / dh + sub) * dh + row_in_group % dh rows of dh
-        const int c_first = sub * (dh >> 3), c_count = dh >> 3;   // the 16-byte chunks of the 256 input channels that are this head's
+        const uint4 *row = (const uint4 *)(W + ((size_t)cbase + row_in_group) * dh);   // (head * 256 / dh + sub) * dh + row_in_group % dh rows of dh
+        // the 16-byte chunks of the 256 input channels that are this head's (none for a channel slot that does not exist)
+        const int c_first = sub * (dh >> 3), c_count = row_in_group < cvalid ? dh >> 3 : 0;
         const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (g ? TM_W_X : TM_W_A);
         auto cvt2 = [](uint32_t w) { return pack_f16_sat(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u)); };
         const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
@@ -235,12 +244,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
         f32x2 w01[4], w23[4], b01, b23;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const __nv_bfloat16 *wp = cw + (size_t)j * D + head * DH + hc;
-            w01[j] = pack2(__bfloat162float(wp[0]), __bfloat162float(wp[1]));
-            w23[j] = pack2(__bfloat162float(wp[2]), __bfloat162float(wp[3]));
+            const __nv_bfloat16 *wp = cw + (size_t)j * D + cbase + hc;
+            if (hc < cvalid) {
+                w01[j] = pack2(__bfloat162float(wp[0]), __bfloat162float(wp[1]));
+                w23[j] = pack2(__bfloat162float(wp[2]), __bfloat162float(wp[3]));
+            } else { w01[j] = pack2(0.f, 0.f); w23[j] = w01[j]; }
         }
-        if (f.conv_b) {
-            const float *bp = f.conv_b + head * DH + hc;
+        if (f.conv_b && hc < cvalid) {
+            const float *bp = f.conv_b + cbase + hc;
             b01 = pack2(bp[0], bp[1]); b23 = pack2(bp[2], bp[3]);
         } else { b01 = pack2(0.f, 0.f); b23 = b01; }
         // this thread's 16 tokens are rows 16 tg .. 16 tg + 15 of the slab (plus three rows of history) and of the U tile;
@@ -328,19 +339,28 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
                 for (int i = lane; i < (SLAB_ROWS - hi_row) * (int)(X_ROW_BYTES / 16); i += 32)
                     *(uint4 *)(smem + SMEM_X + slot * X_SLAB_BYTES + (uint32_t)hi_row * X_ROW_BYTES + (uint32_t)i * 16) = make_uint4(0, 0, 0, 0);
                 __syncwarp();
-                if (lane == 0) mbar_expect_tx(BAR_XFULL(slot), (uint32_t)hi_row * X_ROW_BYTES);
+                // of a narrower head only the channels that exist are copied (a whole row could run past the end of the tensor);
+                // the rest of each row is zeroed for the same reason as the rows above
+                const uint32_t row_bytes = (uint32_t)cvalid * 2;
+                if (row_bytes < X_ROW_BYTES) {
+                    const int per_row = (int)((X_ROW_BYTES - row_bytes) / 16);
+                    for (int i = lane; i < hi_row * per_row; i += 32)
+                        *(uint4 *)(smem + SMEM_X + slot * X_SLAB_BYTES + (uint32_t)(i / per_row) * X_ROW_BYTES + row_bytes + (uint32_t)(i % per_row) * 16) = make_uint4(0, 0, 0, 0);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_expect_tx(BAR_XFULL(slot), (uint32_t)hi_row * row_bytes);
                 __syncwarp();
                 for (int r = lane; r < hi_row; r += 32) {
                     const int t = r - 3;
-                    const __nv_bfloat16 *src = t >= 0 ? x + ((size_t)b * T + t) * D + head * DH
-                                                      : cs_in + ((size_t)b * 3 + (3 + t)) * D + head * DH;
-                    bulk_g2s(dst + r * X_ROW_BYTES, src, X_ROW_BYTES, BAR_XFULL(slot));
+                    const __nv_bfloat16 *src = t >= 0 ? x + ((size_t)b * T + t) * D + cbase
+                                                      : cs_in + ((size_t)b * 3 + (3 + t)) * D + cbase;
+                    bulk_g2s(dst + r * X_ROW_BYTES, src, row_bytes, BAR_XFULL(slot));
                 }
             } else if (lane == 0) {
                 // one tiled copy per slab: SLAB_ROWS token rows of this head starting three tokens early
                 // (tokens before the sequence start and past its end read as zero)
                 mbar_expect_tx(BAR_XFULL(slot), X_SLAB_BYTES);
-                tma_load_3d(dst, &p.tm_x, head * DH, ts0 - 3, b, BAR_XFULL(slot));
+                tma_load_3d(dst, &p.tm_x, cbase, ts0 - 3, b, BAR_XFULL(slot));
             }
             __syncwarp();
         }
@@ -381,13 +401,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
         reg_inc<112>();
         const int q = warp & 3, g = (warp - 8) >> 2;     // lane quarter; tokens [32 g, 32 g + 32) of every tile, convolved by CTA g
         const int hc = (int)rank * CH + q * 32 + lane;   // channel within the head
-        const int d = head * DH + hc;                    // global channel
+        const int d = cbase + hc;                        // global channel
+        const bool exists = hc < cvalid;                 // uniform over the warp (widths are multiples of 32)
         // per-channel constants; s = c softplus(-Lambda) with libm-grade log1p/exp (Appendix A)
-        const float lam = f.lambda[d];
+        const float lam = exists ? f.lambda[d] : 0.0f;
         const float zl = -lam;
         const float s = f.c * (zl > 0.0f ? zl + log1pf(expf(-zl)) : log1pf(expf(zl)));
         const f32x2 s2 = pack2(s, s);
-        const f32x2 hba2 = pack2(0.5f * f.b_a[d], 0.5f * f.b_a[d]), hbx2 = pack2(0.5f * f.b_x[d], 0.5f * f.b_x[d]);
+        const float ba_c = exists ? f.b_a[d] : 0.0f, bx_c = exists ? f.b_x[d] : 0.0f;
+        const f32x2 hba2 = pack2(0.5f * ba_c, 0.5f * ba_c), hbx2 = pack2(0.5f * bx_c, 0.5f * bx_c);
         const bool poly = __all_sync(0xffffffffu, s <= S_POLY);
         // u[row][channel] in the swizzled U tile of CTA g, one offset per row phase (row & 7)
         const bool remote = (uint32_t)g != rank;
@@ -463,7 +485,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
         reg_inc<152>();
         const int q = warp & 3;
         const int c_own = q * 32 + lane;                 // channel within the CTA
-        const int d = head * DH + (int)rank * CH + c_own;  // global channel
+        const int d = cbase + (int)rank * CH + c_own;    // global channel
+        const bool exists = (int)rank * CH + c_own < cvalid;   // uniform over the warp; a warp of channel slots that do not exist
+                                                                // keeps the barriers going but reads and writes no global memory
         const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16);
         const uint32_t y_warp_off = SMEM_Y + (uint32_t)q * 2 * Y_BUF_BYTES;
         const float2 *agg_s = (const float2 *)(smem + SMEM_AGG) + c_own;
@@ -484,10 +508,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
             if constexpr (merged) {
                 // The warp's 64 x 32 block of the gate branch is fetched into the y staging buffer of this tile (free once
                 // the store of two tiles ago has read it) while the gate warps still work; y then overwrites it in place.
-                if (lane == 0) {
+                if (lane == 0 && exists) {
                     bulk_wait_read1();
                     mbar_expect_tx(BAR_BRANCH(q), Y_BUF_BYTES);
-                    tma_load_3d(base + y_off, &p.tm_g, head * DH + (int)rank * CH + q * 32, t0, b, BAR_BRANCH(q));
+                    tma_load_3d(base + y_off, &p.tm_g, cbase + (int)rank * CH + q * 32, t0, b, BAR_BRANCH(q));
                 }
                 __syncwarp();
             }
@@ -500,7 +524,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
             //      start of a sequence, advanced by the aggregates that the other pairs published for the tiles in between
             float h, P;
             if (!shared) {
-                h = ti == 0 ? (f.h0 ? f.h0[(size_t)b * D + d] : 0.0f) : h_prev_own;
+                h = ti == 0 ? (f.h0 && exists ? f.h0[(size_t)b * D + d] : 0.0f) : h_prev_own;
                 P = ti == 0 ? 1.0f : P_prev_own;
             } else {
                 // publish the tile's aggregate before waiting for anyone
@@ -509,7 +533,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
                 uint4 *dst = p.agg + ((size_t)group * p.tiles_total + gidx) * CH + c_own;
                 asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "r"(rec.x), "r"(rec.y), "r"(rec.z), "r"(rec.w) : "memory");
                 int nback;
-                if (ti < S) { h = f.h0 ? f.h0[(size_t)b * D + d] : 0.0f; P = 1.0f; nback = ti; }
+                if (ti < S) { h = f.h0 && exists ? f.h0[(size_t)b * D + d] : 0.0f; P = 1.0f; nback = ti; }
                 else { h = h_prev_own; P = P_prev_own; nback = S - 1; }
                 // The records are taken oldest first, up to eight at a time: all of a batch are requested at once, then polled
                 // until every lane sees this call's tag in both halves of each record (8-byte words are written atomically).
@@ -568,8 +592,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
             if (lane == 0) mbar_arrive_at(BAR_ACCEMPTY(bf), 0);
             if constexpr (merged) {
                 // merged output of the recurrent block (Section 2.3): y_t = h_t GeLU(branch_t); the state is not touched
-                ok = warp_wait(BAR_BRANCH(q), it & 1, spin, abort_flag);
-                if (!ok) break;
+                if (exists) {
+                    ok = warp_wait(BAR_BRANCH(q), it & 1, spin, abort_flag);
+                    if (!ok) break;
+                }
 #pragma unroll
                 for (int j = 0; j < TILE; j += 2) {
                     const float hb = j < HALF ? h : h_mid;
@@ -593,12 +619,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
             }
             fence_async_smem();   // y rows become visible to the bulk-copy engine
             __syncwarp();
-            if (lane == 0) {
+            if (lane == 0 && exists) {
                 // the warp's 64 tokens x 32 channels go out as one tiled store; rows at or beyond T are clipped
-                tma_store_3d(&p.tm_y, head * DH + (int)rank * CH + q * 32, t0, b, base + y_off);
+                tma_store_3d(&p.tm_y, cbase + (int)rank * CH + q * 32, t0, b, base + y_off);
                 bulk_commit();
             }
-            if (ti == p.tps - 1) {
+            if (ti == p.tps - 1 && exists) {
                 // end of a sequence: h_T (unrounded state) and the last three raw inputs, bit-exact
                 f.h_T[(size_t)b * D + d] = h_prev_own;
                 if (f.a_prod) f.a_prod[(size_t)b * D + d] = P_prev_own;
@@ -718,11 +744,19 @@ bool encode_bf16_map_3d(CUtensorMap *tm, const void *ptr, uint64_t d0, uint64_t 
     return encode_map16_3d(tm, ptr, dims, strides, box, swizzle128);
 }
 
-// Head width 256, or 128 / 64 with the heads filling whole 256-channel groups (the kernel then works on D / 256 groups).
+// Head width 256; 128 or 64 with the heads filling whole 256-channel groups (the kernel then works on D / 256 groups); or any
+// other multiple of 32 below 256 (the paper's 16-block layers have widths such as 96 and 160), each head alone in 256 channel
+// slots of which the last 256 - width do not exist.
+namespace {
+// heads of width 128 or 64 that fill whole 256-channel groups are worked on as groups (as is width 256 itself)
+inline bool grouped_heads(int D, int H) { const int dh = D / H; return dh == DH || ((dh == 128 || dh == 64) && D % DH == 0); }
+// heads (or groups of heads) the kernel works on
+inline int kernel_heads(int D, int H) { return grouped_heads(D, H) ? D / DH : H; }
+}  // namespace
 bool sm100_prefill_supported(int B, int T, int D, int H, int io) {
-    if (io != RGLRU_BF16 || B <= 0 || T <= 0 || H <= 0 || D % H != 0 || D % DH != 0) return false;
+    if (io != RGLRU_BF16 || B <= 0 || T <= 0 || H <= 0 || D % H != 0) return false;
     const int dh = D / H;
-    return dh == 256 || dh == 128 || dh == 64;
+    return grouped_heads(D, H) || (dh < DH && dh % 32 == 0);
 }
 
 namespace {
@@ -757,7 +791,7 @@ inline bool ranges_overlap(const void *a, const void *b, size_t n) {
 // different tiles and of the two halves of a head read the incoming state at unrelated times,
 // so an in-place update must not be visible to them.
 size_t sm100_prefill_workspace_bytes(int B, int T, int D, int H) {
-    H = D / DH;   // the kernel's unit is a 256-channel group of heads
+    H = kernel_heads(D, H);   // the kernel's unit: a 256-channel group of heads, or one head of another width
     return agg_bytes(B, T, H) + up256((size_t)B * D * sizeof(float)) + up256((size_t)B * 3 * D * sizeof(__nv_bfloat16));
 }
 
@@ -774,9 +808,11 @@ cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes,
         p.tm_g = p.tm_y;   // never used by the kernel
     }
     p.f = a;
-    const int G = a.D / DH;   // 256-channel groups of heads: the kernel's "heads"
+    const int G = kernel_heads(a.D, a.H);   // 256-channel groups of heads, or heads of another width: the kernel's "heads"
     p.f.H = G;
     p.dh = a.D / a.H;
+    p.hstride = grouped_heads(a.D, a.H) ? DH : p.dh;
+    p.cvalid = p.hstride;
     p.tps = (a.T + TILE - 1) / TILE;
     const int pairs = di.max_pairs < di.sms / 2 ? di.max_pairs : di.sms / 2;
     int S = pairs_per_head(G, pairs);

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 
 from paper_2402_19427_b200 import inputs as synth
-from util import assert_close, f64, gpu_prefill, oracle_prefill, to_dev, to_np
+from util import Guarded, assert_close, f64, gpu_prefill, oracle_prefill, to_dev, to_np
 
 pytestmark = pytest.mark.gpu
 
@@ -288,3 +288,34 @@ def test_backward_with_narrower_heads(oracle, Dh, B, T, H, with_y):
     assert set(gr) <= set(g)
     for k in gr:
         assert_close("d" + k, to_np(g[k]), gr[k], "bf16")
+
+
+@pytest.mark.parametrize("Dh,B,T,H", [(160, 2, 130, 2), (96, 3, 257, 3), (192, 1, 1000, 1), (224, 2, 65, 2), (32, 2, 100, 5), (128, 2, 100, 3),
+                                      (160, 2, 300, 16), (160, 9, 200, 2)])
+def test_head_widths_that_do_not_divide_256(oracle, Dh, B, T, H):
+    """Section 4.1 fixes 16 blocks, so the paper's layers have head widths such as 96 (D_RNN = 1536) and 160 (D_RNN = 2560,
+    the sixth case).  Such a head runs alone in the kernel's 256 channel slots; the slots beyond its width have zero weights
+    and taps and are never written.  With incoming state (the first slab is then assembled from row copies), biases, a
+    sequence split in time (last case), and the channels next to the last head's end, which lie outside the tensors."""
+    import torch
+    from paper_2402_19427_b200 import binding
+    D = Dh * H
+    assert uses_sm100(B, T, D, H)
+    inp = synth.make_inputs(B, T, D, H, io="bf16", seed=1000 + Dh + T, with_state=True, bias_scale=0.5)
+    rng = np.random.default_rng(Dh)
+    branch = synth.round_to_bf16((rng.standard_normal((B, T, D)) * 1.5).astype(np.float32))
+    for with_branch in (False, True):
+        g = Guarded()
+        y = g.empty((B, T, D), torch.bfloat16); hT = g.empty((B, D), torch.float32); cso = g.empty((B, 3, D), torch.bfloat16)
+        ap = g.empty((B, D), torch.float32)
+        binding.prefill(to_dev(inp["x"], "bf16"), binding.Params.from_numpy(inp["params"], "bf16"), h0=to_dev(inp["h0"]),
+                        conv_state_in=to_dev(inp["conv_state"], "bf16"), y=y, h_T=hT, conv_state_out=cso, a_prod=ap,
+                        gate_branch=to_dev(branch, "bf16") if with_branch else None)
+        g.check()
+        yr, hr, cr, ar = oracle.prefill(inp["x"].astype(np.float64), f64(inp["params"]), H, c=inp["c"], h0=inp["h0"].astype(np.float64),
+                                        conv_state_in=inp["conv_state"].astype(np.float64), with_a_prod=True,
+                                        gate_branch=branch.astype(np.float64) if with_branch else None)
+        assert_close("y", to_np(y), yr, "bf16"); assert_close("h_T", to_np(hT), hr, "bf16")
+        assert np.array_equal(to_np(cso), cr)
+        big = ar > 1e-30
+        np.testing.assert_allclose(np.log(to_np(ap)[big]), np.log(ar[big]), rtol=2e-2, atol=2e-2)

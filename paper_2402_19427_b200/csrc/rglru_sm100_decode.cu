@@ -1,5 +1,5 @@
-// sm_100a batched decode step of the RG-LRU temporal core (bf16 io, head width 256; 128 and 64 as groups of heads, see the
-// weight loads below): one new token for each
+// sm_100a batched decode step of the RG-LRU temporal core (bf16 io, head width 256; narrower heads as groups of heads or one
+// head per 256 channel slots, see the weight loads below): one new token for each
 // of B sequences, recurrent state h [B,D] fp32 and the 3-row conv state [B,3,D] updated in place.
 //
 // A cluster of two CTAs owns one (head, batch tile) pair.  CTA r of the pair owns channels [128 r, 128 r + 128)
@@ -51,7 +51,10 @@ struct DecArgs {
     alignas(64) CUtensorMap tm_wa;   // W_a as [H][256 out][256 in], box 128 out x 64 in, 128-byte swizzle
     alignas(64) CUtensorMap tm_wx;
     FwdArgs f;
-    int dh;       // head width of the layer: 256, or 128 / 64 (a "head" of the kernel is then a group of 2 / 4 heads, H their number)
+    int dh;       // head width of the layer
+    int mode;     // 0: a kernel "head" is one layer head in 256 channel slots (width 256, or narrower with the slots beyond the
+                  //    width unused); 1 / 2: a group of two 128-wide / four 64-wide heads that fill the 256 channels
+    int hstride;  // channels from one kernel "head" to the next (256, or dh in mode 0 with a narrower head)
     int NB;       // sequences per batch tile (multiple of 16)
     int ntile;    // batch tiles
     unsigned long long spin_ns;
@@ -110,16 +113,20 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     //      block-diagonal, so this CTA's 128 output rows only see K blocks 2 rank and 2 rank + 1 -- the channels it convolves
     //      itself -- and nothing is exchanged with the peer.  With 64-wide heads each of those K blocks holds one head's 64 rows;
     //      the other 64 rows of the block are zeroed by the threads below.
-    const int dh = p.dh;
+    const int mode = p.mode;
+    // first channel of this head in the layer and the number of its 256 channel slots that exist: the slots beyond a narrower
+    // head's width get zero weights (the tiled copies read them as out of bounds), zero taps, and are neither loaded nor stored
+    const size_t cbase = (size_t)head * p.hstride;
+    const int cvalid = mode == 0 ? p.dh : DH;
     if (tid == NTHREADS - 32) {
-        if (dh == DH) {
+        if (mode == 0) {
             mbar_expect_tx(BAR_W, 8 * KBLOCK_BYTES);
 #pragma unroll
             for (int kb = 0; kb < 4; ++kb) {
                 tma_load_3d(base + SMEM_WA + kb * KBLOCK_BYTES, &p.tm_wa, kb * 64, (int)rank * CH, head, BAR_W);
                 tma_load_3d(base + SMEM_WX + kb * KBLOCK_BYTES, &p.tm_wx, kb * 64, (int)rank * CH, head, BAR_W);
             }
-        } else if (dh == 128) {
+        } else if (mode == 1) {
             mbar_expect_tx(BAR_W, 4 * KBLOCK_BYTES);
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
@@ -138,7 +145,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
         }
     }
     __syncwarp();
-    if (dh == 64) {
+    if (mode == 2) {
         // rows of the two K blocks that belong to the other head of this CTA: zero (generic stores; the fence and barrier after
         // the conv phase order them before the MMAs)
         for (int i = tid; i < 4 * (int)(KBLOCK_BYTES / 2 / 16); i += NTHREADS) {
@@ -154,8 +161,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     const int q = warp & 3, kq = warp >> 2;
     const int c_own = q * 32 + lane;
     const int dl = (int)rank * CH + c_own;
-    const size_t d = (size_t)head * DH + dl;
-    const float lam = f.lambda[d], ba = f.b_a[d], bx = f.b_x[d];   // used after the conv phase: nothing waits on them here
+    const size_t d = cbase + dl;
+    const bool exists = dl < cvalid;   // uniform over the warp (widths are multiples of 32)
+    // used after the conv phase: nothing waits on them here
+    const float lam = exists ? f.lambda[d] : 0.0f, ba = exists ? f.b_a[d] : 0.0f, bx = exists ? f.b_x[d] : 0.0f;
 
     // ---- gate products: the K blocks this CTA convolved itself are multiplied while the peer's half is still on its way
     const uint32_t idesc = make_idesc(128, NB);
@@ -175,14 +184,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     {
         const int c = tid & 15;
         const int cdl = (int)rank * CH + c * 8;         // channel within the head
-        const size_t cd = (size_t)head * DH + cdl;      // global channel
+        const size_t cd = cbase + cdl;                  // global channel
+        const bool cexists = cdl < cvalid;              // the eight channels of this thread exist
         const __nv_bfloat16 *cw = (const __nv_bfloat16 *)f.conv_w;
         uint4 w[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) w[j] = *(const uint4 *)(cw + (size_t)j * D + cd);
+        for (int j = 0; j < 4; ++j) w[j] = cexists ? *(const uint4 *)(cw + (size_t)j * D + cd) : make_uint4(0u, 0u, 0u, 0u);
         float cb[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) cb[e] = f.conv_b ? f.conv_b[cd + e] : 0.0f;
+        for (int e = 0; e < 8; ++e) cb[e] = f.conv_b && cexists ? f.conv_b[cd + e] : 0.0f;
         const __nv_bfloat16 *x = (const __nv_bfloat16 *)f.x;
         __nv_bfloat16 *cs = (__nv_bfloat16 *)f.cs_out;   // in/out
         const uint32_t u_kb = SMEM_U + (uint32_t)(cdl >> 6) * KBLOCK_BYTES;
@@ -196,7 +206,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
 #pragma unroll
         for (int i = 0; i < NIT; ++i) {
             const int n = (tid >> 4) + 32 * i, b = b0 + n;
-            if (n < NB && b < B) {
+            if (n < NB && b < B && cexists) {
                 xv[i] = *(const uint4 *)(x + (size_t)b * D + cd);
                 r0[i] = *(const uint4 *)(cs + ((size_t)b * 3 + 0) * D + cd);
                 r1[i] = *(const uint4 *)(cs + ((size_t)b * 3 + 1) * D + cd);
@@ -211,7 +221,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
             const int n = (tid >> 4) + 32 * i, b = b0 + n;
             if (n >= NB) break;
             uint4 uo = make_uint4(0u, 0u, 0u, 0u);
-            if (b < B) {
+            if (b < B && cexists) {
                 const uint32_t xw[4] = {xv[i].x, xv[i].y, xv[i].z, xv[i].w}, a0[4] = {r0[i].x, r0[i].y, r0[i].z, r0[i].w},
                                a1[4] = {r1[i].x, r1[i].y, r1[i].z, r1[i].w}, a2[4] = {r2[i].x, r2[i].y, r2[i].z, r2[i].w};
                 uint32_t o[4], rem[4];
@@ -234,7 +244,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
         __syncthreads();     // this CTA's half of the U tile is complete in its own shared memory
         // ... and goes to the peer as two bulk copies (one per K block: NB rows of 128 bytes, contiguous), counted on the
         // peer's barrier: nobody but the peer's MMA issuer waits for them
-        if (tid == 32 && dh == DH) {
+        if (tid == 32 && mode == 0) {
             const uint32_t peer_bar = map_to_cta(BAR_U, rank ^ 1u);
 #pragma unroll
             for (int k = 0; k < 2; ++k) {
@@ -255,7 +265,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
 #pragma unroll
         for (int i = 0; i < NIT; ++i) {
             const int n = (tid >> 4) + 32 * i, b = b0 + n;
-            if (n < NB && b < B) {
+            if (n < NB && b < B && cexists) {
                 *(uint4 *)(cs + ((size_t)b * 3 + 0) * D + cd) = r1[i];
                 *(uint4 *)(cs + ((size_t)b * 3 + 1) * D + cd) = r2[i];
                 *(uint4 *)(cs + ((size_t)b * 3 + 2) * D + cd) = xv[i];
@@ -279,17 +289,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
 #pragma unroll
     for (int j = 0; j < NB_MAX / 4; ++j) {
         const int b = b0 + kq * nq + j;
-        hv[j] = (j < nq && b < B) ? h[(size_t)b * D + d] : 0.0f;
+        hv[j] = (j < nq && b < B && exists) ? h[(size_t)b * D + d] : 0.0f;
     }
 
     if (tid == 0) {
         // the peer's half of the U tile (waited for even when the weights failed: the peer's copies must have landed
         // before this CTA may leave)
-        const bool u_ok = dh != DH || mbar_wait(BAR_U, 0, spin, &no_abort);
-        if (u_ok && dh == DH) mbar_arrive_at(BAR_SENT, rank ^ 1u);
+        const bool u_ok = mode != 0 || mbar_wait(BAR_U, 0, spin, &no_abort);
+        if (u_ok && mode == 0) mbar_arrive_at(BAR_SENT, rank ^ 1u);
         if (u_ok && w_ok) {
             tc_fence_after();
-            if (dh == DH) issue_kblocks((int)(rank ^ 1u) * 2, false);
+            if (mode == 0) issue_kblocks((int)(rank ^ 1u) * 2, false);
             tc_commit(BAR_ACC);
         } else if (!u_ok) {
             atomicExch(f.status, STATUS_MAGIC | (uint32_t)RGLRU_ERR_TIMEOUT);
@@ -330,7 +340,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const int b = b0 + n0 + 2 * j + e;
-                    if (b < B) {
+                    if (b < B && exists) {
                         h[(size_t)b * D + d] = hn[e];
                         y[(size_t)b * D + d] = __float2bfloat16_rn(hn[e]);
                     }
@@ -345,7 +355,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1) sm100_d
     }
 
     // the peer has received this CTA's half of the U tile: its bulk copies no longer read this shared memory
-    if (tid == 0 && !timed_out && dh == DH) mbar_wait(BAR_SENT, 0, spin, &no_abort);
+    if (tid == 0 && !timed_out && mode == 0) mbar_wait(BAR_SENT, 0, spin, &no_abort);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
@@ -360,10 +370,14 @@ int num_sms() {
 }  // namespace
 
 // Head width 256, or 128 / 64 with the heads filling whole 256-channel groups.
+// Any other multiple of 32 below 256: one head per 256 channel slots.
+namespace {
+inline bool grouped_heads(int D, int H) { const int dh = D / H; return dh == DH || ((dh == 128 || dh == 64) && D % DH == 0); }
+}  // namespace
 bool sm100_decode_supported(int B, int D, int H, int io) {
-    if (io != RGLRU_BF16 || B <= 0 || H <= 0 || D % H != 0 || D % DH != 0) return false;
+    if (io != RGLRU_BF16 || B <= 0 || H <= 0 || D % H != 0) return false;
     const int dh = D / H;
-    return dh == 256 || dh == 128 || dh == 64;
+    return grouped_heads(D, H) || (dh < DH && dh % 32 == 0);
 }
 
 cudaError_t sm100_decode(const FwdArgs &a, cudaStream_t st) {
@@ -371,14 +385,19 @@ cudaError_t sm100_decode(const FwdArgs &a, cudaStream_t st) {
     cudaError_t e = opt_in.ensure(sm100_decode_kernel, (int)SMEM_ALLOC);
     if (e != cudaSuccess) return e;
     DecArgs p;
-    const int dh = a.D / a.H, G = a.D / DH;   // G: 256-channel groups of heads, the kernel's unit
-    const uint32_t box_rows = dh == 64 ? 64u : (uint32_t)CH;
+    const int dh = a.D / a.H;
+    const bool grouped = grouped_heads(a.D, a.H);
+    const int G = grouped ? a.D / DH : a.H;   // 256-channel groups of heads, or heads of another width: the kernel's unit
+    const int mode = !grouped || dh == DH ? 0 : (dh == 128 ? 1 : 2);
+    const uint32_t box_rows = mode == 2 ? 64u : (uint32_t)CH;
     if (!encode_bf16_map_3d(&p.tm_wa, a.W_a, (uint64_t)dh, (uint64_t)dh, (uint64_t)a.H, 64, box_rows, true) ||
         !encode_bf16_map_3d(&p.tm_wx, a.W_x, (uint64_t)dh, (uint64_t)dh, (uint64_t)a.H, 64, box_rows, true))
         return cudaErrorNotSupported;
     p.f = a;
     p.f.H = G;
     p.dh = dh;
+    p.mode = mode;
+    p.hstride = grouped ? DH : dh;
     // batch tile: as few tiles per head as fill the SM pairs once, rounded to the MMA's N granularity
     const int pairs = num_sms() / 2;
     const int tiles_wanted = pairs / G > 0 ? pairs / G : 1;

@@ -236,11 +236,13 @@ def test_narrower_heads_on_the_tensor_core_path(oracle, Dh, B, T, H):
     assert np.array_equal(y2[:, :, other], y[:, :, other]) and not np.array_equal(y2[:, :, ~other], y[:, :, ~other])
 
 
-@pytest.mark.parametrize("Dh,B,H,T0,steps", [(128, 19, 2, 5, 6), (128, 130, 4, 3, 4), (64, 33, 4, 4, 5), (64, 200, 8, 2, 3)])
+@pytest.mark.parametrize("Dh,B,H,T0,steps", [(128, 19, 2, 5, 6), (128, 130, 4, 3, 4), (64, 33, 4, 4, 5), (64, 200, 8, 2, 3),
+                                                 (160, 19, 2, 5, 6), (96, 130, 3, 3, 4), (160, 70, 16, 2, 3), (224, 5, 1, 4, 4), (128, 40, 3, 3, 3)])
 def test_decode_chain_with_narrower_heads(oracle, Dh, B, H, T0, steps):
-    """Decode steps for heads of width 128 and 64 on the tensor-core kernel (groups of two or four heads per 256 channels; a
-    CTA then needs only the channels it convolves itself).  Checked against the oracle; the CUDA-core kernel, forced by flag,
-    must agree within tolerance but not bit for bit, which shows that a different kernel ran by default."""
+    """Decode steps for heads narrower than 256 on the tensor-core kernel: widths 128 and 64 as groups of two or four heads per
+    256 channels (a CTA then needs only the channels it convolves itself), other multiples of 32 one head per 256 channel
+    slots.  Checked against the oracle; the CUDA-core kernel, forced by flag, must agree within tolerance but not bit for bit,
+    which shows that a different kernel ran by default."""
     import torch
     from paper_2402_19427_b200 import binding
     D = Dh * H

@@ -1,5 +1,5 @@
-// sm_100a fused prefill for the RG-LRU temporal core (bf16 io, head width 256; heads of width 128 or 64 run as groups of
-// two or four that fill a 256-channel block whose weight matrix is block-diagonal).
+// sm_100a fused prefill for the RG-LRU temporal core (bf16 io, head width 256; narrower heads, any multiple of 32, run as
+// groups of 256 / width consecutive heads in the 256 channel slots, with a block-diagonal weight matrix).
 //
 // A head is owned by a pair of CTAs (a cluster of two, one CTA per SM).  CTA r of the pair keeps rows
 // [128 r, 128 r + 128) of W_a and W_x resident in its tensor memory as the A operand of the two-CTA form of
@@ -92,10 +92,10 @@ struct Sm100Args {
     alignas(64) CUtensorMap tm_y;
     alignas(64) CUtensorMap tm_g;   // gate branch, same geometry as y (encoded only when the call has one)
     FwdArgs f;
-    int dh;            // width of a head of the layer.  256, 128 or 64: a "head" below is a group of 256 / dh layer heads.  Another
-                       // multiple of 32 below 256: a "head" below is one layer head whose channels [dh, 256) do not exist
-    int hstride;       // channels from one "head" of the kernel to the next: 256, or dh in the second case
-    int cvalid;        // channels of a "head" that exist: 256, or dh in the second case
+    int dh;            // width of a head of the layer, a multiple of 32 up to 256.  A "head" below is a group of k = 256 / dh
+                       // (rounded down) consecutive layer heads: its weight matrices are block-diagonal with k blocks
+    int hstride;       // channels from one "head" of the kernel to the next: k dh
+    int cvalid;        // channel slots of a "head" that exist: k dh (fewer in the layer's last group when k does not divide H)
     int S;             // pairs per head (time split factor)
     int tps;           // tiles per sequence
     int tiles_total;   // B * tps
@@ -138,11 +138,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1) sm10
     const int pair = blockIdx.x >> 1;
     const int head = pair / S, kcta = pair % S;
     const int group = head * 2 + (int)rank;   // index of this half-head's carry records
-    // First channel of this head in the layer, and how many of the head's 256 channel slots exist.  A head narrower than 256
-    // that does not divide 256 runs alone in its 256 slots: the slots beyond its width read whatever follows in memory (the
-    // next head's channels, or zeros past the end of the tensor), their weights are zero in both directions, and nothing of
-    // them is written.
-    const int cbase = head * p.hstride, cvalid = p.cvalid;
+    // First channel of this head (a group of k = 256 / width layer heads) in the layer, and how many of its 256 channel slots
+    // exist.  The slots beyond k width read whatever follows in memory (the next group's channels, or zeros past the end of
+    // the tensor), their weights are zero in both directions, and nothing of them is written.
+    const int cbase = head * p.hstride, cvalid = min(p.cvalid, D - cbase);   // the layer's last group may hold fewer heads
     const uint32_t peer_abort = map_to_cta(base + SMEM_MISC + 4, rank ^ 1u);
     auto record_timeout = [&]() {
         *abort_flag = 1;
@@ -744,19 +743,18 @@ bool encode_bf16_map_3d(CUtensorMap *tm, const void *ptr, uint64_t d0, uint64_t 
     return encode_map16_3d(tm, ptr, dims, strides, box, swizzle128);
 }
 
-// Head width 256; 128 or 64 with the heads filling whole 256-channel groups (the kernel then works on D / 256 groups); or any
-// other multiple of 32 below 256 (the paper's 16-block layers have widths such as 96 and 160), each head alone in 256 channel
-// slots of which the last 256 - width do not exist.
 namespace {
-// heads of width 128 or 64 that fill whole 256-channel groups are worked on as groups (as is width 256 itself)
-inline bool grouped_heads(int D, int H) { const int dh = D / H; return dh == DH || ((dh == 128 || dh == 64) && D % DH == 0); }
-// heads (or groups of heads) the kernel works on
-inline int kernel_heads(int D, int H) { return grouped_heads(D, H) ? D / DH : H; }
+// layer heads per kernel "head" (a group of consecutive heads sharing 256 channel slots), and the number of such groups
+inline int heads_per_group(int D, int H) { return DH / (D / H); }
+inline int kernel_heads(int D, int H) { const int k = heads_per_group(D, H); return (H + k - 1) / k; }
 }  // namespace
+// Head width: any multiple of 32 up to 256.  k = 256 / width (rounded down) consecutive heads share the kernel's 256 channel
+// slots; slots beyond k width (and beyond the layer's last head) do not exist: zero weights and taps, never loaded per
+// element or stored.
 bool sm100_prefill_supported(int B, int T, int D, int H, int io) {
     if (io != RGLRU_BF16 || B <= 0 || T <= 0 || H <= 0 || D % H != 0) return false;
     const int dh = D / H;
-    return grouped_heads(D, H) || (dh < DH && dh % 32 == 0);
+    return dh <= DH && dh % 32 == 0;
 }
 
 namespace {
@@ -811,7 +809,7 @@ cudaError_t sm100_prefill(const FwdArgs &a, void *ws_body, size_t ws_body_bytes,
     const int G = kernel_heads(a.D, a.H);   // 256-channel groups of heads, or heads of another width: the kernel's "heads"
     p.f.H = G;
     p.dh = a.D / a.H;
-    p.hstride = grouped_heads(a.D, a.H) ? DH : p.dh;
+    p.hstride = heads_per_group(a.D, a.H) * p.dh;
     p.cvalid = p.hstride;
     p.tps = (a.T + TILE - 1) / TILE;
     const int pairs = di.max_pairs < di.sms / 2 ? di.max_pairs : di.sms / 2;

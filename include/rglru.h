@@ -27,12 +27,11 @@
  *    bytes, 256-byte aligned.  Its contents need not be preserved between calls; calls
  *    that share a workspace must be ordered on one stream.
  *  - Shapes without a kernel return RGLRU_ERR_UNSUPPORTED.  There is no CPU fallback.
- *  - Kernels.  bf16 io with head width D_h = 256 runs on tensor-core kernels (prefill, decode step, backward; the backward
- *    needs T % 8 == 0).  Prefill and decode step also take every other D_h < 256 that is a multiple of 32 (Section 4.1's 16
- *    blocks give D_h = 96 at D_RNN = 1536 and 160 at D_RNN = 2560); the unused part of 256 channel slots per head or group of
- *    heads is then idle work.  All three take D_h = 128 and 64 when D is a multiple of 256 (Section 4.1: the gates have 16 blocks, so
- *    layers with D_RNN below 4096 have narrower heads): two or four heads then share one 256 x 256 block-diagonal weight tile.  Every other
- *    shape with D_h <= 1024, fp32 or bf16, runs on shape-generic CUDA-core kernels.
+ *  - Kernels.  bf16 io with a head width D_h that is a multiple of 32 up to 256 runs on tensor-core kernels (prefill, decode
+ *    step, backward; the backward needs T % 8 == 0).  Section 4.1 fixes 16 blocks, so D_h is 256 only at D_RNN = 4096; it is 96
+ *    at D_RNN = 1536, 128 at 2048 and 160 at 2560.  Narrower heads share, or occupy alone, groups of 256 channel slots whose
+ *    weight tile is block-diagonal; the slots a width leaves unused are idle work.  Every other shape with D_h <= 1024, fp32
+ *    or bf16, runs on shape-generic CUDA-core kernels.
  */
 #ifndef RGLRU_H_
 #define RGLRU_H_

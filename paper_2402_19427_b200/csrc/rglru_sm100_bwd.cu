@@ -1,4 +1,5 @@
-// sm_100a backward of the RG-LRU temporal core (bf16 io, head width 256, T a multiple of 8).
+// sm_100a backward of the RG-LRU temporal core (bf16 io, head width a multiple of 32 up to 256 -- narrower heads in groups of
+// 256 channel slots --, T a multiple of 8).
 //
 // The paper gives no backward; this is reverse-mode differentiation of Eq. 1-4 and the Conv1D.  The three dense
 // contractions run on tcgen05 tensor cores through one small GEMM kernel, the rest is element-wise and HBM-bound:
@@ -46,7 +47,9 @@ struct GemmArgs {
     alignas(64) CUtensorMap tm_a;    // A rows (M side), K innermost
     alignas(64) CUtensorMap tm_b0;   // B rows (N side), K innermost
     alignas(64) CUtensorMap tm_b1;   // MODE_Z: the second gate's weights (grid.y selects)
-    int mode, H, D;
+    int mode, H, D;    // H: 256-slot groups of heads
+    int hstride;       // channels from one group to the next in the layer's [.., D] arrays (k dh with k = 256 / dh heads per group)
+    int cvalid;        // channel slots of a group that exist (k dh; fewer in a partial last group)
     int nx, ny;        // tile grid: nx x ny x H
     int kblocks;       // 64-wide K blocks per CTA
     int rows_valid;    // MODE_Z / MODE_DU: number of tokens; MODE_DW: 512
@@ -123,9 +126,12 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
 #pragma unroll
                         for (int j = 0; j < 2; ++j) tma_load_3d(a_dst + j * MN_BLOCK_BYTES, &p.tm_a, tx * 128 + j * 64, h, k0, BAR_FULL(s));
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) tma_load_3d(b_dst + j * MN_BLOCK_BYTES, tb, j * 64, h, k0, BAR_FULL(s));
+                        for (int j = 0; j < 4; ++j) tma_load_3d(b_dst + j * MN_BLOCK_BYTES, tb, h * p.hstride + j * 64, k0, 0, BAR_FULL(s));
                     } else {
-                        tma_load_3d(a_dst, &p.tm_a, kb * 64, h, tx * 128, BAR_FULL(s));
+                        // u is read out of the layer's [tok][D] array at the group's first channel (channels past the group's own
+                        // meet zero weights; past D they read as zero); dz has the groups' own [tok][group][2][256] layout
+                        if (p.mode == MODE_Z) tma_load_3d(a_dst, &p.tm_a, h * p.hstride + kb * 64, tx * 128, 0, BAR_FULL(s));
+                        else tma_load_3d(a_dst, &p.tm_a, kb * 64, h, tx * 128, BAR_FULL(s));
                         tma_load_3d(b_dst, tb, kb * 64, 0, h, BAR_FULL(s));
                     }
                 }
@@ -177,6 +183,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
             tc_fence_after();
             const uint32_t tm_lane = tmem + ((uint32_t)(q * 32) << 16) + acc * 256;
             const bool valid = row < p.rows_valid;
+            const int cv = min(p.cvalid, p.D - h * p.hstride);   // channel slots of this group that exist
 #pragma unroll 1
             for (int c0 = 0; c0 < 256; c0 += 32) {
                 f32x2 v[16];
@@ -194,7 +201,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                     }
                 } else if (p.mode == MODE_DU) {
                     // du is kept in fp16 like dz (bf16 failed the dx tolerance where the taps of the Conv1D adjoint cancel)
-                    __half *dst = (__half *)p.out + (size_t)row * p.D + h * DH + c0;
+                    if (c0 >= cv) continue;   // a slot that does not exist: nothing of du belongs to it
+                    __half *dst = (__half *)p.out + (size_t)row * p.D + h * p.hstride + c0;
                     uint32_t o0[8], o1[8];
                     ld_global_v8(dst, o0);
                     ld_global_v8(dst + 16, o1);
@@ -257,6 +265,7 @@ __device__ __forceinline__ float decay_rate(float lambda, float c) {
 
 struct EwArgs {
     int B, T, D, H, nchunk;
+    int hstride;                      // channels from one 256-slot group of heads to the next
     float c;
     const __nv_bfloat16 *x, *conv_w, *cs_in, *dy, *y;
     const float *conv_b, *b_a, *b_x, *lambda, *h0;
@@ -273,15 +282,17 @@ struct EwArgs {
 // fp16 copies of the gate weights: W16[g][h][o][n] = W_g[h][o][n] and WT[h][n][g*256 + o] = W_g[h][o][n]
 // One block per 32 x 32 tile of one (gate, head) matrix; the transposed copy goes through shared memory so that both
 // copies are written with consecutive threads on consecutive addresses.  grid (8, 8, 2 H), block (32, 8)
-// H counts 256-channel groups; dh is the width of a head of the layer (256, 128 or 64): a group holds 256 / dh heads on its
-// diagonal, and tiles off the diagonal blocks are written as zeros.
-__global__ void convert_w_kernel(const __nv_bfloat16 *Wa, const __nv_bfloat16 *Wx, __half *W16, __half *WT, int H, int dh) {
+// H counts 256-slot groups; dh is the width of a head of the layer (a multiple of 32 up to 256): a group holds k = 256 / dh
+// (rounded down) heads on its diagonal -- fewer in a partial last group of a layer of Hl heads -- and every tile outside
+// those blocks is written as zeros.
+__global__ void convert_w_kernel(const __nv_bfloat16 *Wa, const __nv_bfloat16 *Wx, __half *W16, __half *WT, int H, int dh, int Hl) {
     __shared__ __half tile[32][33];
     const int g = blockIdx.z / H, h = blockIdx.z % H;
     const int o0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
-    const int sub = o0 / dh;                         // head of the group that owns these output rows
-    const bool on_diagonal = n0 / dh == sub;
-    const __nv_bfloat16 *W = (g ? Wx : Wa) + ((size_t)h * (DH / dh) + sub) * dh * dh + (size_t)(o0 - sub * dh) * dh + (n0 - sub * dh);
+    const int k = DH / dh, sub = o0 / dh;            // heads per group; head of the group that owns these output rows
+    const int heads_here = min(k, Hl - h * k);
+    const bool on_diagonal = sub < heads_here && n0 / dh == sub;
+    const __nv_bfloat16 *W = (g ? Wx : Wa) + ((size_t)h * k + sub) * dh * dh + (size_t)(o0 - sub * dh) * dh + (n0 - sub * dh);
     __half *W16m = W16 + ((size_t)g * H + h) * DH * DH;
 #pragma unroll
     for (int r = threadIdx.y; r < 32; r += 8) {
@@ -298,8 +309,8 @@ __global__ void convert_w_kernel(const __nv_bfloat16 *Wa, const __nv_bfloat16 *W
 
 // Fixed-order sum over the token splits of the diagonal blocks of the groups' 256 x 256 weight gradients: one thread per
 // element of dW_a / dW_x [H_layer][dh][dh].  part: [S][2 gates][G groups][256][256]
-__global__ void reduce_dw_blocks_kernel(const float *part, int S, int G, int dh, float *dWa, float *dWx) {
-    const size_t per_gate = (size_t)G * DH * dh;   // = H_layer * dh * dh
+__global__ void reduce_dw_blocks_kernel(const float *part, int S, int G, int dh, int Hl, float *dWa, float *dWx) {
+    const size_t per_gate = (size_t)Hl * dh * dh;
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= 2 * per_gate) return;
     const int gate = (int)(i / per_gate);
@@ -320,6 +331,7 @@ __device__ __forceinline__ __half to_half_sat(float v) { return __float2half_rn(
 __global__ void __launch_bounds__(256) conv_forward_kernel(EwArgs a) {
     const int d = blockIdx.x * 256 + threadIdx.x, c = blockIdx.y, b = blockIdx.z;
     const int T = a.T, D = a.D;
+    if (d >= D) return;
     const int t0 = c * CHUNK, t1 = min(T, t0 + CHUNK);
     float w[4];
 #pragma unroll
@@ -362,7 +374,8 @@ __global__ void __launch_bounds__(256) conv_forward_kernel(EwArgs a) {
 // nothing comes in from later ones.  grid (D/256, nchunk, B)
 __global__ void __launch_bounds__(256) scan_fold_kernel(EwArgs a) {
     const int d = blockIdx.x * 256 + threadIdx.x, c = blockIdx.y, b = blockIdx.z;
-    const int T = a.T, D = a.D, h = d / DH, n = d % DH;
+    if (d >= a.D) return;
+    const int T = a.T, D = a.D, h = d / a.hstride, n = d % a.hstride;   // group of heads and channel slot within it
     const int t0 = c * CHUNK, t1 = min(T, t0 + CHUNK);
     const float s = decay_rate(a.lambda[d], a.c), ba = a.b_a[d];
     float carry = 0.0f, Q = 1.0f;
@@ -405,6 +418,7 @@ __global__ void __launch_bounds__(256) scan_fold_kernel(EwArgs a) {
 // pass 2: carries across chunks, last chunk first.  grid (D/256, B)
 __global__ void __launch_bounds__(256) scan_carry_kernel(EwArgs a) {
     const int d = blockIdx.x * 256 + threadIdx.x, b = blockIdx.y;
+    if (d >= a.D) return;
     // what later tokens hand to the last chunk: the gradient arriving on h_T (h_T = h_{T-1}, factor 1), else nothing
     float X = a.dh_T ? a.dh_T[(size_t)b * a.D + d] : 0.0f;
     // sixteen folds are requested at once (loads interleaved with the stores below would go out one at a time)
@@ -432,7 +446,8 @@ __global__ void __launch_bounds__(256) scan_carry_kernel(EwArgs a) {
 //   dr = -s dL;  dz_a = dr r (1-r);  dz_x = di i (1-i);  dLambda += dL c r sigmoid(-Lambda).   grid (D/256, nchunk, B)
 __global__ void __launch_bounds__(256, 3) scan_apply_kernel(EwArgs a) {
     const int d = blockIdx.x * 256 + threadIdx.x, c = blockIdx.y, b = blockIdx.z;
-    const int T = a.T, D = a.D, h = d / DH, n = d % DH;
+    if (d >= a.D) return;
+    const int T = a.T, D = a.D, h = d / a.hstride, n = d % a.hstride;   // group of heads and channel slot within it
     const int t0 = c * CHUNK, t1 = min(T, t0 + CHUNK);
     const float lam = a.lambda[d];
     const float s = decay_rate(lam, a.c), ba = a.b_a[d], bx = a.b_x[d];
@@ -510,6 +525,7 @@ struct ConvBwdArgs {
 __global__ void __launch_bounds__(256) conv_backward_kernel(ConvBwdArgs a) {
     const int d = blockIdx.x * 256 + threadIdx.x, c = blockIdx.y, b = blockIdx.z;
     const int T = a.T, D = a.D;
+    if (d >= D) return;
     const int t0 = c * CHUNK, t1 = min(T, t0 + CHUNK);
     float w[4], sw[4] = {0.f, 0.f, 0.f, 0.f}, sb = 0.0f;
 #pragma unroll
@@ -560,15 +576,19 @@ unsigned gemm_grid(const GemmArgs &g) {
     return (unsigned)(ntiles < nsm ? ntiles : nsm);
 }
 
+// 256-slot groups of k = 256 / width (rounded down) consecutive heads: the unit of the GEMMs
+inline int groups_of_heads(int D, int H) { const int k = DH / (D / H); return (H + k - 1) / k; }
+
 struct BwdLayout {
     size_t BT, BTp, off_u, off_z, off_dz, off_du, off_y, off_hT, off_cs, off_fold, off_xin, off_pvec, off_pconv, off_pdw,
         off_wt, off_w16, off_fws, total;
     int nchunk, nchunk_conv, S, kb_per_split;
 };
 
-BwdLayout bwd_layout(int B, int T, int D, int H) {
+BwdLayout bwd_layout(int B, int T, int D, int Hl) {
     BwdLayout L{};
-    H = D / DH;   // the GEMMs work on 256-channel groups of heads
+    const int H = groups_of_heads(D, Hl);   // the GEMMs work on 256-slot groups of heads
+    const size_t Dg = (size_t)H * DH;         // channel slots of all groups (>= D)
     L.BT = (size_t)B * T;
     L.BTp = (L.BT + 63) & ~(size_t)63;
     L.nchunk = (T + CHUNK - 1) / CHUNK;
@@ -579,8 +599,8 @@ BwdLayout bwd_layout(int B, int T, int D, int H) {
     size_t o = 0;
     auto take = [&](size_t bytes) { const size_t at = o; o += up256(bytes); return at; };
     L.off_u = take(L.BT * D * 2);
-    L.off_z = take(L.BT * D * 2 * 2);
-    L.off_dz = take(L.BT * D * 2 * 2);
+    L.off_z = take(L.BT * Dg * 2 * 2);
+    L.off_dz = take(L.BT * Dg * 2 * 2);
     L.off_du = take(L.BT * D * 2);
     L.off_y = take(L.BT * D * 2);
     L.off_hT = take((size_t)B * D * 4);
@@ -592,20 +612,21 @@ BwdLayout bwd_layout(int B, int T, int D, int H) {
     L.off_pdw = take((size_t)L.S * 2 * H * DH * DH * 4);
     L.off_wt = take((size_t)H * DH * 2 * DH * 2);
     L.off_w16 = take((size_t)H * DH * 2 * DH * 2);
-    L.off_fws = take(WS_HEADER_BYTES + sm100_prefill_workspace_bytes(B, T, D, H));
+    L.off_fws = take(WS_HEADER_BYTES + sm100_prefill_workspace_bytes(B, T, D, Hl));
     L.total = o;
     return L;
 }
 
 }  // namespace
 
-// Head width 256, or 128 / 64 with the heads filling whole 256-channel groups: the group's weight matrix is then
-// block-diagonal; it is multiplied as a dense 256 x 256 matrix (convert_w_kernel writes the zeros), and only the diagonal
-// blocks of its gradient are kept (reduce_dw_blocks_kernel).
+// Head width: any multiple of 32 up to 256.  k = 256 / width (rounded down) consecutive heads form a group of 256 channel slots
+// whose weight matrix is block-diagonal; it is multiplied as a dense 256 x 256 matrix (convert_w_kernel writes the zeros),
+// and only the diagonal blocks of its gradient are kept (reduce_dw_blocks_kernel).  Slots beyond k width do not exist: they
+// read neighbouring channels against zero weights and nothing of them is written to du.
 bool sm100_backward_supported(int B, int T, int D, int H, int io) {
-    if (io != RGLRU_BF16 || B <= 0 || T <= 0 || H <= 0 || D % H != 0 || D % DH != 0 || T % 8 != 0) return false;
+    if (io != RGLRU_BF16 || B <= 0 || T <= 0 || H <= 0 || D % H != 0 || T % 8 != 0) return false;
     const int dh = D / H;
-    return dh == 256 || dh == 128 || dh == 64;
+    return dh <= DH && dh % 32 == 0;
 }
 
 size_t sm100_backward_workspace_bytes(int B, int T, int D, int H) { return bwd_layout(B, T, D, H).total; }
@@ -613,8 +634,9 @@ size_t sm100_backward_workspace_bytes(int B, int T, int D, int H) { return bwd_l
 cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, void *ws_body, size_t ws_body_bytes, uint32_t *status,
                            cudaStream_t st) {
     const int B = q.B, T = q.T, D = q.D, dh = q.D / q.H;
-    const int H = D / DH;   // 256-channel groups of heads: the unit of every kernel below
-    const BwdLayout L = bwd_layout(B, T, D, H);
+    const int H = groups_of_heads(D, q.H);   // 256-slot groups of heads: the unit of the GEMMs and of the z / dz arrays
+    const int hstride = (DH / dh) * dh;      // channels from one group to the next
+    const BwdLayout L = bwd_layout(B, T, D, q.H);
     if (ws_body_bytes < L.total) return cudaErrorInvalidValue;
     static PerDeviceOptIn opt_in;
     cudaError_t e = opt_in.ensure(tc_gemm_kernel, (int)GEMM_SMEM_ALLOC);
@@ -631,13 +653,19 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
         f.y = ws + L.off_y; f.h_T = (float *)(ws + L.off_hT); f.cs_out = ws + L.off_cs;
         f.status = status;
         char *fws = ws + L.off_fws;
-        e = sm100_prefill(f, fws + WS_HEADER_BYTES, sm100_prefill_workspace_bytes(B, T, D, H), st);
+        e = sm100_prefill(f, fws + WS_HEADER_BYTES, sm100_prefill_workspace_bytes(B, T, D, q.H), st);
         if (e != cudaSuccess) return e;
         y = f.y;
     }
 
+    if ((size_t)H * DH != (size_t)D) {
+        // Some channel slots of the groups do not exist.  Nothing writes their dz, and although their weights are zero a NaN
+        // bit pattern left in the workspace would still poison du = dz W: clear dz once.
+        if ((e = cudaMemsetAsync(dz, 0, L.BT * (size_t)H * DH * 2 * 2, st)) != cudaSuccess) return e;
+    }
+
     EwArgs a{};
-    a.B = B; a.T = T; a.D = D; a.H = H; a.nchunk = L.nchunk; a.c = q.c;
+    a.B = B; a.T = T; a.D = D; a.H = H; a.nchunk = L.nchunk; a.c = q.c; a.hstride = hstride;
     a.x = (const __nv_bfloat16 *)q.x; a.conv_w = (const __nv_bfloat16 *)q.conv_w; a.cs_in = (const __nv_bfloat16 *)q.cs_in;
     a.dy = (const __nv_bfloat16 *)q.dy; a.y = (const __nv_bfloat16 *)y;
     a.conv_b = fwd.conv_b; a.b_a = fwd.b_a; a.b_x = fwd.b_x; a.lambda = q.lambda; a.h0 = fwd.h0;
@@ -646,18 +674,18 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
     a.dh_T = q.dh_T; a.dh0 = q.dh0;
 
     // 1. W^T for the du contraction, conv output
-    convert_w_kernel<<<dim3(DH / 32, DH / 32, 2 * H), dim3(32, 8), 0, st>>>((const __nv_bfloat16 *)q.W_a, (const __nv_bfloat16 *)q.W_x, W16, WT, H, dh);
-    const dim3 grid_ew(D / 256, L.nchunk, B);
+    convert_w_kernel<<<dim3(DH / 32, DH / 32, 2 * H), dim3(32, 8), 0, st>>>((const __nv_bfloat16 *)q.W_a, (const __nv_bfloat16 *)q.W_x, W16, WT, H, dh, q.H);
+    const dim3 grid_ew((D + 255) / 256, L.nchunk, B);
     conv_forward_kernel<<<grid_ew, 256, 0, st>>>(a);
 
     GemmArgs g{};
-    g.H = H; g.D = D; g.status = status; g.spin_ns = g_spin_limit_ns;
+    g.H = H; g.D = D; g.hstride = hstride; g.cvalid = hstride; g.status = status; g.spin_ns = g_spin_limit_ns;
     const unsigned mtiles = (unsigned)((L.BT + 127) / 128);
     const uint64_t BT = L.BT;
     // 2. z = u W^T per head and gate
     {
-        const uint64_t da[3] = {DH, (uint64_t)H, BT}, sa[2] = {DH * 2, (uint64_t)D * 2};
-        const uint32_t ba[3] = {64, 1, 128};
+        const uint64_t da[3] = {(uint64_t)D, BT, 1}, sa[2] = {(uint64_t)D * 2, (uint64_t)D * BT * 2};   // u [tok][D]
+        const uint32_t ba[3] = {64, 128, 1};
         const uint64_t db[3] = {DH, DH, (uint64_t)H}, sb[2] = {DH * 2, (uint64_t)DH * DH * 2};
         const uint32_t bb[3] = {64, 256, 1};
         if (!encode_map16_3d(&g.tm_a, u, da, sa, ba, true) || !encode_map16_3d(&g.tm_b0, W16, db, sb, bb, true) ||
@@ -669,7 +697,7 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
     }
     // 3. reverse scan and element-wise adjoints
     scan_fold_kernel<<<grid_ew, 256, 0, st>>>(a);
-    scan_carry_kernel<<<dim3(D / 256, B), 256, 0, st>>>(a);
+    scan_carry_kernel<<<dim3((D + 255) / 256, B), 256, 0, st>>>(a);
     scan_apply_kernel<<<grid_ew, 256, 0, st>>>(a);
     // 4. du += dz W
     {
@@ -687,8 +715,8 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
     {
         const uint64_t da[3] = {2 * DH, (uint64_t)H, BT}, sa[2] = {2 * DH * 2, (uint64_t)H * 2 * DH * 2};   // dz [tok][h][gate, channel]
         const uint32_t ba[3] = {64, 1, 64};
-        const uint64_t db[3] = {DH, (uint64_t)H, BT}, sb[2] = {DH * 2, (uint64_t)D * 2};                     // u [tok][h][channel]
-        const uint32_t bb[3] = {64, 1, 64};
+        const uint64_t db[3] = {(uint64_t)D, BT, 1}, sb[2] = {(uint64_t)D * 2, (uint64_t)D * BT * 2};         // u [tok][D]
+        const uint32_t bb[3] = {64, 64, 1};
         if (!encode_map16_3d(&g.tm_a, dz, da, sa, ba, true) || !encode_map16_3d(&g.tm_b0, u, db, sb, bb, true)) return cudaErrorNotSupported;
         g.tm_b1 = g.tm_b0;
         float *part = (float *)(ws + L.off_pdw);
@@ -696,11 +724,11 @@ cudaError_t sm100_backward(const FwdArgs &fwd, BwdArgs &q, const void *y_saved, 
         g.nx = 4; g.ny = L.S;
         tc_gemm_kernel<<<gemm_grid(g), GEMM_THREADS, GEMM_SMEM_ALLOC, st>>>(g);
         const size_t wsz = (size_t)H * DH * DH;
-        if (dh == DH) {
+        if (dh == DH) {   // one head per group: the partial sums already have the layout of dW
             if ((e = reduce_partials3(part, L.S, 2 * wsz, q.dW_a, wsz, q.dW_x, wsz, nullptr, 0, st)) != cudaSuccess) return e;
         } else {
             const size_t nout = (size_t)2 * q.H * dh * dh;
-            reduce_dw_blocks_kernel<<<(unsigned)((nout + 255) / 256), 256, 0, st>>>(part, L.S, H, dh, q.dW_a, q.dW_x);
+            reduce_dw_blocks_kernel<<<(unsigned)((nout + 255) / 256), 256, 0, st>>>(part, L.S, H, dh, q.H, q.dW_a, q.dW_x);
         }
     }
     // 6. per-channel sums, Conv1D adjoint

@@ -263,11 +263,14 @@ def test_decode_chain_with_narrower_heads(oracle, Dh, B, H, T0, steps):
     assert not torch.equal(outs[0][1], outs[1][1])
 
 
-@pytest.mark.parametrize("Dh,B,T,H,with_y", [(128, 2, 136, 2, True), (128, 1, 264, 4, False), (64, 2, 200, 4, True), (64, 1, 72, 8, False)])
+@pytest.mark.parametrize("Dh,B,T,H,with_y", [(128, 2, 136, 2, True), (128, 1, 264, 4, False), (64, 2, 200, 4, True), (64, 1, 72, 8, False),
+                                                 (160, 2, 136, 2, True), (96, 1, 264, 3, False), (160, 1, 200, 16, True), (224, 2, 72, 1, True),
+                                                 (32, 1, 136, 5, True), (128, 2, 72, 3, True)])
 def test_backward_with_narrower_heads(oracle, Dh, B, T, H, with_y):
-    """Tensor-core backward for heads of width 128 and 64: the GEMMs run on 256-channel groups with block-diagonal weights
-    and only the diagonal blocks of the weight gradient are returned.  All gradients, the state gradients included, against
-    the oracle's analytic ones."""
+    """Tensor-core backward for heads narrower than 256 (any multiple of 32): the GEMMs run on groups of 256 channel slots with
+    block-diagonal weights and only the diagonal blocks of the weight gradient are returned; widths that do not fill the
+    256 slots, and a partial last group, leave slots that do not exist.  All gradients, the state gradients included,
+    against the oracle's analytic ones."""
     import torch
     from paper_2402_19427_b200 import binding
     D = Dh * H

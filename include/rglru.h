@@ -217,7 +217,7 @@ int32_t rglru_prefill_host(const rglru_shape_t *shape, const rglru_params_t *par
  *   - status_word: optional device pointer to a 4-byte-aligned uint32 owned by the caller, zero before the
  *     first use.  A device-side wait that runs out is recorded there, and the pointer may be given to
  *     rglru_query_status in place of a workspace.  NULL: such a condition is not reported.
- *   - Only shapes served by the tensor-core prefill (bf16 io, head width 256, or 128 / 64 with D a multiple of 256) are accepted; others return
+ *   - Only shapes served by the tensor-core prefill (bf16 io, head width a multiple of 32 up to 256) are accepted; others return
  *     RGLRU_ERR_UNSUPPORTED.  A shape whose scratch (256 bytes + rglru_workspace_bytes(shape, PREFILL))
  *     exceeds RGLRU_STATIC_SCRATCH_BYTES returns RGLRU_ERR_WORKSPACE; nothing is launched.
  *   - Every GPU on which the library is loaded holds the array until the process exits.

@@ -38,7 +38,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes per prefill launch on the bench workload (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture,
 # profiles/sm100_prefill_kernel_cfg1.md) together with the SHA-256 of the kernel source the capture was taken from:
 # the figure is reported only while the benched kernel source still has that hash, else null.
-NCU_TRAFFIC = {"bytes": 86772992 + 38842368, "kernel_sha256": "604140a06479e4db699c1a4eda30a3cbeb1e57e9f629fe2564afa3ebd99e36c7"}
+NCU_TRAFFIC = {"bytes": 86849536 + 38148608, "kernel_sha256": "1e8f4cb69ef53ec5479321ebb194ff8b7163a5ba6daf54fb5ec124bd59118fd2"}
 KERNEL_SOURCE = os.path.join(ROOT, "paper_2402_19427_b200", "csrc", "rglru_sm100.cu")
 
 

@@ -7,7 +7,8 @@ A sequence may also be split along time, rank r owning tokens [t_r, t_r + T_r). 
 rank's share of the sequence acts on the state as one step h_out = A_r h_in + b_r with A_r = prod_t a_t and b_r its final
 state from a zero start; these steps compose as (A_2 A_1, A_2 b_1 + b_2).  Two small messages per rank suffice: the last
 three raw inputs of the share (the Conv1D history of the next rank), and the pair (A_r, b_r).  Every rank then knows its
-incoming state and runs the real forward.  numpy / torch.distributed only; no arithmetic of Eq. 1-3 lives here.
+incoming state and runs the real forward (prefill_time_share).  numpy / torch.distributed only, apart from that function's
+calls into the CUDA binding; no arithmetic of Eq. 1-3 lives here.
 """
 from __future__ import annotations
 
@@ -86,3 +87,25 @@ def exchange_time_steps(a_prod, h_end, dist, h0=None):
     for r in range(rank):
         h = steps[r][:, 0] * h + steps[r][:, 1]
     return h
+
+
+def prefill_time_share(x_share, params, dist, h0=None, conv_state_in=None, c=8.0, workspace=None):
+    """This rank's share of a prefill whose sequences are split along time: rank r holds tokens [t_r, t_r + T_r) of every
+    sequence as `x_share` [B,T_r,D] on its GPU (T_r >= 3), `params` is the layer on that GPU, `h0` / `conv_state_in` are
+    the state before the first token of the whole sequence (used by rank 0's share).  Two small all-gathers and two runs
+    of the kernel: the first from a zero state, which yields the share as one affine step (prod_t a_t, h_end), the second
+    from the incoming state that the exclusive scan over the ranks' steps gives.  Rank 0 starting from a zero state needs
+    only the first run.  Returns (y [B,T_r,D], h_end [B,D], conv_state [B,3,D]); the last rank's h_end and conv_state are
+    those of the whole sequence.  Imports the CUDA binding: there is no CPU path."""
+    import torch
+    from . import binding
+    B, T_r, D = x_share.shape
+    if T_r < 3:
+        raise ValueError("every time share must hold at least three tokens")
+    hist = exchange_conv_history(x_share[:, -3:].contiguous(), dist, conv_state_in)
+    a_prod = torch.empty(B, D, dtype=torch.float32, device=x_share.device)
+    y, h_zero, cs = binding.prefill(x_share, params, conv_state_in=hist, c=c, workspace=workspace, a_prod=a_prod)
+    h_in = exchange_time_steps(a_prod, h_zero, dist, h0)
+    if dist.get_rank() == 0 and h0 is None:
+        return y, h_zero, cs
+    return binding.prefill(x_share, params, h0=h_in, conv_state_in=hist, c=c, workspace=workspace, y=y)

@@ -94,3 +94,70 @@ def test_call_as_one_affine_step_on_the_gpu(oracle):
     _, hr, _ = oracle.prefill(inp["x"].astype(np.float64), f64(inp["params"]), H, h0=inp["h0"].astype(np.float64),
                               conv_state_in=inp["conv_state"].astype(np.float64))
     assert_close("h_T", to_np(A * h0 + Bv), hr, "bf16")
+
+
+class _ThreadRanks:
+    """Stand-in for torch.distributed inside one process: every "rank" is a host thread, an all-gather is a hand-over through
+    a shared list between two host barriers.  Only the host side waits; the ranks' kernels are independent launches."""
+
+    def __init__(self, world):
+        import threading
+        self.world, self.slots, self.barrier, self.local = world, [None] * world, threading.Barrier(world), threading.local()
+
+    def get_rank(self):
+        return self.local.rank
+
+    def get_world_size(self):
+        return self.world
+
+    def all_gather(self, out_list, tensor):
+        import torch
+        torch.cuda.synchronize()
+        self.slots[self.local.rank] = tensor
+        self.barrier.wait()
+        for i in range(self.world):
+            out_list[i].copy_(self.slots[i])
+        torch.cuda.synchronize()
+        self.barrier.wait()
+
+
+@pytest.mark.parametrize("world,with_state", [(2, True), (3, False)])
+def test_time_shares_on_the_gpu_equal_the_uncut_prefill(oracle, world, with_state):
+    """sharding.prefill_time_share, the GPU path of a prefill cut along time, run by `world` host threads that stand for the
+    ranks (one GPU here): Conv1D history and affine steps are exchanged, every share is then computed from its true incoming
+    state, and the concatenation matches the oracle's uncut prefill; the last share ends in the final state."""
+    import threading
+    import torch
+    from paper_2402_19427_b200 import binding, sharding
+    B, T, D, H = 2, 450, 512, 2
+    inp = synth.make_inputs(B, T, D, H, io="bf16", seed=41, with_state=True, bias_scale=0.3)
+    params = binding.Params.from_numpy(inp["params"], "bf16")
+    x = to_dev(inp["x"], "bf16")
+    h0 = to_dev(inp["h0"]) if with_state else None
+    cs = to_dev(inp["conv_state"], "bf16") if with_state else None
+    ranks = _ThreadRanks(world)
+    out, errs = [None] * world, []
+
+    def run(r):
+        try:
+            ranks.local.rank = r
+            torch.cuda.set_device(0)
+            t0, tc = sharding.split_range(T, world, r)
+            out[r] = sharding.prefill_time_share(x[:, t0:t0 + tc].contiguous(), params, ranks, h0=h0, conv_state_in=cs)
+            torch.cuda.synchronize()
+        except Exception as e:   # noqa: BLE001
+            errs.append(e)
+            ranks.barrier.abort()
+
+    threads = [threading.Thread(target=run, args=(r,)) for r in range(world)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errs, errs
+    yr, hr, cr = oracle.prefill(inp["x"].astype(np.float64), f64(inp["params"]), H, c=inp["c"],
+                                h0=inp["h0"].astype(np.float64) if with_state else None,
+                                conv_state_in=inp["conv_state"].astype(np.float64) if with_state else None)
+    assert_close("y", np.concatenate([to_np(o[0]) for o in out], 1), yr, "bf16")
+    assert_close("h_T", to_np(out[-1][1]), hr, "bf16")
+    assert np.array_equal(to_np(out[-1][2]), cr)

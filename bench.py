@@ -116,10 +116,14 @@ def graph_times_us(fn, calls, reps, torch):
     return [t / calls for t in event_times_us(graph.replay, reps, torch)]
 
 
-def time_prefill_config(binding, dev, index, peaks, peak_kind, reps=20):
-    """One of the other prefill shapes as a side record: `reps` launches over rotating buffer sets, median and min."""
+def time_prefill_config(binding, dev, index, peaks, peak_kind, reps=20, heads=None, merged=False):
+    """One of the other prefill shapes as a side record: `reps` launches over rotating buffer sets, median and min.  `heads`
+    overrides the head count of the config (the paper's 16 blocks); `merged` adds the gate branch of the recurrent block
+    (y = h GeLU(branch), one more bf16 read per element) and the decay-product output."""
     import torch
     cfg = dict(synth.CONFIGS[index])
+    if heads is not None:
+        cfg["H"] = heads
     B, T, D, H = cfg["B"], cfg["T"], cfg["D"], cfg["H"]
     dt = torch.bfloat16
     pr = synth.make_inputs(1, 4, D, H, io="bf16", seed=synth.BASE_SEED + index)["params"]
@@ -132,9 +136,12 @@ def time_prefill_config(binding, dev, index, peaks, peak_kind, reps=20):
     ws = binding.alloc_workspace(shape, binding.OP_PREFILL, dev)
     hT = torch.empty(B, D, dtype=torch.float32, device=dev)
     cso = torch.empty(B, 3, D, dtype=dt, device=dev)
+    gbs = [torch.randn(B, T, D, device=dev, generator=g).to(dt) for _ in range(nset)] if merged else None
+    ap = torch.empty(B, D, dtype=torch.float32, device=dev) if merged else None
 
     def one(i):
-        binding.prefill(xs[i % nset], params, y=ys[i % nset], h_T=hT, conv_state_out=cso, workspace=ws)
+        binding.prefill(xs[i % nset], params, y=ys[i % nset], h_T=hT, conv_state_out=cso, workspace=ws,
+                        gate_branch=gbs[i % nset] if merged else None, a_prod=ap)
 
     for i in range(3):
         one(i)
@@ -144,8 +151,10 @@ def time_prefill_config(binding, dev, index, peaks, peak_kind, reps=20):
     if status != binding.OK:
         raise binding.RglruError(status, "device status after the side measurement")
     nbytes, flops = algorithmic_work(cfg)
+    if merged:
+        nbytes += B * T * D * 2 + B * D * 4
     med = float(np.median(us))
-    return {"workload": workload_name(cfg), "us_median": med, "us_min": float(np.min(us)), "reps": reps,
+    return {"workload": workload_name(cfg) + (" + gate branch (GeLU merge) and decay product" if merged else ""), "us_median": med, "us_min": float(np.min(us)), "reps": reps,
             "launch": f"{2 * nset} calls per CUDA-graph replay",
             "tokens_per_s": B * T / (med * 1e-6), "buffer_sets": nset, "roofline": roofline(nbytes, flops, med * 1e-6, peaks, peak_kind)}
 
@@ -398,6 +407,9 @@ def run_ours(args):
         # the other prefill shapes: the long sequence (every tile through the decoupled look-back) and the training shape of config 4
         extra["prefill_long"] = time_prefill_config(binding, dev, 2, peaks, peak_kind)
         extra["prefill_cfg4_forward"] = time_prefill_config(binding, dev, 4, peaks, peak_kind)
+        # the bench shape with the paper's 16 blocks (head width 160, one head per 256 channel slots), and with the merged output
+        extra["prefill_16_blocks"] = time_prefill_config(binding, dev, WORKLOAD, peaks, peak_kind, heads=16)
+        extra["prefill_gelu_merge"] = time_prefill_config(binding, dev, WORKLOAD, peaks, peak_kind, merged=True)
         extra.update(measure_extras(binding, dev, peaks))
 
     if rank == 0:
